@@ -1,0 +1,274 @@
+"""Pins of the CPU oracle against things other than itself: hand-computed examples of
+Eq. 4, dot products and box sums a person can verify, float64 cross-correlation from a
+library routine, exact rational arithmetic, library pooling, and the invariants the paper
+states (outputs inside [0, max_int], h_i requantises to max_int, concatenation and
+addition operands share one ratio)."""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+from scipy import signal
+
+from oracle import layers as L
+from oracle import planner as P
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+ONE = ([1], [0], [0])   # mul, shift, h_i of an identity requantisation
+
+
+def _examples():
+    rows = []
+    with open(os.path.join(GOLDEN, "round_shift_examples.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if len(line) == 4:
+                rows.append(tuple(int(v) for v in line))
+    return rows
+
+
+# ---------------------------------------------------------------- Eq. 4 bracket
+def test_round_shift_hand_examples():
+    rows = _examples()
+    assert len(rows) >= 20
+    for Y, mul, shift, V in rows:
+        assert L.round_shift(Y * mul, shift) == V, (Y, mul, shift)
+
+
+def test_round_shift_equals_exact_rational_rounding():
+    rng = np.random.default_rng(7)
+    for _ in range(2000):
+        v = int(rng.integers(-2 ** 40, 2 ** 40))
+        s = int(rng.integers(0, 41))
+        exact = P.round_half_up(Fraction(v, 1 << s))
+        assert L.round_shift(v, s) == exact
+        if s:
+            assert exact == (v + (1 << (s - 1))) >> s     # python ints: floor shift
+
+
+def test_layer_applies_hand_examples_through_the_whole_tail():
+    """1x1 kernel with weight 1 and C_in = 1: Y = x + b, so the layer output must be the
+    golden V for Y reachable with an 8-bit x and an int32 bias."""
+    for Y, mul, shift, V in _examples():
+        x = np.array([[[[7]]]], dtype=np.uint8)
+        W = np.ones((1, 1, 1, 1), dtype=np.int8)
+        out, ovf = L.conv(x, W, [Y - 7], [mul], [shift], [2 ** 31 - 1], out_dtype=L.S8,
+                          brelu=False, out_lo=-128, out_hi=127)
+        assert not ovf
+        assert int(out[0, 0, 0, 0]) == max(-128, min(127, V))
+
+
+# ---------------------------------------------------------------- hand-checkable layers
+def test_single_pixel_dot_product():
+    x = np.array([[[[3, 0, 255, 17]]]], dtype=np.uint8)
+    W = np.array([[[[2, -5, 1, -1]]], [[[-127, 127, 0, 4]]]], dtype=np.int8)
+    b = np.array([10, -20], dtype=np.int32)
+    # 3*2 + 255 - 17 + 10 = 254 ;  -381 + 68 - 20 = -333
+    out, _ = L.conv(x, W, b, *ONE, out_dtype=L.I32, brelu=False)
+    assert out.reshape(-1).tolist() == [254, -333]
+    # BReLU to [0, 200], then *3/4 rounded half up: 200*3/4 = 150 ; 0
+    out, _ = L.conv(x, W, b, [3], [2], [200])
+    assert out.reshape(-1).tolist() == [150, 0]
+    # raw-128 input: (3-128)*2 + (255-128) - (17-128) + 640 + 10 = 638 ... (0-128)*-5 = 640
+    out, _ = L.conv(x, W, b, *ONE, in_dtype=L.U8_RAW128, out_dtype=L.I32, brelu=False)
+    assert int(out[0, 0, 0, 0]) == (3 - 128) * 2 + (0 - 128) * -5 + (255 - 128) - (17 - 128) + 10
+
+
+def test_one_hot_kernel_shifts_and_ones_kernel_box_sums():
+    rng = np.random.default_rng(3)
+    x = rng.integers(0, 256, size=(1, 3, 3, 1), dtype=np.uint8)
+    for r in range(3):
+        for s in range(3):
+            W = np.zeros((1, 3, 3, 1), dtype=np.int8)
+            W[0, r, s, 0] = 1
+            out, _ = L.conv(x, W, [0], *ONE, pad=1, out_dtype=L.I32, brelu=False)
+            padded = np.zeros((5, 5), dtype=np.int64)
+            padded[1:4, 1:4] = x[0, :, :, 0]
+            assert np.array_equal(out[0, :, :, 0], padded[r:r + 3, s:s + 3])
+    W = np.ones((1, 3, 3, 1), dtype=np.int8)
+    out, _ = L.conv(x, W, [0], *ONE, pad=1, out_dtype=L.I32, brelu=False)
+    xi = x[0, :, :, 0].astype(np.int64)
+    assert int(out[0, 1, 1, 0]) == xi.sum()
+    assert int(out[0, 0, 0, 0]) == xi[:2, :2].sum()
+    assert int(out[0, 2, 1, 0]) == xi[1:, :].sum()
+    # raw-128 input: padding is zero AFTER the re-normalisation, so a corner sums four values
+    out, _ = L.conv(x, W, [0], *ONE, pad=1, in_dtype=L.U8_RAW128, out_dtype=L.I32, brelu=False)
+    assert int(out[0, 0, 0, 0]) == (xi[:2, :2] - 128).sum()
+
+
+# ---------------------------------------------------------------- library cross-correlation
+def _xcorr_f64(xv, W, stride, pad):
+    """float64 cross-correlation of integer values with scipy (exact below 2^53)."""
+    n, h, w, c = xv.shape
+    co, kh, kw, _ = W.shape
+    xp = np.zeros((n, h + 2 * pad, w + 2 * pad, c), dtype=np.float64)
+    xp[:, pad:pad + h, pad:pad + w, :] = xv
+    full_h, full_w = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    out = np.zeros((n, full_h, full_w, co))
+    for i in range(n):
+        for o in range(co):
+            for ch in range(c):
+                out[i, :, :, o] += signal.correlate2d(xp[i, :, :, ch], W[o, :, :, ch].astype(np.float64), mode="valid")
+    return out[:, ::stride, ::stride, :]
+
+
+@pytest.mark.parametrize("k,stride,pad,c_in,c_out,h,w", [
+    (1, 1, 0, 16, 5, 5, 7), (3, 1, 1, 3, 4, 6, 5), (3, 2, 1, 16, 3, 7, 9), (5, 1, 2, 1, 6, 8, 6),
+    (5, 2, 0, 3, 2, 9, 9), (7, 2, 3, 3, 4, 11, 10), (3, 1, 0, 48, 2, 5, 5), (3, 2, 2, 64, 3, 6, 7),
+    (1, 2, 0, 16, 4, 6, 6), (7, 1, 3, 1, 2, 7, 7), (3, 1, 3, 2, 2, 4, 4),
+])
+@pytest.mark.parametrize("in_dtype", [L.U8, L.U8_RAW128, L.S8])
+def test_plain_integer_convolution_equals_float64_cross_correlation(k, stride, pad, c_in, c_out, h, w, in_dtype):
+    rng = np.random.default_rng(k * 100 + stride * 10 + pad + c_in)
+    if in_dtype == L.S8:
+        x = rng.integers(-128, 128, size=(2, h, w, c_in), dtype=np.int8)
+        xv = x.astype(np.float64)
+    else:
+        x = rng.integers(0, 256, size=(2, h, w, c_in), dtype=np.uint8)
+        xv = x.astype(np.float64) - (128 if in_dtype == L.U8_RAW128 else 0)
+    W = rng.integers(-127, 128, size=(c_out, k, k, c_in), dtype=np.int8)
+    b = rng.integers(-4096, 4097, size=(c_out,), dtype=np.int32)
+    out, ovf = L.conv(x, W, b, *ONE, stride=stride, pad=pad, in_dtype=in_dtype, out_dtype=L.I32,
+                      brelu=False, check_partial=True)
+    assert not ovf
+    ref = _xcorr_f64(xv, W, stride, pad) + b.astype(np.float64)
+    assert out.shape == ref.shape
+    assert np.array_equal(out.astype(np.float64), ref)
+
+
+def test_tail_matches_exact_rationals_on_a_random_layer():
+    rng = np.random.default_rng(11)
+    x = rng.integers(0, 256, size=(1, 6, 6, 16), dtype=np.uint8)
+    W = rng.integers(-127, 128, size=(8, 3, 3, 16), dtype=np.int8)
+    b = rng.integers(-4096, 4097, size=(8,), dtype=np.int32)
+    mul = rng.integers(100, 400, size=8).astype(np.int32)
+    shift = rng.integers(14, 18, size=8).astype(np.int32)
+    h_i = rng.integers(20000, 90000, size=8).astype(np.int32)
+    Y = _xcorr_f64(x.astype(np.float64), W, 1, 1) + b
+    out, _ = L.conv(x, W, b, mul, shift, h_i, pad=1)           # per-channel parameters
+    for idx in np.ndindex(*Y.shape):
+        co = idx[3]
+        y = min(max(int(Y[idx]), 0), int(h_i[co]))
+        v = P.round_half_up(Fraction(y * int(mul[co]), 1 << int(shift[co])))
+        assert int(out[idx]) == min(max(v, 0), 255)
+
+
+# ---------------------------------------------------------------- invariants
+def test_outputs_stay_in_range_and_requant_is_monotone():
+    rng = np.random.default_rng(5)
+    q = P.brelu_params(6.0, 24498.7, 255)
+    assert L.round_shift(q["h_i"] * q["mul"], q["shift"]) == 255
+    ys = np.sort(rng.integers(-10 ** 6, 10 ** 6, size=500))
+    prev = -1
+    for y in ys:
+        yc = min(max(int(y), 0), q["h_i"])
+        v = L.round_shift(yc * q["mul"], q["shift"])
+        assert 0 <= v <= 255 and v >= prev
+        prev = v
+
+
+def test_mul_shift_scaling_and_bias_linearity():
+    rng = np.random.default_rng(6)
+    x = rng.integers(0, 256, size=(1, 5, 5, 16), dtype=np.uint8)
+    W = rng.integers(-127, 128, size=(4, 3, 3, 16), dtype=np.int8)
+    b = rng.integers(-4096, 4097, size=(4,), dtype=np.int32)
+    a, _ = L.conv(x, W, b, [200], [16], [80000], pad=1)
+    c, _ = L.conv(x, W, b, [400], [17], [80000], pad=1)
+    assert np.array_equal(a, c)                     # doubling mul and adding 1 to shift
+    # adding c * 2^shift / mul (integral) to the bias adds c to the unclamped output
+    u0, _ = L.conv(x, W, b, [256], [16], [0], pad=1, brelu=False, out_dtype=L.S8, out_lo=-128, out_hi=127,
+                   out_zero=0)
+    u1, _ = L.conv(x, W, b + 3 * 256, [256], [16], [0], pad=1, brelu=False, out_dtype=L.S8, out_lo=-128,
+                   out_hi=127)
+    inside = (u0.astype(int) > -120) & (u0.astype(int) < 120)
+    assert inside.any()
+    assert np.array_equal(u1.astype(int)[inside], u0.astype(int)[inside] + 3)
+
+
+def test_clamp_then_requant_equals_requant_then_clamp_when_h_i_maps_to_max_int():
+    q = P.brelu_params_from_h_ri(146992, 1.0, 255)
+    for y in list(range(-5, 5)) + list(range(q["h_i"] - 2000, q["h_i"] + 2000, 7)):
+        pre = L.round_shift(min(max(y, 0), q["h_i"]) * q["mul"], q["shift"])
+        post = min(max(L.round_shift(y * q["mul"], q["shift"]), 0), 255)
+        assert pre == post
+
+
+def test_concat_through_channel_offsets_equals_host_concatenation():
+    rng = np.random.default_rng(8)
+    x = rng.integers(0, 256, size=(2, 6, 7, 64), dtype=np.uint8)
+    Wa = rng.integers(-127, 128, size=(16, 5, 5, 64), dtype=np.int8)
+    Wb = rng.integers(-127, 128, size=(32, 3, 3, 64), dtype=np.int8)
+    ba = rng.integers(-4096, 4097, size=(16,), dtype=np.int32)
+    bb = rng.integers(-4096, 4097, size=(32,), dtype=np.int32)
+    cat = np.full((2, 6, 7, 48), 77, dtype=np.uint8)
+    L.conv(x, Wa, ba, [130], [17], [257103], pad=2, out=cat, out_c_offset=0)
+    L.conv(x, Wb, bb, [136], [17], [245760], pad=1, out=cat, out_c_offset=16)
+    a, _ = L.conv(x, Wa, ba, [130], [17], [257103], pad=2)
+    b, _ = L.conv(x, Wb, bb, [136], [17], [245760], pad=1)
+    assert np.array_equal(cat, np.concatenate([a, b], axis=3))
+    # reading a channel slice of the concatenated tensor
+    Wc = rng.integers(-127, 128, size=(4, 3, 3, 32), dtype=np.int8)
+    s1, _ = L.conv(cat, Wc, [0] * 4, *ONE, pad=1, in_c_offset=16, c_in=32, out_dtype=L.I32, brelu=False)
+    s2, _ = L.conv(np.ascontiguousarray(cat[..., 16:48]), Wc, [0] * 4, *ONE, pad=1, out_dtype=L.I32, brelu=False)
+    assert np.array_equal(s1, s2)
+
+
+def test_fused_skip_equals_raw_convolution_followed_by_add_requant():
+    rng = np.random.default_rng(9)
+    x = rng.integers(0, 256, size=(2, 5, 6, 16), dtype=np.uint8)
+    W = rng.integers(-127, 128, size=(32, 1, 1, 16), dtype=np.int8)
+    b = rng.integers(-4096, 4097, size=(32,), dtype=np.int32)
+    for skip_dtype, lo, hi, zero in ((L.U8, 0, 256, 0), (L.I32, -200000, 200000, 0), (L.U8_RAW128, 0, 256, 128)):
+        npdt = np.int32 if skip_dtype == L.I32 else np.uint8
+        S = rng.integers(lo, hi, size=(2, 5, 6, 32)).astype(npdt)
+        fused, _ = L.conv(x, W, b, [150], [17], [220000], skip=S, skip_dtype=skip_dtype, skip_mul=811, skip_shift=3)
+        Y, _ = L.conv(x, W, b, *ONE, out_dtype=L.I32, brelu=False)
+        two, _ = L.add_requant(S, Y, a_dtype=L.U8 if skip_dtype != L.I32 else L.I32, b_dtype=L.I32, a_zero=zero,
+                               mul_a=811, sh_a=3, mul_b=1, sh_b=0, brelu=True, h_i=220000, mul=150, shift=17)
+        assert np.array_equal(fused, two)
+        # and against exact rationals on a few elements
+        for idx in [(0, 0, 0, 0), (1, 4, 5, 31), (0, 2, 3, 7)]:
+            s = int(S[idx]) - zero
+            y = int(Y[idx]) + P.round_half_up(Fraction(s * 811, 8))
+            v = P.round_half_up(Fraction(min(max(y, 0), 220000) * 150, 1 << 17))
+            assert int(fused[idx]) == min(max(v, 0), 255)
+
+
+def test_overflow_is_reported():
+    x = np.full((1, 8, 8, 64), 255, dtype=np.uint8)
+    W = np.full((1, 7, 7, 64), 127, dtype=np.int8)
+    _, ovf = L.conv(x, W, [2 ** 31 - 1 - 255 * 127 * 64 * 49 + 100], *ONE, pad=3, out_dtype=L.I32, brelu=False)
+    assert ovf
+    _, ovf = L.conv(x, W, [0], *ONE, pad=3, out_dtype=L.I32, brelu=False, check_partial=True)
+    assert not ovf
+    # partial sums can overflow while the final sum does not: + then - of large products
+    x2 = np.full((1, 1, 1, 2 * 70000), 255, dtype=np.uint8)
+    W2 = np.concatenate([np.full(70000, 127), np.full(70000, -127)]).astype(np.int8).reshape(1, 1, 1, -1)
+    _, ovf = L.conv(x2, W2, [0], *ONE, out_dtype=L.I32, brelu=False)
+    assert not ovf
+    _, ovf = L.conv(x2, W2, [0], *ONE, out_dtype=L.I32, brelu=False, check_partial=True)
+    assert ovf
+
+
+# ---------------------------------------------------------------- pooling
+def test_maxpool_equals_library_maxpool():
+    rng = np.random.default_rng(10)
+    for (h, w, k, s, p) in [(9, 11, 3, 2, 1), (8, 8, 3, 2, 1), (7, 5, 2, 2, 0), (6, 6, 3, 1, 1)]:
+        x = rng.integers(0, 256, size=(2, h, w, 5), dtype=np.uint8)
+        ref = torch.nn.functional.max_pool2d(torch.from_numpy(x.astype(np.float32)).permute(0, 3, 1, 2), k, s, p)
+        got = L.maxpool(x, k, s, p)
+        assert np.array_equal(got, ref.permute(0, 2, 3, 1).numpy().astype(np.uint8))
+
+
+def test_avgpool_is_rounded_exact_mean():
+    rng = np.random.default_rng(12)
+    x = rng.integers(0, 256, size=(3, 7, 7, 9), dtype=np.uint8)
+    m, s = P.avgpool_mul_shift(49)
+    assert (m, s) == (1337, 16)           # 65536/49 = 1337.47
+    got = L.avgpool_requant(x, m, s)
+    for n in range(3):
+        for c in range(9):
+            tot = int(x[n, :, :, c].astype(np.int64).sum())
+            assert int(got[n, 0, 0, c]) == min(255, P.round_half_up(Fraction(tot * m, 1 << s)))
+            assert abs(int(got[n, 0, 0, c]) - tot / 49.0) <= 1.0
