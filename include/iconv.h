@@ -1,0 +1,181 @@
+/*
+ * iconv.h -- C ABI of the B200 (sm_100a) integer-arithmetic-only convolution layer.
+ *
+ * The operations are those of "Efficient Integer-Arithmetic-Only Convolutional Neural
+ * Networks" (Zhao, Liu, Li).  One layer (Section 3.1, Figure 1, integer branch):
+ *
+ *     U_i = X_i (*) W_i            int8 weights x 8-bit activations, int32 accumulation
+ *     Y_i = U_i + b_i              int32 bias
+ *     Y_i += [S * skip_mul / 2^skip_shift]      residual ratio synchronisation (Section 4.1)
+ *     Y_i = min(max(Y_i, 0), h_i)  Bounded ReLU with l = 0 (Eq. 5, Section 3.3)
+ *     V_i = [Y_i * mul / 2^shift]  requantisation (Eq. 4)
+ *     out = clamp(V_i + out_zero, out_lo, out_hi), stored at a channel offset
+ *                                  (concatenation without a copy, Section 4.2.2)
+ *
+ * "[.]" is round-to-nearest with ties toward +infinity: [v / 2^s] = floor((v + 2^(s-1)) / 2^s).
+ *
+ * Conventions for every entry point
+ *   - Plain C, no exceptions cross the boundary.  Every function returns an iconv_status
+ *     (0 = success, negative = error); iconv_last_error() gives the text of the calling
+ *     thread's last error.  Nothing falls back to the CPU or to a vendor library.
+ *   - "host" / "device" on a pointer says where the memory lives.  Device pointers must be
+ *     16-byte aligned unless stated otherwise.
+ *   - Activations are NHWC.  A tensor may be a channel slice of a wider tensor: the pixel
+ *     stride is *_c_total channels and the slice starts at *_c_offset.
+ *   - Weights are [c_out][kh][kw][c_in] int8.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Forward calls only enqueue work on it and return; they never synchronise.
+ */
+#ifndef ICONV_H_
+#define ICONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ICONV_API __attribute__((visibility("default")))
+#else
+#define ICONV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ICONV_OK = 0,
+    ICONV_ERR_ARG = -1,          /* null pointer, bad enum, negative size */
+    ICONV_ERR_SHAPE = -2,        /* empty output, slice outside its tensor */
+    ICONV_ERR_ALIGN = -3,        /* pointer or channel offset not aligned as required */
+    ICONV_ERR_OVERFLOW = -4,     /* worst-case |Y| could exceed int32 */
+    ICONV_ERR_UNSUPPORTED = -5,  /* valid request that no kernel implements */
+    ICONV_ERR_CUDA = -6,         /* a CUDA call failed; text in iconv_last_error() */
+    ICONV_ERR_TIMEOUT = -7       /* a bounded device-side wait ran out (reported by iconv_check) */
+} iconv_status;
+
+typedef enum {
+    ICONV_U8 = 0,        /* unsigned 8-bit activation */
+    ICONV_S8 = 1,        /* signed 8-bit activation */
+    ICONV_I32 = 2,       /* raw int32 Y (projection skips, logits) */
+    ICONV_U8_RAW128 = 3  /* raw uint8 image; 128 is subtracted on load (Section 3.4.1).
+                            Padding is zero AFTER the subtraction. */
+} iconv_dtype;
+
+/* Kernel families; ICONV_KERNEL_AUTO lets the plan choose. */
+typedef enum {
+    ICONV_KERNEL_AUTO = 0,
+    ICONV_KERNEL_DIRECT = 1,   /* CUDA-core direct convolution, any shape */
+    ICONV_KERNEL_UMMA = 2,     /* tcgen05.mma kind::i8 implicit GEMM, TMA im2col staging */
+    ICONV_KERNEL_THIN = 3      /* bandwidth-bound layers: c_in <= 4 or c_out == 1 */
+} iconv_kernel;
+
+/*
+ * Layer descriptor.  All pointers are HOST pointers; iconv_plan copies what they point
+ * to, so the caller may free them after the call.
+ */
+typedef struct {
+    int32_t n, h, w, c_in;             /* input extent (c_in = width of the slice convolved) */
+    int32_t c_out, kh, kw, stride, pad;
+    int32_t in_dtype, in_c_total, in_c_offset;      /* ICONV_U8 | ICONV_S8 | ICONV_U8_RAW128 */
+    int32_t out_dtype, out_c_total, out_c_offset;   /* ICONV_U8 | ICONV_S8 | ICONV_I32 (raw Y) */
+    int32_t brelu;                     /* 1: clamp Y to [0, h_i] before Eq. 4 */
+    int32_t per_channel;               /* 0: mul/shift/h_i hold 1 entry; 1: c_out entries */
+    int32_t out_lo, out_hi, out_zero;  /* final saturation and zero point of the stored value */
+    int32_t skip_dtype;                /* -1: none, else an iconv_dtype */
+    int32_t skip_c_total, skip_c_offset;
+    int32_t skip_mul, skip_shift;      /* Y += [ (S - 128 if RAW128) * skip_mul / 2^skip_shift ] */
+    int32_t kernel;                    /* iconv_kernel; AUTO unless a test forces a family */
+    const int8_t *weights;             /* host [c_out][kh][kw][c_in] */
+    const int32_t *bias;               /* host [c_out] */
+    const int32_t *mul;                /* host [1 or c_out], 1 <= mul < 2^31 (ignored for I32 out) */
+    const int32_t *shift;              /* host [1 or c_out], 0 <= shift <= 40 */
+    const int32_t *h_i;                /* host [1 or c_out], 0 <= h_i (ignored unless brelu) */
+} iconv_desc;
+
+typedef struct iconv_plan_s iconv_plan_t;
+
+/*
+ * iconv_plan -- validate a layer, choose its kernel, upload its parameters (Section 3.1's
+ * W_i, b_i; Eq. 4's mul, shift; Section 3.3's h_i) and build its TMA descriptors.
+ * Allocates device memory with cudaMalloc on the current device; call it outside any
+ * stream capture.  Rejects layers whose worst-case |Y| (c_in*kh*kw * 255 * 127 + |b| +
+ * skip bound) reaches 2^31 with ICONV_ERR_OVERFLOW.  *plan_out is owned by the caller
+ * and released with iconv_plan_destroy.
+ */
+ICONV_API int iconv_plan(const iconv_desc *desc, iconv_plan_t **plan_out);
+ICONV_API int iconv_plan_destroy(iconv_plan_t *plan);
+
+/* Which kernel family the plan selected (an iconv_kernel), or a negative status. */
+ICONV_API int iconv_plan_kernel(const iconv_plan_t *plan);
+
+/*
+ * iconv_forward -- one layer forward (Section 3.1 / Eq. 4 / Eq. 5 as listed at the top).
+ * x, skip, out: DEVICE pointers owned by the caller.  x holds n*h*w*in_c_total elements
+ * of in_dtype; out holds n*h_out*w_out*out_c_total elements of out_dtype, of which only
+ * the slice [out_c_offset, out_c_offset + c_out) of each pixel is written; skip (NULL when
+ * skip_dtype < 0) holds n*h_out*w_out*skip_c_total elements.  Asynchronous on cuda_stream.
+ * The plan is not modified: concurrent forwards on different streams are allowed.
+ */
+ICONV_API int iconv_forward(const iconv_plan_t *plan, const void *x, const void *skip, void *out,
+                  void *cuda_stream);
+
+/*
+ * Device-side waits (mbarrier phases) are bounded.  A kernel whose wait runs out records
+ * it in a per-device status word and returns early.  iconv_check synchronises the stream
+ * and returns ICONV_ERR_TIMEOUT if any kernel recorded one since the last call,
+ * ICONV_ERR_CUDA on a CUDA error, ICONV_OK otherwise.
+ */
+ICONV_API int iconv_check(void *cuda_stream);
+
+/* Feature-map addition with ratio synchronisation as a stand-alone step (Sections 3.4.2,
+ * 4.1):  Y = [(A - a_zero) * mul_a / 2^sh_a] + [(B - b_zero) * mul_b / 2^sh_b], then the
+ * same BReLU / Eq. 4 / zero point / saturation tail as a convolution output. */
+typedef struct {
+    int64_t n_elems;
+    int32_t a_dtype, b_dtype, out_dtype;     /* ICONV_U8 | ICONV_S8 | ICONV_I32 */
+    int32_t a_zero, b_zero;
+    int32_t mul_a, sh_a, mul_b, sh_b;        /* (1, 0) for an operand already at the target ratio */
+    int32_t brelu, h_i, mul, shift, out_zero, out_lo, out_hi;
+} iadd_desc;
+
+/* a, b, out: DEVICE pointers to n_elems contiguous elements.  Asynchronous. */
+ICONV_API int iadd_requant(const iadd_desc *desc, const void *a, const void *b, void *out, void *cuda_stream);
+
+/* ResNet glue (Section 4.1 only says that pooling layers exist; a maximum needs no
+ * rescaling, the average is an integer sum followed by Eq. 4 with mul ~ 2^shift / (h*w)).
+ * x, out: DEVICE, uint8 NHWC, contiguous.  c must be a multiple of 16 for ipool_max. */
+ICONV_API int ipool_max(const void *x, void *out, int32_t n, int32_t h, int32_t w, int32_t c,
+              int32_t k, int32_t stride, int32_t pad, void *cuda_stream);
+ICONV_API int ipool_avg_requant(const void *x, void *out, int32_t n, int32_t h, int32_t w, int32_t c,
+                      int32_t mul, int32_t shift, int32_t max_int, void *cuda_stream);
+
+/* ---- host-side parameter arithmetic (no GPU involved) ------------------------------- */
+
+/* Eq. 2: delta = max|W_f| / 127. */
+ICONV_API int iq_weight_delta(const float *w_f, int64_t count, double *delta);
+/* Eq. 1: w_i = clamp([w_f / delta], -127, 127), computed in double. */
+ICONV_API int iq_quantize_weights(const float *w_f, int64_t count, double delta, int8_t *w_i);
+/* The mul_shift() named by Eq. 9: the smallest shift in [shift_min, 40] whose
+ * mul = [r * 2^shift] reaches 2^6; fails with ICONV_ERR_ARG unless 1 <= mul < 2^31. */
+ICONV_API int iq_mul_shift(double r, int32_t shift_min, int32_t *mul, int32_t *shift);
+/* Section 3.3, Eq. 7-13: from h_rf and ratio_Y to mul, shift, h_i (and h_f, ratio_V). */
+ICONV_API int iq_brelu_params(double h_rf, double ratio_y, int32_t max_int, int32_t shift_min,
+                    int32_t *h_ri, int32_t *mul, int32_t *shift, int32_t *h_i,
+                    double *h_f, double *ratio_v);
+/* Section 4.1: rescale of a skip operand of ratio_s toward ratio_y, and the factor by
+ * which the convolution's quantisation step moves so that both ratios agree exactly. */
+ICONV_API int iq_skip_sync(double ratio_y, double ratio_s, int32_t shift_min,
+                 int32_t *skip_mul, int32_t *skip_shift, double *ratio_y_new, double *delta_scale);
+/* Algorithm 2: ratio synchronisation of n_branches concatenated feature maps.  Outputs are
+ * host arrays of n_branches entries; *ratio_v_min receives the common ratio. */
+ICONV_API int iconcat_plan(int32_t n_branches, const double *ratio_y, const double *ratio_v,
+                 int32_t shift_min, int32_t *mul, int32_t *shift,
+                 double *delta_scale, double *ratio_y_new, double *ratio_v_min);
+
+/* Text of the calling thread's last error (never NULL; valid until its next failing call). */
+ICONV_API const char *iconv_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ICONV_H_ */

@@ -58,7 +58,7 @@ def mul_shift(r, shift_min: int = 16, mul_min: int = MUL_MIN):
 
 def brelu_params(h_rf: float, ratio_Y: float, max_int: int, shift_min: int = 16):
     """Section 3.3.  Returns dict(h_ri, mul, shift, ratio_V, h_f, h_i)."""
-    h_ri = max(1, round_half_up(Fraction(h_rf) * Fraction(ratio_Y)))          # Eq. 8
+    h_ri = max(1, round_half_up(float(h_rf) * float(ratio_Y)))                # Eq. 8 (double product)
     return brelu_params_from_h_ri(h_ri, ratio_Y, max_int, shift_min)
 
 

@@ -1,0 +1,193 @@
+"""ctypes binding of ``libiconv_b200.so``: the same names as ``include/iconv.h``, argument
+marshalling only.  Tensors are passed as raw device addresses (``torch.Tensor.data_ptr()``)
+and streams as raw ``cudaStream_t`` handles."""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libiconv_b200.so")
+
+OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_OVERFLOW, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
+U8, S8, I32, U8_RAW128 = 0, 1, 2, 3
+KERNEL_AUTO, KERNEL_DIRECT, KERNEL_UMMA, KERNEL_THIN = 0, 1, 2, 3
+DTYPE_CODE = {"u8": U8, "s8": S8, "i32": I32, "u8_raw128": U8_RAW128}
+KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin"}
+
+EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_forward", "iconv_check",
+           "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
+           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iconcat_plan", "iconv_last_error")
+
+
+class IconvError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__("iconv status %d: %s" % (status, text))
+        self.status = status
+
+
+class iconv_desc(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in (
+        "n", "h", "w", "c_in", "c_out", "kh", "kw", "stride", "pad",
+        "in_dtype", "in_c_total", "in_c_offset", "out_dtype", "out_c_total", "out_c_offset",
+        "brelu", "per_channel", "out_lo", "out_hi", "out_zero",
+        "skip_dtype", "skip_c_total", "skip_c_offset", "skip_mul", "skip_shift", "kernel")] + [
+        ("weights", C.c_void_p), ("bias", C.c_void_p), ("mul", C.c_void_p), ("shift", C.c_void_p),
+        ("h_i", C.c_void_p)]
+
+
+class iadd_desc(C.Structure):
+    _fields_ = [("n_elems", C.c_int64)] + [(k, C.c_int32) for k in (
+        "a_dtype", "b_dtype", "out_dtype", "a_zero", "b_zero", "mul_a", "sh_a", "mul_b", "sh_b",
+        "brelu", "h_i", "mul", "shift", "out_zero", "out_lo", "out_hi")]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("%s is missing: build it with `python -m paper_2006_11735_b200.build` "
+                          "(there is no fallback path)" % LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, dbl = C.c_void_p, C.c_int32, C.c_int64, C.c_double
+    P = C.POINTER
+    lib.iconv_plan.argtypes = [P(iconv_desc), P(vp)]
+    lib.iconv_plan_destroy.argtypes = [vp]
+    lib.iconv_plan_kernel.argtypes = [vp]
+    lib.iconv_forward.argtypes = [vp, vp, vp, vp, vp]
+    lib.iconv_check.argtypes = [vp]
+    lib.iadd_requant.argtypes = [P(iadd_desc), vp, vp, vp, vp]
+    lib.ipool_max.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
+    lib.ipool_avg_requant.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
+    lib.iq_weight_delta.argtypes = [vp, i64, P(dbl)]
+    lib.iq_quantize_weights.argtypes = [vp, i64, dbl, vp]
+    lib.iq_mul_shift.argtypes = [dbl, i32, P(i32), P(i32)]
+    lib.iq_brelu_params.argtypes = [dbl, dbl, i32, i32, P(i32), P(i32), P(i32), P(i32), P(dbl), P(dbl)]
+    lib.iq_skip_sync.argtypes = [dbl, dbl, i32, P(i32), P(i32), P(dbl), P(dbl)]
+    lib.iconcat_plan.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, P(dbl)]
+    lib.iconv_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "iconv_last_error":
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+def iconv_last_error() -> str:
+    return lib.iconv_last_error().decode()
+
+
+def _check(rc):
+    if rc != OK:
+        raise IconvError(rc, iconv_last_error())
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.atleast_1d(np.asarray(a)), dtype=np.int32)
+
+
+def iconv_plan(*, n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, in_dtype=U8, in_c_total=None, in_c_offset=0,
+               out_dtype=U8, out_c_total=None, out_c_offset=0, brelu=1, out_lo=0, out_hi=255, out_zero=0,
+               skip_dtype=-1, skip_c_total=0, skip_c_offset=0, skip_mul=1, skip_shift=0, kernel=KERNEL_AUTO,
+               weights, bias, mul=None, shift=None, h_i=None):
+    """Plan one layer; returns an opaque handle (int).  Arrays are host numpy arrays."""
+    weights = np.ascontiguousarray(weights, dtype=np.int8)
+    assert weights.shape == (c_out, kh, kw, c_in), weights.shape
+    bias = _i32(bias)
+    d = iconv_desc(n=n, h=h, w=w, c_in=c_in, c_out=c_out, kh=kh, kw=kw, stride=stride, pad=pad,
+                   in_dtype=in_dtype, in_c_total=c_in if in_c_total is None else in_c_total, in_c_offset=in_c_offset,
+                   out_dtype=out_dtype, out_c_total=c_out if out_c_total is None else out_c_total,
+                   out_c_offset=out_c_offset, brelu=int(brelu), per_channel=0,
+                   out_lo=out_lo, out_hi=out_hi, out_zero=out_zero, skip_dtype=skip_dtype,
+                   skip_c_total=skip_c_total, skip_c_offset=skip_c_offset, skip_mul=int(skip_mul),
+                   skip_shift=int(skip_shift), kernel=kernel)
+    keep = [weights, bias]
+    d.weights, d.bias = weights.ctypes.data, bias.ctypes.data
+    if mul is not None:
+        mul, shift, h_i = _i32(mul), _i32(shift), _i32(h_i)
+        assert mul.shape == shift.shape == h_i.shape and mul.shape[0] in (1, c_out)
+        d.per_channel = int(mul.shape[0] == c_out and c_out > 1)
+        d.mul, d.shift, d.h_i = mul.ctypes.data, shift.ctypes.data, h_i.ctypes.data
+        keep += [mul, shift, h_i]
+    plan = C.c_void_p()
+    _check(lib.iconv_plan(C.byref(d), C.byref(plan)))
+    return plan.value
+
+
+def iconv_plan_destroy(plan):
+    _check(lib.iconv_plan_destroy(plan))
+
+
+def iconv_plan_kernel(plan) -> int:
+    rc = lib.iconv_plan_kernel(plan)
+    if rc < 0:
+        _check(rc)
+    return rc
+
+
+def iconv_forward(plan, x_ptr, skip_ptr, out_ptr, stream=0):
+    _check(lib.iconv_forward(plan, x_ptr, skip_ptr, out_ptr, stream))
+
+
+def iconv_check(stream=0):
+    _check(lib.iconv_check(stream))
+
+
+def iadd_requant(a_ptr, b_ptr, out_ptr, stream=0, **kw):
+    _check(lib.iadd_requant(C.byref(iadd_desc(**kw)), a_ptr, b_ptr, out_ptr, stream))
+
+
+def ipool_max(x_ptr, out_ptr, n, h, w, c, k=3, stride=2, pad=1, stream=0):
+    _check(lib.ipool_max(x_ptr, out_ptr, n, h, w, c, k, stride, pad, stream))
+
+
+def ipool_avg_requant(x_ptr, out_ptr, n, h, w, c, mul, shift, max_int=255, stream=0):
+    _check(lib.ipool_avg_requant(x_ptr, out_ptr, n, h, w, c, mul, shift, max_int, stream))
+
+
+def iq_weight_delta(w_f) -> float:
+    w_f = np.ascontiguousarray(w_f, dtype=np.float32)
+    out = C.c_double()
+    _check(lib.iq_weight_delta(w_f.ctypes.data, w_f.size, C.byref(out)))
+    return out.value
+
+
+def iq_quantize_weights(w_f, delta: float):
+    w_f = np.ascontiguousarray(w_f, dtype=np.float32)
+    out = np.empty(w_f.shape, dtype=np.int8)
+    _check(lib.iq_quantize_weights(w_f.ctypes.data, w_f.size, float(delta), out.ctypes.data))
+    return out
+
+
+def iq_mul_shift(r: float, shift_min: int = 16):
+    m, s = C.c_int32(), C.c_int32()
+    _check(lib.iq_mul_shift(float(r), shift_min, C.byref(m), C.byref(s)))
+    return m.value, s.value
+
+
+def iq_brelu_params(h_rf: float, ratio_y: float, max_int: int = 255, shift_min: int = 16):
+    h_ri, m, s, h_i = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+    h_f, rv = C.c_double(), C.c_double()
+    _check(lib.iq_brelu_params(float(h_rf), float(ratio_y), max_int, shift_min, C.byref(h_ri), C.byref(m),
+                               C.byref(s), C.byref(h_i), C.byref(h_f), C.byref(rv)))
+    return dict(h_ri=h_ri.value, mul=m.value, shift=s.value, h_i=h_i.value, h_f=h_f.value, ratio_V=rv.value)
+
+
+def iq_skip_sync(ratio_y: float, ratio_s: float, shift_min: int = 8):
+    m, s, ry, ds = C.c_int32(), C.c_int32(), C.c_double(), C.c_double()
+    _check(lib.iq_skip_sync(float(ratio_y), float(ratio_s), shift_min, C.byref(m), C.byref(s), C.byref(ry),
+                            C.byref(ds)))
+    return dict(skip_mul=m.value, skip_shift=s.value, ratio_Y_new=ry.value, delta_scale=ds.value)
+
+
+def iconcat_plan(ratio_y, ratio_v, shift_min: int = 16):
+    ry = np.ascontiguousarray(ratio_y, dtype=np.float64)
+    rv = np.ascontiguousarray(ratio_v, dtype=np.float64)
+    n = ry.shape[0]
+    mul, shift = np.zeros(n, np.int32), np.zeros(n, np.int32)
+    scale, ry_new = np.zeros(n, np.float64), np.zeros(n, np.float64)
+    rmin = C.c_double()
+    _check(lib.iconcat_plan(n, ry.ctypes.data, rv.ctypes.data, shift_min, mul.ctypes.data, shift.ctypes.data,
+                            scale.ctypes.data, ry_new.ctypes.data, C.byref(rmin)))
+    return dict(ratio_V_min=rmin.value, mul=mul.tolist(), shift=shift.tolist(), delta_scale=scale.tolist(),
+                ratio_Y_new=ry_new.tolist())

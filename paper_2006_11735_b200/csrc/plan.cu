@@ -1,0 +1,39 @@
+// Kernel selection for a planned layer.
+#include "plan.h"
+
+namespace iconv {
+
+int choose_kernel(iconv_plan_t *p)
+{
+    const int want = p->d.kernel;
+    if (want == ICONV_KERNEL_DIRECT) {
+        p->kernel = ICONV_KERNEL_DIRECT;
+        return ICONV_OK;
+    }
+    if (want == ICONV_KERNEL_UMMA) {
+        const int rc = umma_supported(p);
+        if (rc != ICONV_OK) return rc;
+        p->kernel = ICONV_KERNEL_UMMA;
+        return umma_setup(p);
+    }
+    if (want == ICONV_KERNEL_THIN) {
+        const int rc = thin_supported(p);
+        if (rc != ICONV_OK) return rc;
+        p->kernel = ICONV_KERNEL_THIN;
+        return ICONV_OK;
+    }
+    // AUTO: thin layers first (they are bandwidth-bound), then the tensor-core path,
+    // the direct kernel for whatever is left.
+    if (thin_supported(p) == ICONV_OK) {
+        p->kernel = ICONV_KERNEL_THIN;
+        return ICONV_OK;
+    }
+    if (umma_supported(p) == ICONV_OK) {
+        p->kernel = ICONV_KERNEL_UMMA;
+        return umma_setup(p);
+    }
+    p->kernel = ICONV_KERNEL_DIRECT;
+    return ICONV_OK;
+}
+
+}  // namespace iconv

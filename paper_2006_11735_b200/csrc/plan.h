@@ -1,0 +1,42 @@
+// The opaque plan behind iconv_plan_t and the launchers each kernel family provides.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "common.cuh"
+
+struct iconv_plan_s {
+    iconv_desc d;            // host pointers cleared after planning
+    int h_out = 0, w_out = 0;
+    int kernel = ICONV_KERNEL_DIRECT;
+    // plain device copies (direct and thin kernels)
+    int8_t *w_dev = nullptr;
+    int32_t *bias_dev = nullptr, *mul_dev = nullptr, *shift_dev = nullptr, *h_i_dev = nullptr;
+    // tensor-core path: weights repacked [c_out_pad][taps][c_in_pad], per-channel epilogue
+    // parameters interleaved {bias, mul, shift, h_i}, TMA descriptors
+    int8_t *w_packed = nullptr;
+    int32_t *params_packed = nullptr;
+    CUtensorMap tmap_w;      // 2-D tiled map over the packed weights
+    int block_n = 0, kc = 0, c_in_pad = 0, c_out_pad = 0, stages = 0, swizzle_bytes = 0;
+    int wide_requant = 1;    // 1: 64-bit product in the epilogue; 0: proven to fit 32 bits
+};
+
+namespace iconv {
+
+int choose_kernel(iconv_plan_t *p);      // fills p->kernel and the kernel-specific fields
+
+int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
+int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
+int umma_supported(const iconv_plan_t *p);   // ICONV_OK or the reason it is not
+int umma_setup(iconv_plan_t *p);
+int thin_supported(const iconv_plan_t *p);
+
+int launch_add_requant(const iadd_desc &d, const void *a, const void *b, void *out, cudaStream_t stream);
+int launch_maxpool(const void *x, void *out, int n, int h, int w, int c, int k, int stride, int pad,
+                   cudaStream_t stream);
+int launch_avgpool(const void *x, void *out, int n, int h, int w, int c, int mul, int shift, int max_int,
+                   cudaStream_t stream);
+int *device_status_ptr();
+
+}  // namespace iconv

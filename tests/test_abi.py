@@ -1,0 +1,111 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header
+declares, validates descriptors without touching a GPU, and its host-side parameter
+arithmetic agrees with the oracle's planner."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import planner as P
+from paper_2006_11735_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "iconv.h")).read()
+    return sorted(set(re.findall(r"^ICONV_API\s+(?:const\s+)?\w+\s*\*?\s*(\w+)\s*\(", text, flags=re.M)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared()
+    assert len(names) >= 15
+    assert set(names) == set(B.EXPORTS)
+    for n in names:
+        assert hasattr(B.lib, n), n
+
+
+def _desc_kw(**over):
+    kw = dict(n=1, h=8, w=8, c_in=16, c_out=16, kh=3, kw=3, stride=1, pad=1,
+              weights=np.ones((16, 3, 3, 16), np.int8), bias=np.zeros(16, np.int32),
+              mul=[200], shift=[16], h_i=[80000])
+    kw.update(over)
+    return kw
+
+
+@pytest.mark.parametrize("over,status", [
+    (dict(h=0), B.ERR_ARG),
+    (dict(stride=0), B.ERR_ARG),
+    (dict(in_dtype=B.I32), B.ERR_ARG),
+    (dict(out_dtype=B.U8_RAW128), B.ERR_ARG),
+    (dict(kernel=9), B.ERR_ARG),
+    (dict(h=2, w=2, kh=5, kw=5, pad=1, weights=np.ones((16, 5, 5, 16), np.int8)), B.ERR_SHAPE),
+    (dict(in_c_total=16, in_c_offset=8), B.ERR_SHAPE),
+    (dict(out_c_total=24, out_c_offset=16), B.ERR_SHAPE),
+    (dict(skip_dtype=B.U8, skip_c_total=8), B.ERR_SHAPE),
+    (dict(mul=[0]), B.ERR_ARG),
+    (dict(shift=[41]), B.ERR_ARG),
+    (dict(h_i=[-1]), B.ERR_ARG),
+    (dict(out_hi=300), B.ERR_ARG),
+    (dict(skip_dtype=B.U8, skip_c_total=16, skip_mul=0), B.ERR_ARG),
+    (dict(c_in=70000, kh=1, kw=1, pad=0, weights=np.full((16, 1, 1, 70000), 127, np.int8)), B.ERR_OVERFLOW),
+    (dict(bias=np.full(16, 2 ** 31 - 1, np.int64).astype(np.int32)), B.ERR_OVERFLOW),
+])
+def test_plan_rejects_bad_descriptors_before_touching_the_gpu(over, status):
+    with pytest.raises(B.IconvError) as e:
+        B.iconv_plan(**_desc_kw(**over))
+    assert e.value.status == status
+    assert B.iconv_last_error()
+
+
+def test_null_arguments():
+    assert B.lib.iconv_plan(None, None) == B.ERR_ARG
+    assert B.lib.iconv_forward(None, None, None, None, None) == B.ERR_ARG
+    assert B.lib.iconv_plan_destroy(None) == B.OK
+    assert B.lib.iadd_requant(None, None, None, None, None) == B.ERR_ARG
+    assert B.lib.ipool_max(None, None, 1, 8, 8, 15, 3, 2, 1, None) == B.ERR_ALIGN
+
+
+def test_weight_quantisation_matches_oracle_planner():
+    rng = np.random.default_rng(0)
+    w = rng.normal(0, 0.05, size=20000).astype(np.float32)
+    d = B.iq_weight_delta(w)
+    assert d == P.weight_delta(w)
+    for scale in (1.0, 0.9973, 1.0041, 0.5):
+        assert np.array_equal(B.iq_quantize_weights(w, d * scale), P.quantize_weights(w, d * scale))
+
+
+def test_mul_shift_and_brelu_params_match_oracle_planner():
+    rng = np.random.default_rng(1)
+    for _ in range(500):
+        r = float(np.exp(rng.uniform(np.log(1e-8), np.log(3e4))))
+        smin = int(rng.integers(0, 20))
+        try:
+            want = P.mul_shift(r, smin)
+        except ValueError:
+            with pytest.raises(B.IconvError):
+                B.iq_mul_shift(r, smin)
+            continue
+        assert B.iq_mul_shift(r, smin) == want
+    for _ in range(500):
+        h_rf = float(np.exp(rng.uniform(np.log(1e-3), np.log(50))))
+        ry = float(np.exp(rng.uniform(np.log(10), np.log(1e6))))
+        for max_int in (255, 127, 15):
+            got = B.iq_brelu_params(h_rf, ry, max_int)
+            want = P.brelu_params(h_rf, ry, max_int)
+            for k in ("h_ri", "mul", "shift", "h_i"):
+                assert got[k] == want[k], (k, h_rf, ry)
+            assert got["ratio_V"] == want["ratio_V"] and got["h_f"] == want["h_f"]
+
+
+def test_skip_sync_and_concat_plan_match_oracle_planner():
+    rng = np.random.default_rng(2)
+    for _ in range(200):
+        ry = float(np.exp(rng.uniform(np.log(1e3), np.log(1e7))))
+        rs = float(np.exp(rng.uniform(np.log(1), np.log(1e4))))
+        assert B.iq_skip_sync(ry, rs) == P.skip_sync(ry, rs)
+        k = int(rng.integers(1, 5))
+        rys = np.exp(rng.uniform(np.log(1e3), np.log(1e6), size=k)).tolist()
+        rvs = np.exp(rng.uniform(np.log(10), np.log(500), size=k)).tolist()
+        assert B.iconcat_plan(rys, rvs) == P.concat_sync(rys, rvs)

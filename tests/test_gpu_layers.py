@@ -1,0 +1,169 @@
+"""GPU parity of single layers: every kernel family against the CPU oracle, bit for bit,
+through the C-ABI, on shapes that span several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layers as L
+from paper_2006_11735_b200 import binding as B
+
+from gpu_util import Fenced, dev, gpu_conv, oracle_conv
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(seed, n, h, w, c_in, c_out, k, in_dtype=B.U8, per_channel=False):
+    rng = np.random.default_rng(seed)
+    if in_dtype == B.S8:
+        X = rng.integers(-128, 128, size=(n, h, w, c_in), dtype=np.int8)
+    else:
+        X = rng.integers(0, 256, size=(n, h, w, c_in), dtype=np.uint8)
+    W = np.clip(np.floor(rng.normal(0, 40, size=(c_out, k, k, c_in)) + 0.5), -127, 127).astype(np.int8)
+    b = rng.integers(-4096, 4097, size=(c_out,), dtype=np.int32)
+    sigma = 40.0 * 100.0 * np.sqrt(c_in * k * k)
+    npar = c_out if per_channel else 1
+    h_i = np.maximum(1, (sigma * rng.uniform(1.0, 3.0, size=npar))).astype(np.int32)
+    shift = rng.integers(16, 20, size=npar).astype(np.int32)
+    mul = np.maximum(1, np.floor(255.0 * 2.0 ** shift / h_i + 0.5)).astype(np.int32)
+    return X, W, b, mul, shift, h_i
+
+
+GENERIC_SHAPES = [
+    # n, h, w, c_in, c_out, k, stride, pad
+    (1, 32, 32, 64, 64, 3, 1, 1),
+    (2, 9, 7, 16, 16, 3, 1, 1),
+    (1, 13, 11, 3, 8, 7, 2, 3),
+    (2, 10, 12, 1, 64, 5, 1, 2),
+    (1, 12, 10, 48, 1, 3, 1, 1),
+    (2, 8, 8, 64, 16, 5, 1, 2),
+    (1, 15, 9, 48, 32, 1, 1, 0),
+    (3, 7, 7, 128, 32, 3, 2, 1),
+    (1, 6, 6, 5, 3, 3, 1, 0),
+    (1, 1, 1, 256, 100, 1, 1, 0),
+]
+
+
+@pytest.mark.parametrize("shape", GENERIC_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("in_dtype", [B.U8, B.U8_RAW128, B.S8])
+def test_direct_kernel_matches_oracle(shape, in_dtype):
+    n, h, w, c_in, c_out, k, stride, pad = shape
+    X, W, b, mul, shift, h_i = _layer(sum(shape), n, h, w, c_in, c_out, k, in_dtype)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, in_dtype=in_dtype, kernel=B.KERNEL_DIRECT)
+    want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, in_dtype=in_dtype)
+    assert fam == B.KERNEL_DIRECT
+    assert np.array_equal(got, want)
+    zeros = (want == 0).mean()
+    assert 0.05 < zeros < 0.95
+
+
+@pytest.mark.parametrize("kernel", [B.KERNEL_DIRECT, B.KERNEL_AUTO])
+def test_raw_int32_output_signed_output_per_channel_and_offsets(kernel):
+    X, W, b, mul, shift, h_i = _layer(5, 2, 9, 10, 32, 48, 3, per_channel=True)
+    got, _ = gpu_conv(X, W, b, mul, shift, h_i, pad=1, out_dtype=B.I32, brelu=False, kernel=kernel)
+    want = oracle_conv(X, W, b, mul, shift, h_i, pad=1, out_dtype=B.I32, brelu=False)
+    assert np.array_equal(got, want)
+    # per-channel parameters, 8-bit output inside a wider tensor at a channel offset
+    got, _ = gpu_conv(X, W, b, mul, shift, h_i, pad=1, out_c_total=80, out_c_offset=16, kernel=kernel)
+    want = oracle_conv(X, W, b, mul, shift, h_i, pad=1, out_c_total=80, out_c_offset=16)
+    assert np.array_equal(got, want)
+    assert (got[..., :16] == 0x5A).all() and (got[..., 64:] == 0x5A).all()
+    # signed output without BReLU, zero point and saturation
+    got, _ = gpu_conv(X, W, b, [3], [12], [0], pad=1, out_dtype=B.S8, brelu=False, out_lo=-100, out_hi=90,
+                      out_zero=-7, kernel=kernel)
+    want = oracle_conv(X, W, b, [3], [12], [0], pad=1, out_dtype=B.S8, brelu=False, out_lo=-100, out_hi=90,
+                       out_zero=-7)
+    assert np.array_equal(got, want)
+    assert (want == -100).any() and (want == 90).any() and (want < 0).any()
+    # input read as a channel slice of a wider tensor
+    Xw = np.random.default_rng(1).integers(0, 256, size=(2, 9, 10, 64), dtype=np.uint8)
+    got, _ = gpu_conv(Xw, W, b, mul, shift, h_i, pad=1, in_c_offset=16, c_in=32, kernel=kernel)
+    want = oracle_conv(Xw, W, b, mul, shift, h_i, pad=1, in_c_offset=16, c_in=32)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("kernel", [B.KERNEL_DIRECT, B.KERNEL_AUTO])
+@pytest.mark.parametrize("skip_dtype", [B.U8, B.I32, B.U8_RAW128, B.S8])
+def test_fused_skip_matches_oracle(kernel, skip_dtype):
+    X, W, b, mul, shift, h_i = _layer(6, 2, 7, 9, 64, 64, 1)
+    rng = np.random.default_rng(7)
+    if skip_dtype == B.I32:
+        S = rng.integers(-300000, 300000, size=(2, 7, 9, 64)).astype(np.int32)
+        sm, ss = 300, 8
+    elif skip_dtype == B.S8:
+        S = rng.integers(-128, 128, size=(2, 7, 9, 64), dtype=np.int8)
+        sm, ss = 25028137, 8
+    else:
+        S = rng.integers(0, 256, size=(2, 7, 9, 64), dtype=np.uint8)
+        sm, ss = 428623, 8
+    h_i = h_i * 4
+    got, _ = gpu_conv(X, W, b, mul, shift, h_i, skip=S, skip_dtype=skip_dtype, skip_mul=sm, skip_shift=ss, kernel=kernel)
+    want = oracle_conv(X, W, b, mul, shift, h_i, skip=S, skip_dtype=skip_dtype, skip_mul=sm, skip_shift=ss)
+    assert np.array_equal(got, want)
+    assert 0.02 < (want == 0).mean() < 0.98
+
+
+def test_empty_batch_and_forward_argument_errors():
+    X, W, b, mul, shift, h_i = _layer(8, 1, 8, 8, 16, 16, 3)
+    plan = B.iconv_plan(n=0, h=8, w=8, c_in=16, c_out=16, kh=3, kw=3, pad=1, weights=W, bias=b, mul=mul,
+                        shift=shift, h_i=h_i)
+    B.iconv_forward(plan, None, None, None, 0)          # nothing to do, no error
+    B.iconv_plan_destroy(plan)
+    plan = B.iconv_plan(n=1, h=8, w=8, c_in=16, c_out=16, kh=3, kw=3, pad=1, weights=W, bias=b, mul=mul,
+                        shift=shift, h_i=h_i)
+    with pytest.raises(B.IconvError) as e:
+        B.iconv_forward(plan, None, None, None, 0)
+    assert e.value.status == B.ERR_ARG
+    B.iconv_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("n_elems", [0, 1, 15, 16, 1000, 4096 + 5, 1 << 20])
+@pytest.mark.parametrize("a_dtype,b_dtype,out_dtype", [(B.U8, B.U8, B.U8), (B.U8, B.I32, B.U8), (B.I32, B.I32, B.I32),
+                                                        (B.S8, B.U8, B.S8)])
+def test_iadd_requant_matches_oracle(n_elems, a_dtype, b_dtype, out_dtype):
+    rng = np.random.default_rng(n_elems + a_dtype)
+
+    def draw(dt):
+        if dt == B.I32:
+            return rng.integers(-200000, 200000, size=n_elems).astype(np.int32)
+        if dt == B.S8:
+            return rng.integers(-128, 128, size=n_elems, dtype=np.int8)
+        return rng.integers(0, 256, size=n_elems, dtype=np.uint8)
+
+    A, Bv = draw(a_dtype), draw(b_dtype)
+    lo, hi = {B.U8: (0, 255), B.S8: (-128, 127), B.I32: (-2 ** 31, 2 ** 31 - 1)}[out_dtype]
+    kw = dict(a_dtype=a_dtype, b_dtype=b_dtype, out_dtype=out_dtype, a_zero=128 if a_dtype == B.U8 else 0, b_zero=0,
+              mul_a=811 if a_dtype != B.I32 else 3, sh_a=3, mul_b=1 if b_dtype == B.I32 else 500, sh_b=0,
+              brelu=int(out_dtype == B.U8), h_i=150000, mul=150 if out_dtype != B.I32 else 1,
+              shift=16 if out_dtype != B.I32 else 0, out_zero=0 if out_dtype != B.S8 else -3, out_lo=lo, out_hi=hi)
+    want, _ = L.add_requant(A, Bv, **kw)
+    np_out = {B.U8: np.uint8, B.S8: np.int8, B.I32: np.int32}[out_dtype]
+    out = Fenced((n_elems,), np_out)
+    if n_elems:
+        ad, bd = dev(A), dev(Bv)
+        B.iadd_requant(ad.data_ptr(), bd.data_ptr(), out.ptr, torch.cuda.current_stream().cuda_stream,
+                       n_elems=n_elems, **kw)
+    else:
+        B.iadd_requant(None, None, None, 0, n_elems=0, **kw)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.get(), want) if n_elems else True
+
+
+def test_pooling_matches_oracle():
+    rng = np.random.default_rng(3)
+    for (n, h, w, c, k, s, p) in [(2, 16, 14, 64, 3, 2, 1), (1, 9, 9, 16, 3, 2, 1), (3, 7, 8, 32, 2, 2, 0)]:
+        x = rng.integers(0, 256, size=(n, h, w, c), dtype=np.uint8)
+        want = L.maxpool(x, k, s, p)
+        out = Fenced(want.shape, np.uint8)
+        xd = dev(x)
+        B.ipool_max(xd.data_ptr(), out.ptr, n, h, w, c, k, s, p, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.get(), want)
+    for (n, h, w, c) in [(3, 7, 7, 2048), (2, 2, 2, 40), (1, 5, 3, 7)]:
+        x = rng.integers(0, 256, size=(n, h, w, c), dtype=np.uint8)
+        mul = (2 ** 16 * 2 + h * w) // (2 * h * w)
+        want = L.avgpool_requant(x, mul, 16)
+        out = Fenced(want.shape, np.uint8)
+        xd = dev(x)
+        B.ipool_avg_requant(xd.data_ptr(), out.ptr, n, h, w, c, mul, 16, 255, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.get(), want)

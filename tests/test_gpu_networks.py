@@ -1,0 +1,36 @@
+"""GPU parity of whole networks: every layer of small instances of the five
+configurations against the oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import networks as ON
+from paper_2006_11735_b200 import binding as B
+from paper_2006_11735_b200.network import Network
+from workloads import networks as N
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [
+    N.single_conv(),
+    N.vdsr(n=2, h=40, w=48),
+    N.vrcnn(n=2, h=40, w=56),
+    N.resnet50(n=2, h=64, w=64),
+    N.resnet152(n=1, h=64, w=64),
+]
+
+
+@pytest.mark.parametrize("net", SMALL, ids=lambda n: n.name)
+@pytest.mark.parametrize("kernel", [B.KERNEL_DIRECT, B.KERNEL_AUTO], ids=["direct", "auto"])
+def test_every_layer_of_small_networks_matches_oracle(net, kernel):
+    params = ON.calibrate(net)
+    x = ON.net_input(net)
+    want = ON.forward(net, params, x)
+    g = Network(net, params, kernel=kernel)
+    out = g.forward(torch.from_numpy(x).cuda())
+    B.iconv_check(torch.cuda.current_stream().cuda_stream)
+    for op in net.ops:
+        got = g.tensors[op.dst].cpu().numpy()
+        assert np.array_equal(got, want[op.dst]), "%s: %d mismatches" % (op.name, (got != want[op.dst]).sum())
+    assert np.array_equal(out.cpu().numpy(), want[net.output])
+    g.close()
