@@ -167,3 +167,54 @@ def test_pooling_matches_oracle():
         B.ipool_avg_requant(xd.data_ptr(), out.ptr, n, h, w, c, mul, 16, 255, torch.cuda.current_stream().cuda_stream)
         torch.cuda.synchronize()
         assert np.array_equal(out.get(), want)
+
+
+UMMA_SHAPES = [
+    # n, h, w, c_in, c_out, k, stride, pad
+    (1, 32, 32, 64, 64, 3, 1, 1),       # configuration 1
+    (2, 9, 7, 16, 16, 3, 1, 1),         # one ragged tile
+    (3, 13, 11, 32, 32, 3, 1, 1),       # several tiles + tail, 32-byte swizzle
+    (2, 12, 12, 64, 16, 5, 1, 2),       # VRCNN 5x5 branch
+    (2, 12, 12, 64, 32, 3, 1, 1),
+    (2, 11, 13, 48, 16, 3, 1, 1),       # 48 channels: chunk wider than the tensor
+    (2, 11, 13, 48, 32, 1, 1, 0),
+    (2, 14, 14, 128, 128, 3, 2, 1),     # stride 2, 128-byte swizzle
+    (2, 14, 14, 256, 512, 1, 2, 0),     # strided projection, two N tiles
+    (1, 9, 9, 256, 64, 1, 1, 0),
+    (2, 7, 7, 512, 512, 3, 1, 1),       # long reduction: 36 pipeline iterations
+    (5, 1, 1, 2048, 1000, 1, 1, 0),     # fully connected, padded N
+    (1, 20, 20, 64, 256, 1, 1, 0),
+    (2, 6, 10, 64, 48, 3, 1, 1),        # N = 48
+]
+
+
+@pytest.mark.parametrize("shape", UMMA_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_tensor_core_kernel_matches_oracle(shape):
+    n, h, w, c_in, c_out, k, stride, pad = shape
+    X, W, b, mul, shift, h_i = _layer(sum(shape) + 1, n, h, w, c_in, c_out, k)
+    if c_out % 16:
+        got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, out_dtype=B.I32, brelu=False,
+                            kernel=B.KERNEL_UMMA)
+        want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, out_dtype=B.I32, brelu=False)
+    else:
+        got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, kernel=B.KERNEL_UMMA)
+        want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad)
+        assert 0.05 < (want == 0).mean() < 0.95
+    assert fam == B.KERNEL_UMMA
+    bad = np.argwhere(got != want)
+    assert bad.shape[0] == 0, "%d mismatches, first at %s: got %s want %s" % (
+        bad.shape[0], bad[0], got[tuple(bad[0])], want[tuple(bad[0])])
+
+
+def test_tensor_core_kernel_signed_activations_and_large_batch_tail():
+    X, W, b, mul, shift, h_i = _layer(77, 7, 19, 17, 64, 64, 3, in_dtype=B.S8)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.S8, kernel=B.KERNEL_UMMA)
+    want = oracle_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.S8)
+    assert fam == B.KERNEL_UMMA and np.array_equal(got, want)
+
+
+def test_tensor_core_kernel_rejects_what_it_cannot_take():
+    X, W, b, mul, shift, h_i = _layer(78, 1, 8, 8, 3, 16, 3)
+    with pytest.raises(B.IconvError) as e:
+        gpu_conv(X, W, b, mul, shift, h_i, pad=1, kernel=B.KERNEL_UMMA)
+    assert e.value.status == B.ERR_UNSUPPORTED
