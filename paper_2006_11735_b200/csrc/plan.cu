@@ -6,7 +6,7 @@ namespace iconv {
 int choose_kernel(iconv_plan_t *p)
 {
     const int want = p->d.kernel;
-    if (want == ICONV_KERNEL_DIRECT) {
+    if (want == ICONV_KERNEL_DIRECT || p->d.n == 0) {
         p->kernel = ICONV_KERNEL_DIRECT;
         return ICONV_OK;
     }
@@ -29,8 +29,14 @@ int choose_kernel(iconv_plan_t *p)
         return ICONV_OK;
     }
     if (umma_supported(p) == ICONV_OK) {
-        p->kernel = ICONV_KERNEL_UMMA;
-        return umma_setup(p);
+        const int rc = umma_setup(p);
+        if (rc == ICONV_OK) {
+            p->kernel = ICONV_KERNEL_UMMA;
+            return ICONV_OK;
+        }
+        if (rc != ICONV_ERR_UNSUPPORTED) return rc;
+        cudaFree(p->w_packed);               // geometry the TMA descriptor cannot express
+        p->w_packed = nullptr;
     }
     p->kernel = ICONV_KERNEL_DIRECT;
     return ICONV_OK;

@@ -76,12 +76,27 @@ class Network:
     def kernels(self) -> dict:
         return {k: B.KERNEL_NAME[B.iconv_plan_kernel(p)] for k, p in self.plans.items()}
 
-    def forward(self, x: torch.Tensor = None) -> torch.Tensor:
-        """x: uint8 device tensor [n][h][w][c] (or None to reuse the resident input)."""
-        stream = torch.cuda.current_stream(self.device).cuda_stream
+    def conv_macs(self) -> dict:
+        """True multiply-accumulates per forward of every convolution (M * N * K)."""
+        out = {}
+        for op in self.net.convs():
+            dst = self.net.tensors[op.dst]
+            out[op.name] = self.n * dst.h * dst.w * op.c_out * op.c_in * op.k * op.k
+        return out
+
+    def forward(self, x: torch.Tensor = None, marks: list = None) -> torch.Tensor:
+        """x: uint8 device tensor [n][h][w][c] (or None to reuse the resident input).
+        marks: if a list, receives (op name, event recorded after that op's launch); the
+        first entry (None, event) marks the start."""
+        ts = torch.cuda.current_stream(self.device)
+        stream = ts.cuda_stream
         T = self.tensors
         if x is not None:
             T[self.net.input] = x
+        if marks is not None:
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record(ts)
+            marks.append((None, ev))
         for kind, op, p in self.steps:
             src = self.net.tensors[op.src]
             if kind == "conv":
@@ -93,6 +108,10 @@ class Network:
             else:
                 B.ipool_avg_requant(T[op.src].data_ptr(), T[op.dst].data_ptr(), self.n, src.h, src.w, src.c,
                                     p["mul"], p["shift"], self.net.max_int, stream)
+            if marks is not None:
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record(ts)
+                marks.append((op.name, ev))
         return T[self.net.output]
 
     def close(self):
