@@ -66,7 +66,10 @@ typedef enum {
     ICONV_KERNEL_AUTO = 0,
     ICONV_KERNEL_DIRECT = 1,   /* CUDA-core direct convolution, any shape */
     ICONV_KERNEL_UMMA = 2,     /* tcgen05.mma kind::i8 implicit GEMM, TMA im2col staging */
-    ICONV_KERNEL_THIN = 3      /* bandwidth-bound layers: c_in <= 4 or c_out == 1 */
+    ICONV_KERNEL_THIN = 3,     /* bandwidth-bound layers: c_in <= 4 or c_out == 1 */
+    ICONV_KERNEL_STEM = 4      /* 7x7/2 layer over a 3-channel image: space-to-depth repack into
+                                  plan-owned scratch, then the tensor-core kernel.  Forwards of
+                                  one such plan must not overlap on the GPU (they share the scratch). */
 } iconv_kernel;
 
 /*

@@ -11,9 +11,9 @@ LIB_PATH = os.path.join(_HERE, "libiconv_b200.so")
 
 OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_OVERFLOW, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
 U8, S8, I32, U8_RAW128 = 0, 1, 2, 3
-KERNEL_AUTO, KERNEL_DIRECT, KERNEL_UMMA, KERNEL_THIN = 0, 1, 2, 3
+KERNEL_AUTO, KERNEL_DIRECT, KERNEL_UMMA, KERNEL_THIN, KERNEL_STEM = 0, 1, 2, 3, 4
 DTYPE_CODE = {"u8": U8, "s8": S8, "i32": I32, "u8_raw128": U8_RAW128}
-KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin"}
+KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin", KERNEL_STEM: "stem"}
 
 EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_forward", "iconv_check",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",

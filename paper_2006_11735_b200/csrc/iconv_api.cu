@@ -58,7 +58,7 @@ static int validate(const iconv_desc &d, int &h_out, int &w_out)
         set_error("iconv_plan: bad skip_dtype");
         return ICONV_ERR_ARG;
     }
-    if (d.kernel < ICONV_KERNEL_AUTO || d.kernel > ICONV_KERNEL_THIN) {
+    if (d.kernel < ICONV_KERNEL_AUTO || d.kernel > ICONV_KERNEL_STEM) {
         set_error("iconv_plan: bad kernel selector");
         return ICONV_ERR_ARG;
     }
@@ -157,6 +157,8 @@ extern "C" int iconv_plan_destroy(iconv_plan_t *p)
     cudaFree(p->h_i_dev);
     cudaFree(p->w_packed);
     cudaFree(p->params_packed);
+    cudaFree(p->workspace);
+    if (p->inner) iconv_plan_destroy(p->inner);
     delete p;
     return ICONV_OK;
 }
@@ -237,6 +239,7 @@ extern "C" int iconv_forward(const iconv_plan_t *p, const void *x, const void *s
     switch (p->kernel) {
     case ICONV_KERNEL_UMMA: return launch_umma(p, a, st);
     case ICONV_KERNEL_THIN: return launch_thin(p, a, st);
+    case ICONV_KERNEL_STEM: return launch_stem(p, a, st);
     default: return launch_direct(a, st);
     }
 }

@@ -22,11 +22,25 @@ int choose_kernel(iconv_plan_t *p)
         p->kernel = ICONV_KERNEL_THIN;
         return ICONV_OK;
     }
+    if (want == ICONV_KERNEL_STEM) {
+        const int rc = stem_supported(p);
+        if (rc != ICONV_OK) return rc;
+        p->kernel = ICONV_KERNEL_STEM;
+        return stem_setup(p);
+    }
     // AUTO: thin layers first (they are bandwidth-bound), then the tensor-core path,
     // the direct kernel for whatever is left.
     if (thin_supported(p) == ICONV_OK) {
         p->kernel = ICONV_KERNEL_THIN;
         return ICONV_OK;
+    }
+    if (stem_supported(p) == ICONV_OK) {
+        const int rc = stem_setup(p);
+        if (rc == ICONV_OK) {
+            p->kernel = ICONV_KERNEL_STEM;
+            return ICONV_OK;
+        }
+        if (rc != ICONV_ERR_UNSUPPORTED) return rc;
     }
     if (umma_supported(p) == ICONV_OK) {
         const int rc = umma_setup(p);

@@ -19,7 +19,12 @@ struct iconv_plan_s {
     int32_t *params_packed = nullptr;
     CUtensorMap tmap_w;      // 2-D tiled map over the packed weights
     int block_n = 0, kc = 0, c_in_pad = 0, c_out_pad = 0, stages = 0, swizzle_bytes = 0;
-    int wide_requant = 1;    // 1: 64-bit product in the epilogue; 0: proven to fit 32 bits
+    int epi = 0;             // epilogue variant of the tensor-core kernel
+    int half_n = 0, piece_bytes = 0;   // epilogue column split and staged piece width
+    // stem path: repacked image (plan-owned scratch) and the plan of the GEMM that follows
+    iconv_plan_s *inner = nullptr;
+    void *workspace = nullptr;
+    size_t workspace_bytes = 0;
 };
 
 namespace iconv {
@@ -31,6 +36,9 @@ int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int umma_supported(const iconv_plan_t *p);   // ICONV_OK or the reason it is not
 int umma_setup(iconv_plan_t *p);
 int thin_supported(const iconv_plan_t *p);
+int stem_supported(const iconv_plan_t *p);
+int stem_setup(iconv_plan_t *p);
+int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 
 int launch_add_requant(const iadd_desc &d, const void *a, const void *b, void *out, cudaStream_t stream);
 int launch_maxpool(const void *x, void *out, int n, int h, int w, int c, int k, int stride, int pad,

@@ -218,3 +218,17 @@ def test_tensor_core_kernel_rejects_what_it_cannot_take():
     with pytest.raises(B.IconvError) as e:
         gpu_conv(X, W, b, mul, shift, h_i, pad=1, kernel=B.KERNEL_UMMA)
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("shape", [(2, 30, 26, 64), (1, 33, 31, 16), (3, 16, 16, 32)], ids=str)
+@pytest.mark.parametrize("in_dtype", [B.U8_RAW128, B.U8, B.S8])
+def test_stem_path_matches_oracle(shape, in_dtype):
+    n, h, w, c_out = shape
+    X, W, b, mul, shift, h_i = _layer(h * w + c_out, n, h, w, 3, c_out, 7, in_dtype)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=2, pad=3, in_dtype=in_dtype, kernel=B.KERNEL_STEM)
+    want = oracle_conv(X, W, b, mul, shift, h_i, stride=2, pad=3, in_dtype=in_dtype)
+    assert fam == B.KERNEL_STEM
+    assert np.array_equal(got, want)
+    assert 0.05 < (want == 0).mean() < 0.95
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=2, pad=3, in_dtype=in_dtype)
+    assert fam == B.KERNEL_STEM and np.array_equal(got, want)      # AUTO picks it too
