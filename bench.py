@@ -152,6 +152,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--per-layer", action="store_true", help="print the per-layer table to stderr")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="images per GPU; 0 = the full workload (256). Smaller batches are for profiler "
+                         "captures only and are named in config.workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -172,7 +175,8 @@ def main():
     dev = torch.device("cuda", local_rank)
     D.init("nccl")
 
-    net = N.resnet50()                      # 256 images per GPU (weak scaling: every rank its own batch)
+    net = N.resnet50(n=args.batch) if args.batch > 0 else N.resnet50()   # 256 images per GPU (weak scaling)
+    workload = WORKLOAD if net.n == 256 else "resnet50_b%d_224x224x3 (reduced batch: profiling only)" % net.n
     params = load_params("resnet50")
     g = Network(net, params, device=dev)
     x_host = torch.from_numpy(net_input(net)).pin_memory()
@@ -260,7 +264,7 @@ def main():
         line = {"metric": METRIC, "value": total_images / (ms * 1e-3), "unit": UNIT, "n_gpus": size,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "global_batch": net.n * size, "parallelism": "dp%d" % size,
+                "config": {"workload": workload, "global_batch": net.n * size, "parallelism": "dp%d" % size,
                            "l2": "per-step activation traffic (~7 GB) far exceeds the 126 MB L2",
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
                 "clocks": clocks,

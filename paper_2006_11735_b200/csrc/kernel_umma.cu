@@ -5,19 +5,27 @@
 //               channel chunk) brings 128 consecutive output pixels x KC channels into
 //               shared memory, K-major, hardware-swizzled; out-of-image taps arrive as 0.
 //   B operand   int8 weights, repacked at plan time to [c_out_pad][tap][c_in_pad] and
-//               fetched by tiled TMA into the same K-major swizzled layout.
-//   D           int32 accumulators in tensor memory (TMEM), two buffers of BLOCK_N columns,
-//               so the epilogue of one tile overlaps the MMAs of the next.
+//               fetched by tiled TMA into the same K-major swizzled layout.  When the whole
+//               packed filter bank fits beside the pipeline it is loaded once per CTA and
+//               stays resident; otherwise its tiles travel through the stages with A.
+//   D           int32 accumulators in tensor memory (TMEM): two buffers of up to 256 columns
+//               or four of up to 128, so the epilogue of one tile overlaps the MMAs of the next.
 //   MMA         tcgen05.mma.cta_group::1.kind::i8, M=128, N=BLOCK_N, K=32 per instruction,
 //               u8 (or s8) x s8 -> s32, issued by one thread.
-//   Epilogue    four warps read TMEM (32 lanes each), add the bias and the rescaled skip,
-//               apply BReLU, Eq. 4, zero point and saturation, and store 16 output
-//               channels per 16-byte store at the layer's channel offset.
+//   Epilogue    up to sixteen warps read TMEM (32 lanes = 32 output pixels each), apply bias,
+//               rescaled skip, BReLU, Eq. 4, zero point and saturation, stage 16 output
+//               channels per 16-byte shared-memory store and hand 32-row pieces to TMA
+//               stores aimed at the layer's channel offset.
 //
 // Persistent CTAs (one per SM) walk the tiles round-robin.  Warp 0 produces (TMA), warp 1
-// issues MMAs and owns the TMEM allocation, warps 2-5 run the epilogue.  All mbarrier
+// issues MMAs and owns the TMEM allocation, the others run the epilogue.  All mbarrier
 // waits are bounded: on expiry the CTA records a code in the device status word, drains
 // its copies in flight, frees its TMEM and returns.
+//
+// Measured on B200 and built into the structure: one thread needs 300-400 cycles per TMA
+// instruction and per MMA-group + commit round, whatever the box or instruction size, so
+// stages are as large as shared memory allows and nothing but the barrier traffic sits in
+// the per-stage loops (no divisions: counters and multiply-shift reciprocals).
 #include <cuda.h>
 
 #include <vector>
@@ -29,45 +37,58 @@ namespace iconv {
 namespace {
 
 constexpr int BLOCK_M = 128;
-constexpr int NUM_THREADS = 320;          // TMA warp, MMA warp, eight epilogue warps
-constexpr int WARP_COLS = 128;            // columns one epilogue warp handles per tile (256 / 2)
+constexpr int EPI_WARPS_MAX = 16;
+constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS_MAX);   // TMA warp, MMA warp, epilogue warps
+constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces (+ the skip rows of one tile)
+constexpr int MAX_STAGES = 12;
+constexpr int MAX_TMEM_BUFS = 4;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds at the boost clock
+constexpr int MAX_SMEM = 227 * 1024;
+constexpr int RESIDENT_B_MAX = 80 * 1024;
 
-// Epilogue variants, chosen at plan time.
-enum { EPI_WIDE = 0,             // any descriptor: 64-bit products, run-time branches
-       EPI_RAW = 1,              // int32 Y out, no skip: bias add only
-       EPI_NARROW_NOSKIP = 2,    // BReLU + Eq. 4 proven to fit 32 bits
-       EPI_NARROW_SKIP8 = 3,     // ... with an 8-bit skip whose rescale fits 32 bits
-       EPI_NARROW_SKIPWIDE = 4   // ... with an int32 (or unproven) skip added in 64 bits
+// Epilogue variants, chosen at plan time.  "32-bit" variants rely on bounds the plan proves
+// from the layer's actual weights and parameters; whatever cannot be proven runs EPI_WIDE.
+enum {
+    EPI_WIDE = 0,        // any descriptor: 64-bit products, run-time branches, direct skip loads
+    EPI_RAW = 1,         // int32 Y out, no skip: bias add only
+    EPI_FAST = 2,        // u8 out, no skip: V = sat_u8((U*mul + C) >> shift), clamps folded into the saturation
+    EPI_FAST_SKIP8 = 3,  // ... with an 8-bit skip staged by TMA
+    EPI_SAFE = 4,        // explicit BReLU clamp, 32-bit Eq. 4, optional zero point / range tail
+    EPI_SAFE_SKIP8 = 5,  // ... with an 8-bit skip staged by TMA
+    EPI_SAFE_SKIP32 = 6  // ... with an int32 skip (projection), rescaled in 64 bits
 };
-constexpr int MAX_STAGES = 8;
-constexpr unsigned long long WAIT_LIMIT_NS = 4000000000ull;
-constexpr int EPI_SMEM = 8 * 8192;        // per epilogue warp: output staging + skip staging
-constexpr int SMEM_BUDGET = 140 * 1024;    // pipeline stages; barriers, parameters and epilogue staging come on top
-constexpr int MAX_SMEM = 225 * 1024;
 
 struct UmmaArgs {
     long long m_total;
     int m_tiles, n_tiles;
     int block_n, kc, cchunks, taps;
-    int stages, stage_a_bytes, stage_bytes;
-    int tmem_cols;
+    int stages, stage_a_bytes, stage_bytes, b_tile_bytes, resident_b;
+    int tmem_cols, nbuf, lg_nbuf;   // accumulator buffers (2 or 4)
+    int epi_warps, cs, bi;          // epilogue warps, column split per tile, tiles in flight
+    int part_n;                     // columns one epilogue warp handles per tile
+    int piece_bytes;                // row width of one staged output piece (16 ... 128 bytes)
     unsigned idesc;
     unsigned long long desc_hi;     // upper 32 bits of the shared-memory matrix descriptors
+    // per-layer epilogue scalars (per-channel layers read the arrays instead)
+    int q_mul, q_shift, q_half, q_h;
     int skip_half;                  // 2^(skip_shift-1), or 0
-    int half_n;                     // columns of the tile taken by the first epilogue warp of a quadrant
-    int piece_bytes;                // row width of one staged output piece (16, 32, 64 or 128 bytes)
+    unsigned skip_xor;              // 0x80808080 turns int8 skip bytes into offset-binary
+    int tail;                       // 1: out_zero / out_lo / out_hi are not provably no-ops
+    const int32_t *c_a;             // [c_out_pad] per-channel additive constant of the variant
+    const int32_t *c_mul, *c_shift, *c_h;   // [c_out_pad] copies for per-channel layers
     int *status;
+    // exact division of a tile index by n_tiles and of a pixel index by w_out and by
+    // h_out * w_out without a divide instruction: q = umulhi(x, mul) >> shr  (x < 2^31)
+    unsigned div_nt_mul, div_nt_shr, div_w_mul, div_w_shr, div_hw_mul, div_hw_shr;
 };
+
+__device__ __forceinline__ unsigned fast_div(unsigned x, unsigned mul, unsigned shr)
+{
+    return mul ? (__umulhi(x, mul) >> shr) : x;
+}
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long globaltimer()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -81,12 +102,13 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+// Non-blocking probe of a barrier phase.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -95,17 +117,46 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 
 // Bounded wait.  Returns false when the limit ran out or another role already gave up.
+// The limit is counted on the SM's own cycle counter, read only every 1024 failed polls:
+// a wait that succeeds costs no timer read.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer();
+    if (mbar_test_wait(bar, parity)) return true;
+    long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 0) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((i & 1023u) == 0) {
             if (*abort_flag) return false;
-            if (globaltimer() - t0 > WAIT_LIMIT_NS) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_CYCLES) return false;
         }
     }
+}
+
+// The same wait taken by one lane on behalf of its warp (32 lanes polling one barrier word
+// only add shared-memory traffic).  Backs off between polls; __syncwarp orders the other
+// lanes' later reads after lane 0's acquire.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane)
+{
+    int ok = 1;
+    if (lane == 0) {
+        ok = 0;
+        long long t0 = 0;
+        for (uint32_t i = 0;; ++i) {
+            if (mbar_test_wait(bar, parity)) { ok = 1; break; }
+            if (i >= 8) __nanosleep(32);
+            if ((i & 1023u) == 1023u) {
+                if (*abort_flag) break;
+                const long long now = clock64();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > WAIT_LIMIT_CYCLES) break;
+            }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
 }
 
 __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w,
@@ -154,7 +205,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int *r)
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -165,6 +216,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// d = { sat8(v3), sat8(v2), sat8(v1), sat8(v0) } (v0 in the low byte), unsigned or signed saturation
+template <bool SIGNED>
+__device__ __forceinline__ unsigned pack4_sat(int v0, int v1, int v2, int v3)
+{
+    unsigned hi, d;
+    if (SIGNED) {
+        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0));
+        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v1), "r"(v0), "r"(hi));
+    } else {
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0));
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v1), "r"(v0), "r"(hi));
+    }
+    return d;
+}
+
 // Shared-memory matrix descriptor of a K-major, hardware-swizzled tile whose rows are one
 // swizzle span wide: start address, stride between 8-row groups, descriptor version 1
 // and the swizzle mode (the constant upper half comes from the host).
@@ -173,17 +239,13 @@ __device__ __forceinline__ unsigned long long smem_desc(uint32_t addr, unsigned 
     return hi | (unsigned long long)((addr & 0x3FFFFu) >> 4) | (1ull << 16);
 }
 
-struct WarpParams {
-    int bias[WARP_COLS], mul[WARP_COLS], shift[WARP_COLS], h_i[WARP_COLS];
-};
-
 struct Shared {
-    WarpParams params[8];
-    unsigned long long skip_full[8];
+    unsigned long long skip_full[EPI_WARPS_MAX];
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
-    unsigned long long tmem_full[2];
-    unsigned long long tmem_empty[2];
+    unsigned long long tmem_full[MAX_TMEM_BUFS];
+    unsigned long long tmem_empty[MAX_TMEM_BUFS];
+    unsigned long long b_full;
     unsigned long long drain;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -195,6 +257,149 @@ __device__ __forceinline__ void give_up(Shared *sh, int *status, int code)
     atomicCAS(status, 0, code);
 }
 
+// One group of 16 consecutive output channels of one pixel: accumulators in, 16 output
+// values (8-bit variants) or 16 int32 (raw) out.  `sk` holds the 16 staged skip bytes.
+template <int EPI>
+__device__ __forceinline__ void epilogue16(const int *acc, int *V, int co0, long long m, bool row_ok, uint4 sk,
+                                           const ConvArgs &a, const UmmaArgs &u)
+{
+    const int4 *ca4 = (const int4 *)(u.c_a + co0);
+    if (EPI == EPI_RAW) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int4 c = __ldg(ca4 + g);
+            V[4 * g] = acc[4 * g] + c.x; V[4 * g + 1] = acc[4 * g + 1] + c.y;
+            V[4 * g + 2] = acc[4 * g + 2] + c.z; V[4 * g + 3] = acc[4 * g + 3] + c.w;
+        }
+        return;
+    }
+    if (EPI == EPI_FAST) {
+        // (U + b) * mul + half = U * mul + C with C = b * mul + half; the shift is arithmetic and the
+        // u8 saturation that follows stands for both BReLU clamps (proven at plan time)
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int4 c = __ldg(ca4 + g);
+            V[4 * g] = (acc[4 * g] * u.q_mul + c.x) >> u.q_shift;
+            V[4 * g + 1] = (acc[4 * g + 1] * u.q_mul + c.y) >> u.q_shift;
+            V[4 * g + 2] = (acc[4 * g + 2] * u.q_mul + c.z) >> u.q_shift;
+            V[4 * g + 3] = (acc[4 * g + 3] * u.q_mul + c.w) >> u.q_shift;
+        }
+        return;
+    }
+    if (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8) {
+        // Y = U + ((s * skip_mul + C) >> skip_shift) with C = (b << skip_shift) + skip_half - z * skip_mul,
+        // where s is the stored byte as an unsigned number and z its zero (0, or 128 for raw-128 and
+        // offset-binary int8): the bias rides inside the rounding shift, which is exact.
+        const unsigned w4[4] = {sk.x ^ u.skip_xor, sk.y ^ u.skip_xor, sk.z ^ u.skip_xor, sk.w ^ u.skip_xor};
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int4 c = __ldg(ca4 + g);
+            const int cc[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int sv = (int)__byte_perm(w4[g], 0, 0x4440 + e);
+                int y = acc[4 * g + e] + ((sv * a.skip_mul + cc[e]) >> a.skip_shift);
+                if (EPI == EPI_FAST_SKIP8) {
+                    V[4 * g + e] = (y * u.q_mul + u.q_half) >> u.q_shift;
+                } else {
+                    int h = u.q_h, mul = u.q_mul, shift = u.q_shift, half = u.q_half;
+                    if (a.per_channel) {
+                        h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
+                        shift = __ldg(u.c_shift + co0 + 4 * g + e); half = (int)(1u << (shift - 1));
+                    }
+                    y = max(min(y, h), 0);
+                    int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
+                    if (u.tail) v = min(max(v + a.out_zero, a.out_lo), a.out_hi);
+                    V[4 * g + e] = v;
+                }
+            }
+        }
+        return;
+    }
+    if (EPI == EPI_SAFE || EPI == EPI_SAFE_SKIP32) {
+        int4 s32[4] = {make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0)};
+        if (EPI == EPI_SAFE_SKIP32 && row_ok) {
+            const int4 *sp = (const int4 *)((const int32_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0);
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+                s32[g] = (co0 + 4 * g < a.c_out) ? __ldg(sp + g) : make_int4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int4 c = __ldg(ca4 + g);
+            const int cc[4] = {c.x, c.y, c.z, c.w};
+            const int ss[4] = {s32[g].x, s32[g].y, s32[g].z, s32[g].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                int h = u.q_h, mul = u.q_mul, shift = u.q_shift, half = u.q_half;
+                if (a.per_channel) {
+                    h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
+                    shift = __ldg(u.c_shift + co0 + 4 * g + e); half = (int)(1u << (shift - 1));
+                }
+                int y;
+                if (EPI == EPI_SAFE_SKIP32) {
+                    long long Y = (long long)acc[4 * g + e] + cc[e] + round_shift64((long long)ss[e] * a.skip_mul, a.skip_shift);
+                    Y = Y < 0 ? 0 : (Y > (long long)h ? (long long)h : Y);
+                    y = (int)Y;
+                } else {
+                    y = max(min(acc[4 * g + e] + cc[e], h), 0);
+                }
+                int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
+                if (u.tail) v = min(max(v + a.out_zero, a.out_lo), a.out_hi);
+                V[4 * g + e] = v;
+            }
+        }
+        return;
+    }
+    // EPI_WIDE: everything at run time, 64-bit products, skip read straight from global memory
+    {
+        uint4 sk8 = make_uint4(0, 0, 0, 0);
+        int4 s32[4] = {make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0)};
+        if (a.skip_dtype >= 0 && row_ok && co0 < a.c_out) {
+            if (a.skip_dtype == ICONV_I32) {
+                const int4 *sp = (const int4 *)((const int32_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0);
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    s32[g] = (co0 + 4 * g < a.c_out) ? __ldg(sp + g) : make_int4(0, 0, 0, 0);
+            } else {
+                sk8 = __ldg((const uint4 *)((const uint8_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0));
+            }
+        }
+        const unsigned w4[4] = {sk8.x, sk8.y, sk8.z, sk8.w};
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int4 c = __ldg(ca4 + g);
+            const int cc[4] = {c.x, c.y, c.z, c.w};
+            const int ss[4] = {s32[g].x, s32[g].y, s32[g].z, s32[g].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                long long Y = (long long)acc[4 * g + e] + cc[e];
+                if (a.skip_dtype >= 0) {
+                    int sv;
+                    if (a.skip_dtype == ICONV_I32) {
+                        sv = ss[e];
+                    } else {
+                        const unsigned byte = (w4[g] >> (8 * e)) & 0xffu;
+                        sv = a.skip_dtype == ICONV_S8 ? (int)(int8_t)byte
+                                                      : (int)byte - (a.skip_dtype == ICONV_U8_RAW128 ? 128 : 0);
+                    }
+                    Y += round_shift64((long long)sv * a.skip_mul, a.skip_shift);
+                }
+                if (a.out_dtype == ICONV_I32) {
+                    V[4 * g + e] = (int)Y;
+                } else {
+                    int h = u.q_h, mul = u.q_mul, shift = u.q_shift;
+                    if (a.per_channel) {
+                        h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
+                        shift = __ldg(u.c_shift + co0 + 4 * g + e);
+                    }
+                    V[4 * g + e] = requant_tail(Y, a.brelu, h, mul, shift, a.out_zero, a.out_lo, a.out_hi);
+                }
+            }
+        }
+    }
+}
+
 }  // namespace
 
 template <int EPI>
@@ -203,28 +408,30 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                  const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_skip,
                  const __grid_constant__ ConvArgs a, const __grid_constant__ UmmaArgs u)
 {
+    constexpr bool SKIP8 = (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8);
     extern __shared__ uint8_t smem_raw[];
     // tiles need the alignment of the widest swizzle pattern (8 rows x 128 bytes)
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    Shared *sh = (Shared *)(tiles + (size_t)u.stages * u.stage_bytes);
-    // per epilogue warp: 4 KB output staging + 4 KB skip staging, 1024-byte aligned
+    uint8_t *b_res = tiles + (size_t)u.stages * u.stage_bytes;                 // resident filter bank (may be empty)
+    const int k_iters = u.taps * u.cchunks;
+    Shared *sh = (Shared *)(b_res + (u.resident_b ? (size_t)u.b_tile_bytes * k_iters * u.n_tiles : 0));
     uint8_t *epi_smem = (uint8_t *)(((uintptr_t)(sh + 1) + 1023) & ~(uintptr_t)1023);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_tiles = u.m_tiles * u.n_tiles;
-    const int k_iters = u.taps * u.cchunks;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < u.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
             mbar_init(smem_u32(&sh->empty[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < u.nbuf; ++b) {
             mbar_init(smem_u32(&sh->tmem_full[b]), 1);
-            mbar_init(smem_u32(&sh->tmem_empty[b]), 8);
+            mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)(4 * u.cs));
         }
-        for (int w = 0; w < 8; ++w) mbar_init(smem_u32(&sh->skip_full[w]), 1);
+        for (int w = 0; w < EPI_WARPS_MAX; ++w) mbar_init(smem_u32(&sh->skip_full[w]), 1);
+        mbar_init(smem_u32(&sh->b_full), 1);
         mbar_init(smem_u32(&sh->drain), 1);
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -236,25 +443,38 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t tmem_base = sh->tmem_base;
 
     int issued = 0;        // producer: k-iterations whose loads were issued
+    int b_issued = 0;      // producer: resident filter bank requested
     int skip_issued = 0;   // epilogue lane 0: skip prefetches issued
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            int it = 0;
+        if (lane == 0 && (int)blockIdx.x < num_tiles) {
+            if (u.resident_b) {
+                const uint32_t bf = smem_u32(&sh->b_full);
+                mbar_expect_tx(bf, (uint32_t)(u.block_n * u.kc * k_iters * u.n_tiles));
+                for (int nt = 0; nt < u.n_tiles; ++nt)
+                    for (int ki = 0; ki < k_iters; ++ki)
+                        tma_load_2d(smem_u32(b_res + (size_t)(nt * k_iters + ki) * u.b_tile_bytes), &tmap_w, bf,
+                                    ki * u.kc, nt * u.block_n);
+                b_issued = 1;
+            }
+            int it = 0, stage = 0;
+            uint32_t parity = 0;
             bool ok = true;
+            const int hw = a.h_out * a.w_out;
+            const uint32_t tx = (uint32_t)(BLOCK_M * u.kc + (u.resident_b ? 0 : u.block_n * u.kc));
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m_tile = tile / u.n_tiles, n_tile = tile % u.n_tiles;
-                const long long m0 = (long long)m_tile * BLOCK_M;
-                const int q = (int)(m0 % a.w_out);
-                const int p = (int)((m0 / a.w_out) % a.h_out);
-                const int img = (int)(m0 / ((long long)a.w_out * a.h_out));
+                const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
+                const int n_tile = tile - m_tile * u.n_tiles;
+                const unsigned m0 = (unsigned)m_tile * BLOCK_M;
+                const int img = (int)fast_div(m0, u.div_hw_mul, u.div_hw_shr);
+                const unsigned rem = m0 - (unsigned)img * (unsigned)hw;
+                const int p = (int)fast_div(rem, u.div_w_mul, u.div_w_shr);
+                const int q = (int)rem - p * a.w_out;
                 const int cw = q * a.stride - a.pad, ch = p * a.stride - a.pad;
+                int r = 0, s = 0, kx = 0;
                 for (int tap = 0; tap < u.taps && ok; ++tap) {
-                    const unsigned short r = (unsigned short)(tap / a.kw), s = (unsigned short)(tap % a.kw);
-                    for (int cc = 0; cc < u.cchunks; ++cc, ++it) {
-                        const int stage = it % u.stages;
-                        const uint32_t parity = (uint32_t)((it / u.stages) & 1);
+                    for (int cc = 0; cc < u.cchunks; ++cc, ++it, kx += u.kc) {
                         if (!mbar_wait(smem_u32(&sh->empty[stage]), parity ^ 1u, &sh->abort_flag)) {
                             give_up(sh, u.status, 1);
                             ok = false;
@@ -262,207 +482,165 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         }
                         const uint32_t full = smem_u32(&sh->full[stage]);
                         const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes);
-                        mbar_expect_tx(full, (uint32_t)(BLOCK_M * u.kc + u.block_n * u.kc));
-                        tma_load_im2col_4d(sa, &tmap_x, full, cc * u.kc, cw, ch, img, s, r);
-                        tma_load_2d(sa + u.stage_a_bytes, &tmap_w, full, (tap * u.cchunks + cc) * u.kc,
-                                    n_tile * u.block_n);
+                        mbar_expect_tx(full, tx);
+                        tma_load_im2col_4d(sa, &tmap_x, full, cc * u.kc, cw, ch, img, (unsigned short)s,
+                                           (unsigned short)r);
+                        if (!u.resident_b) tma_load_2d(sa + u.stage_a_bytes, &tmap_w, full, kx, n_tile * u.block_n);
                         issued = it + 1;
+                        if (++stage == u.stages) { stage = 0; parity ^= 1u; }
                     }
+                    if (++s == a.kw) { s = 0; ++r; }
                 }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            int it = 0, t = 0;
+        if (lane == 0 && (int)blockIdx.x < num_tiles) {
+            int t = 0, stage = 0;
+            uint32_t parity = 0;
             bool ok = true;
+            if (u.resident_b && !mbar_wait(smem_u32(&sh->b_full), 0, &sh->abort_flag)) {
+                give_up(sh, u.status, 6);
+                ok = false;
+            }
+            const int kj = u.kc >> 5;   // MMAs per stage: 32 bytes of K each
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
-                const int buf = t & 1;
-                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> 1) & 1) ^ 1), &sh->abort_flag)) {
+                const int buf = t & (u.nbuf - 1);
+                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
                     give_up(sh, u.status, 2);
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * u.block_n);
-                for (int ki = 0; ki < k_iters; ++ki, ++it) {
-                    const int stage = it % u.stages;
-                    if (!mbar_wait(smem_u32(&sh->full[stage]), (uint32_t)((it / u.stages) & 1), &sh->abort_flag)) {
+                uint32_t sb = 0;
+                if (u.resident_b) {
+                    const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
+                    sb = smem_u32(b_res + (size_t)((tile - m_tile * u.n_tiles) * k_iters) * u.b_tile_bytes);
+                }
+                for (int ki = 0; ki < k_iters; ++ki) {
+                    if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
                         give_up(sh, u.status, 3);
                         ok = false;
                         break;
                     }
-                    tc_fence_after();
                     const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes);
                     const unsigned long long da = smem_desc(sa, u.desc_hi);
-                    const unsigned long long db = smem_desc(sa + u.stage_a_bytes, u.desc_hi);
-                    for (int j = 0; j < u.kc / 32; ++j)   // 32 bytes of K per instruction: +2 in 16-byte units
+                    const unsigned long long db = smem_desc(u.resident_b ? sb : sa + u.stage_a_bytes, u.desc_hi);
+                    for (int j = 0; j < kj; ++j)   // +2 in 16-byte units per 32 bytes of K
                         umma_i8(d_tmem, da + 2ull * j, db + 2ull * j, u.idesc, (uint32_t)((ki | j) != 0));
                     umma_commit(smem_u32(&sh->empty[stage]));   // frees the stage when these MMAs are done
+                    if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+                    sb += (uint32_t)u.b_tile_bytes;
                 }
                 if (ok) umma_commit(smem_u32(&sh->tmem_full[buf]));
             }
         }
         __syncwarp();
-    } else {
+    } else if (warp < 2 + u.epi_warps) {
         // ---------------------------------------------------------------- epilogue
-        // Eight warps.  warp % 4 fixes the TMEM lane quadrant (32 output pixels) a warp may
-        // read; the two warps of a quadrant split the tile's columns in halves.  A warp
-        // works alone: it keeps its own copy of its channels' parameters, prefetches its
-        // own part of an 8-bit skip tensor by TMA, stages its outputs in its own swizzled
-        // shared-memory buffer and writes them with its own TMA stores (which also clip
-        // the ragged last tile), so no cross-warp barrier exists that a warp which gave up
-        // could strand.
+        // warp % 4 fixes the TMEM lane quadrant (32 output pixels) a warp may read.  The warps
+        // of a quadrant form `cs * bi` slots: `cs` slots split a tile's columns, `bi` groups
+        // of them take alternate tiles (each on its own accumulator buffer).  A warp works
+        // alone: it prefetches its own part of an 8-bit skip tensor by TMA, stages its
+        // outputs in its own two swizzled shared-memory pieces and writes them with its own
+        // TMA stores (which also clip the ragged last tile and the channels beyond c_out), so
+        // no cross-warp barrier exists that a warp which gave up could strand.
         const int ew = warp - 2;
         const int quad = warp & 3;
-        const int half = ew >> 2;
-        const int col_lo = half * u.half_n;
-        const int ncols = min(u.block_n - col_lo, u.half_n);          // may be <= 0 for narrow tiles
-        WarpParams *wp = &sh->params[ew];
-        uint8_t *obuf = epi_smem + (size_t)ew * 8192;                 // 32 rows x 128 bytes, 1024-aligned
-        uint8_t *sbuf = obuf + 4096;
+        const int slot = ew >> 2;
+        const int part = slot % u.cs;
+        const int turn = slot / u.cs;
+        const int col_lo = part * u.part_n;
+        const int ncols = min(u.block_n - col_lo, u.part_n);
+        uint8_t *obuf = epi_smem + (size_t)ew * EPI_WARP_SMEM;        // two pieces of 32 rows x piece_bytes
+        uint8_t *sbuf = obuf + EPI_WARP_SMEM / 2;                     // skip rows of one tile (8-bit variants)
         const uint32_t skip_bar = smem_u32(&sh->skip_full[ew]);
-        const int esz = a.out_dtype == ICONV_I32 ? 4 : 1;
-        const int pcols = u.piece_bytes / esz;                        // columns per staged piece
-        const int swz_shift = u.piece_bytes == 128 ? 0 : (u.piece_bytes == 64 ? 1 : 2);
-        const int swz_mask = u.piece_bytes / 16 - 1;
-        const int q_mul = __ldg(a.mul), q_shift = __ldg(a.shift), q_h_i = __ldg(a.h_i);
-        const unsigned row_off = (unsigned)lane * (unsigned)u.piece_bytes;
-        const unsigned row_swz = u.piece_bytes >= 32 ? (((unsigned)lane >> swz_shift) & (unsigned)swz_mask) : 0u;
-        int t = 0, staged_n_tile = -1;
-        bool ok = ncols > 0;
+        constexpr int esz = (EPI == EPI_RAW) ? 4 : 1;
+        const int esz_rt = (EPI == EPI_WIDE && a.out_dtype == ICONV_I32) ? 4 : esz;
+        const int pb = u.piece_bytes;
+        const int pcols = pb / esz_rt;                                // columns per staged piece
+        const int piece_smem = 32 * pb;
+        const int swz_shift = pb == 128 ? 0 : (pb == 64 ? 1 : 2);
+        const unsigned row_off = (unsigned)lane * (unsigned)pb;
+        const unsigned row_swz = pb >= 32 ? (((unsigned)lane >> swz_shift) & (unsigned)(pb / 16 - 1)) : 0u;
+        const int tile_step = u.bi * (int)gridDim.x;
+        int mine = 0, pieces = 0;
+        bool ok = true;
 
         // first skip prefetch
-        if (EPI == EPI_NARROW_SKIP8 && ok && lane == 0 && (int)blockIdx.x < num_tiles) {
-            const int tile0 = blockIdx.x;
+        if (SKIP8 && lane == 0 && (int)blockIdx.x + turn * (int)gridDim.x < num_tiles) {
+            const int tile0 = blockIdx.x + turn * gridDim.x;
+            const int mt0 = (int)fast_div((unsigned)tile0, u.div_nt_mul, u.div_nt_shr);
             mbar_expect_tx(skip_bar, (uint32_t)(32 * ncols));
             for (int c = 0; c < ncols; c += pcols)
-                tma_load_2d(smem_u32(sbuf + (size_t)(c / pcols) * 32 * u.piece_bytes), &tmap_skip, skip_bar,
-                            (tile0 % u.n_tiles) * u.block_n + col_lo + c, (tile0 / u.n_tiles) * BLOCK_M + quad * 32);
+                tma_load_2d(smem_u32(sbuf + (size_t)(c / pcols) * piece_smem), &tmap_skip, skip_bar,
+                            (tile0 - mt0 * u.n_tiles) * u.block_n + col_lo + c, mt0 * BLOCK_M + quad * 32);
             skip_issued = 1;
         }
 
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
-            const int m_tile = tile / u.n_tiles, n_tile = tile % u.n_tiles;
-            const int buf = t & 1;
+        for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles && ok; t += u.bi, tile += tile_step, ++mine) {
+            const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
+            const int n_tile = tile - m_tile * u.n_tiles;
+            const int buf = t & (u.nbuf - 1);
             const int n0 = n_tile * u.block_n + col_lo;                // first channel of this warp
-            if (n_tile != staged_n_tile) {
-                __syncwarp();
-                for (int lc = lane; lc < ncols; lc += 32) {
-                    const int co = n0 + lc;
-                    const bool in = co < a.c_out;
-                    wp->bias[lc] = in ? __ldg(a.bias + co) : 0;
-                    if (a.per_channel) {
-                        wp->mul[lc] = in ? __ldg(a.mul + co) : 1;
-                        wp->shift[lc] = in ? __ldg(a.shift + co) : 1;
-                        wp->h_i[lc] = in ? __ldg(a.h_i + co) : 0;
-                    }
-                }
-                __syncwarp();
-                staged_n_tile = n_tile;
-            }
-            if (!mbar_wait(smem_u32(&sh->tmem_full[buf]), (uint32_t)((t >> 1) & 1), &sh->abort_flag)) {
+            if (!mbar_wait_warp(smem_u32(&sh->tmem_full[buf]), (uint32_t)((t >> u.lg_nbuf) & 1), &sh->abort_flag, lane)) {
                 give_up(sh, u.status, 4);
                 break;
             }
             tc_fence_after();
-            if (EPI == EPI_NARROW_SKIP8) {
-                if (!mbar_wait(skip_bar, (uint32_t)(t & 1), &sh->abort_flag)) {
+            if (SKIP8) {
+                if (!mbar_wait_warp(skip_bar, (uint32_t)(mine & 1), &sh->abort_flag, lane)) {
                     give_up(sh, u.status, 5);
                     break;
                 }
             }
             const long long m = (long long)m_tile * BLOCK_M + quad * 32 + lane;
             const bool row_ok = m < u.m_total;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.block_n + col_lo);
 
-            for (int pc = 0; pc < ncols; pc += pcols) {
-                // the previous TMA store must have finished reading the staging buffer
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                __syncwarp();
-                for (int cc = 0; cc < pcols; cc += 16) {
-                    const int lc0 = pc + cc;                           // column within this warp's range
-                    uint32_t acc[16];
-                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.block_n + col_lo + lc0), acc);
-                    const int co0 = n0 + lc0;
-                    uint4 sk8 = make_uint4(0, 0, 0, 0);
-                    int4 sk32[4];
-                    if (EPI == EPI_NARROW_SKIP8) {
-                        const unsigned chunk = (unsigned)(cc >> 4);
-                        sk8 = *(const uint4 *)(sbuf + (size_t)(pc / pcols) * 32 * u.piece_bytes + row_off + ((chunk ^ row_swz) << 4));
-                    } else if ((EPI == EPI_NARROW_SKIPWIDE || EPI == EPI_WIDE) && row_ok && co0 < a.c_out) {
-                        if (a.skip_dtype == ICONV_I32) {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g)
-                                if (co0 + 4 * g < a.c_out)
-                                    sk32[g] = __ldg((const int4 *)((const int32_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0) + g);
-                        } else if (a.skip_dtype >= 0) {
-                            sk8 = __ldg((const uint4 *)((const uint8_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0));
-                        }
+            for (int pc = 0; pc < ncols; pc += pcols, ++pieces) {
+                uint8_t *ob = obuf + (size_t)(pieces & 1) * piece_smem;
+                // the store issued two pieces ago must have finished reading this buffer
+                if (pieces >= 2) {
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                }
+                for (int cc = 0; cc < pcols; cc += 32) {
+                    int acc[32];
+                    const bool two = cc + 16 < pcols;
+                    tmem_ld16(t_row + (uint32_t)(pc + cc), acc);
+                    if (two) tmem_ld16(t_row + (uint32_t)(pc + cc + 16), acc + 16);
+                    uint4 sk[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+                    if (SKIP8) {
+                        const uint8_t *sp = sbuf + (size_t)(pc / pcols) * piece_smem + row_off;
+                        sk[0] = *(const uint4 *)(sp + (((unsigned)(cc >> 4) ^ row_swz) << 4));
+                        if (two) sk[1] = *(const uint4 *)(sp + (((unsigned)((cc >> 4) + 1) ^ row_swz) << 4));
                     }
                     tmem_ld_wait();
-                    const unsigned skw[4] = {sk8.x, sk8.y, sk8.z, sk8.w};
-                    unsigned packed[4];
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const int4 b4 = *(const int4 *)(wp->bias + lc0 + 4 * g);
-                        const int bias4[4] = {b4.x, b4.y, b4.z, b4.w};
-                        int mul4[4] = {q_mul, q_mul, q_mul, q_mul}, shift4[4] = {q_shift, q_shift, q_shift, q_shift};
-                        int h4[4] = {q_h_i, q_h_i, q_h_i, q_h_i};
-                        if (EPI != EPI_RAW && a.per_channel) {
-                            const int4 m4 = *(const int4 *)(wp->mul + lc0 + 4 * g);
-                            const int4 s4 = *(const int4 *)(wp->shift + lc0 + 4 * g);
-                            const int4 hh = *(const int4 *)(wp->h_i + lc0 + 4 * g);
-                            mul4[0] = m4.x; mul4[1] = m4.y; mul4[2] = m4.z; mul4[3] = m4.w;
-                            shift4[0] = s4.x; shift4[1] = s4.y; shift4[2] = s4.z; shift4[3] = s4.w;
-                            h4[0] = hh.x; h4[1] = hh.y; h4[2] = hh.z; h4[3] = hh.w;
-                        }
-                        const int s32v[4] = {sk32[g].x, sk32[g].y, sk32[g].z, sk32[g].w};
-                        int V[4];
+                    for (int hf = 0; hf < 2; ++hf) {
+                        if (hf == 1 && !two) break;
+                        int V[16];
+                        epilogue16<EPI>(acc + 16 * hf, V, n0 + pc + cc + 16 * hf, m, row_ok, sk[hf], a, u);
+                        if (esz_rt == 4) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int k = 4 * g + e;
-                            int sv = 0;   // skip value in the integer domain of the addition
-                            if (EPI == EPI_NARROW_SKIP8 || EPI == EPI_NARROW_SKIPWIDE || EPI == EPI_WIDE) {
-                                if (a.skip_dtype == ICONV_I32) {
-                                    sv = s32v[e];
-                                } else {
-                                    const unsigned byte = (skw[g] >> (8 * e)) & 0xffu;
-                                    sv = a.skip_dtype == ICONV_S8 ? (int)(int8_t)byte
-                                                                  : (int)byte - (a.skip_dtype == ICONV_U8_RAW128 ? 128 : 0);
-                                }
+                            for (int g = 0; g < 4; ++g) {
+                                const unsigned chunk = (unsigned)(((cc + 16 * hf) >> 2) + g);     // 4 columns = 16 bytes
+                                *(int4 *)(ob + row_off + ((chunk ^ row_swz) << 4)) = make_int4(V[4 * g], V[4 * g + 1], V[4 * g + 2], V[4 * g + 3]);
                             }
-                            if (EPI == EPI_RAW) {
-                                V[e] = (int)acc[k] + bias4[e];
-                            } else if (EPI == EPI_NARROW_NOSKIP || EPI == EPI_NARROW_SKIP8) {
-                                // every intermediate is proven at plan time to fit 32 bits
-                                int y = (int)acc[k] + bias4[e];
-                                if (EPI == EPI_NARROW_SKIP8) y += (sv * a.skip_mul + u.skip_half) >> a.skip_shift;
-                                y = max(min(y, h4[e]), 0);
-                                const unsigned v = ((unsigned)y * (unsigned)mul4[e] + (1u << (shift4[e] - 1))) >> shift4[e];
-                                V[e] = min(max((int)v + a.out_zero, a.out_lo), a.out_hi);
-                            } else if (EPI == EPI_NARROW_SKIPWIDE) {
-                                long long Y = (long long)(int)acc[k] + bias4[e] + round_shift64((long long)sv * a.skip_mul, a.skip_shift);
-                                Y = Y < 0 ? 0 : (Y > (long long)h4[e] ? (long long)h4[e] : Y);
-                                const unsigned v = ((unsigned)Y * (unsigned)mul4[e] + (1u << (shift4[e] - 1))) >> shift4[e];
-                                V[e] = min(max((int)v + a.out_zero, a.out_lo), a.out_hi);
-                            } else {
-                                long long Y = (long long)(int)acc[k] + bias4[e];
-                                if (a.skip_dtype >= 0) Y += round_shift64((long long)sv * a.skip_mul, a.skip_shift);
-                                V[e] = a.out_dtype == ICONV_I32
-                                           ? (int)Y
-                                           : requant_tail(Y, a.brelu, h4[e], mul4[e], shift4[e], a.out_zero, a.out_lo, a.out_hi);
-                            }
-                        }
-                        if (a.out_dtype == ICONV_I32) {
-                            const unsigned chunk = (unsigned)((cc >> 2) + g);          // 4 columns = 16 bytes
-                            *(int4 *)(obuf + row_off + ((chunk ^ row_swz) << 4)) = make_int4(V[0], V[1], V[2], V[3]);
                         } else {
-                            packed[g] = (V[0] & 0xff) | ((V[1] & 0xff) << 8) | ((V[2] & 0xff) << 16) | ((unsigned)(V[3] & 0xff) << 24);
+                            uint4 o;
+                            if (EPI == EPI_FAST || EPI == EPI_FAST_SKIP8 || a.out_dtype == ICONV_U8) {
+                                o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
+                                o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
+                            } else {
+                                o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
+                                o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
+                            }
+                            const unsigned chunk = (unsigned)((cc >> 4) + hf);
+                            *(uint4 *)(ob + row_off + ((chunk ^ row_swz) << 4)) = o;
                         }
-                    }
-                    if (a.out_dtype != ICONV_I32) {
-                        const unsigned chunk = (unsigned)(cc >> 4);
-                        *(uint4 *)(obuf + row_off + ((chunk ^ row_swz) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     }
                 }
                 // hand the staged piece to the TMA unit (the store clips rows beyond the last
@@ -471,7 +649,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 __syncwarp();
                 if (lane == 0) {
                     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                 ::"l"(&tmap_out), "r"(smem_u32(obuf)), "r"(n0 + pc), "r"(m_tile * BLOCK_M + quad * 32)
+                                 ::"l"(&tmap_out), "r"(smem_u32(ob)), "r"(n0 + pc), "r"(m_tile * BLOCK_M + quad * 32)
                                  : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
@@ -480,22 +658,15 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
-                const int next = tile + gridDim.x;
-                if (EPI == EPI_NARROW_SKIP8 && next < num_tiles) {     // prefetch the next tile's skip rows
+                const int next = tile + tile_step;
+                if (SKIP8 && next < num_tiles) {     // prefetch the next tile's skip rows
+                    const int mtn = (int)fast_div((unsigned)next, u.div_nt_mul, u.div_nt_shr);
                     mbar_expect_tx(skip_bar, (uint32_t)(32 * ncols));
                     for (int c = 0; c < ncols; c += pcols)
-                        tma_load_2d(smem_u32(sbuf + (size_t)(c / pcols) * 32 * u.piece_bytes), &tmap_skip, skip_bar,
-                                    (next % u.n_tiles) * u.block_n + col_lo + c, (next / u.n_tiles) * BLOCK_M + quad * 32);
+                        tma_load_2d(smem_u32(sbuf + (size_t)(c / pcols) * piece_smem), &tmap_skip, skip_bar,
+                                    (next - mtn * u.n_tiles) * u.block_n + col_lo + c, mtn * BLOCK_M + quad * 32);
                     ++skip_issued;
                 }
-            }
-        }
-        // a warp with no columns still has to release the accumulators it never reads
-        if (ncols <= 0) {
-            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
-                const int buf = t & 1;
-                if (!mbar_wait(smem_u32(&sh->tmem_full[buf]), (uint32_t)((t >> 1) & 1), &sh->abort_flag)) break;
-                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
             }
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -510,6 +681,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // nothing touches this CTA's shared memory or TMEM after it returns.
         volatile int never = 0;
         if (warp == 0 && lane == 0) {
+            if (b_issued) mbar_wait(smem_u32(&sh->b_full), 0, &never);
             for (int s = 0; s < u.stages; ++s) {
                 int last = -1;
                 for (int i = issued - 1; i >= 0 && i >= issued - u.stages; --i)
@@ -521,7 +693,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             umma_commit(smem_u32(&sh->drain));
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }
-        if (warp >= 2 && lane == 0 && skip_issued > 0)
+        if (warp >= 2 && warp < 2 + u.epi_warps && lane == 0 && skip_issued > 0)
             mbar_wait(smem_u32(&sh->skip_full[warp - 2]), (uint32_t)((skip_issued - 1) & 1), &never);
         __syncthreads();
     }
@@ -559,6 +731,18 @@ int load_driver_entry_points()
     return ICONV_OK;
 }
 
+// Multiplier and shift with umulhi(x, mul) >> shr == x / d for every 0 <= x < 2^31
+// (mul == 0 stands for d == 1): mul = ceil(2^(31 + ceil(log2 d)) / d) fits 32 bits.
+void find_divisor(unsigned d, unsigned &mul, unsigned &shr)
+{
+    if (d <= 1) { mul = 0; shr = 0; return; }
+    unsigned lg = 0;
+    while ((1ull << lg) < d) ++lg;
+    const unsigned long long pw = 1ull << (31 + lg);
+    mul = (unsigned)((pw + d - 1) / d);
+    shr = lg - 1;
+}
+
 CUtensorMapSwizzle swizzle_of(int kc)
 {
     return kc == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (kc == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
@@ -586,32 +770,72 @@ int encode_activation_map(const iconv_plan_t *p, const void *x, CUtensorMap *map
     return ICONV_OK;
 }
 
-}  // namespace
+long long labs64(long long v) { return v < 0 ? -v : v; }
 
-// Picks the cheapest epilogue whose 32-bit arithmetic is provably exact for this layer.
-// After the BReLU clamp 0 <= Y <= h_i, so Y * mul + 2^(shift-1) fits an unsigned 32-bit
-// word whenever h_i * mul + 2^(shift-1) < 2^32; an 8-bit skip's rescale fits a signed word
-// whenever 255 * skip_mul + 2^(skip_shift-1) < 2^31.
-static int choose_epilogue(const iconv_desc &d)
+// Picks the cheapest epilogue whose 32-bit arithmetic is provably exact for this layer and
+// fills the per-channel additive constant of that variant (c_a, c_out_pad entries).
+//   worst[co] = sum |w| * max|x|: no accumulator of channel co can exceed it in magnitude.
+int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_a, int &tail)
 {
+    const long long K = (long long)d.kh * d.kw * d.c_in;
+    const long long xmax = d.in_dtype == ICONV_U8 ? 255 : 128;
+    c_a.assign((size_t)c_out_pad, 0);
+    for (int co = 0; co < d.c_out; ++co) c_a[co] = d.bias[co];
+    tail = 1;
     if (d.out_dtype == ICONV_I32) return d.skip_dtype < 0 ? EPI_RAW : EPI_WIDE;
     if (!d.brelu) return EPI_WIDE;
     const int np = d.per_channel ? d.c_out : 1;
+    bool tail_free = d.out_zero == 0 && d.out_lo <= 0;
     for (int i = 0; i < np; ++i) {
         if (d.shift[i] < 1 || d.shift[i] > 31) return EPI_WIDE;
-        if ((unsigned long long)d.h_i[i] * (unsigned long long)d.mul[i] + (1ull << (d.shift[i] - 1)) >= (1ull << 32)) return EPI_WIDE;
+        const unsigned long long top = (unsigned long long)d.h_i[i] * (unsigned long long)d.mul[i] + (1ull << (d.shift[i] - 1));
+        if (top >= (1ull << 32)) return EPI_WIDE;
+        if ((long long)(top >> d.shift[i]) > d.out_hi) tail_free = false;
     }
-    if (d.skip_dtype < 0) return EPI_NARROW_NOSKIP;
-    if (d.skip_dtype != ICONV_I32 && d.skip_shift <= 30 &&
-        255ll * d.skip_mul + (d.skip_shift ? (1ll << (d.skip_shift - 1)) : 0) < (1ll << 31))
-        return EPI_NARROW_SKIP8;
-    return EPI_NARROW_SKIPWIDE;
+    tail = tail_free ? 0 : 1;
+
+    const bool skip8 = d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32;
+    long long skip_bound = 0;      // bound of |rescaled skip|
+    if (skip8) {
+        // t = s * skip_mul + C, C = (b << skip_shift) + half - z * skip_mul, must fit int32 for every byte s
+        if (d.skip_shift > 30) return EPI_WIDE;
+        const long long z = d.skip_dtype == ICONV_U8 ? 0 : 128;
+        const long long half = d.skip_shift ? (1ll << (d.skip_shift - 1)) : 0;
+        for (int co = 0; co < d.c_out; ++co) {
+            const long long C = ((long long)d.bias[co] << d.skip_shift) + half - z * d.skip_mul;
+            if (labs64(C) + 255ll * d.skip_mul >= (1ll << 31)) return EPI_WIDE;
+            c_a[co] = (int32_t)C;
+        }
+        skip_bound = ((255ll * d.skip_mul) >> d.skip_shift) + 1;
+    }
+    // the fast form: no clamp before the multiplication, the u8 saturation does both clamps
+    bool fast = !d.per_channel && d.out_dtype == ICONV_U8 && d.out_zero == 0 && d.out_lo == 0 && d.out_hi == 255 &&
+                d.skip_dtype != ICONV_I32;
+    if (fast) {
+        const long long mul = d.mul[0], half = 1ll << (d.shift[0] - 1);
+        // BReLU's upper clamp may only be dropped when h_i already maps to the saturation bound
+        if ((long long)(((unsigned long long)d.h_i[0] * (unsigned long long)mul + (unsigned long long)half) >> d.shift[0]) < 255) fast = false;
+        for (int co = 0; co < d.c_out && fast; ++co) {
+            long long sw = 0;
+            const int8_t *wr = d.weights + (long long)co * K;
+            for (long long k = 0; k < K; ++k) sw += wr[k] < 0 ? -(long long)wr[k] : wr[k];
+            const long long ymax = sw * xmax + labs64(d.bias[co]) + skip_bound;
+            if (ymax * mul + half >= (1ll << 31)) fast = false;
+        }
+        if (fast) {
+            if (!skip8)
+                for (int co = 0; co < d.c_out; ++co) c_a[co] = (int32_t)((long long)d.bias[co] * mul + half);
+            return skip8 ? EPI_FAST_SKIP8 : EPI_FAST;
+        }
+    }
+    if (d.skip_dtype < 0) return EPI_SAFE;
+    return skip8 ? EPI_SAFE_SKIP8 : EPI_SAFE_SKIP32;
 }
 
 // Tiled 2-D map over a channel slice of an NHWC tensor seen as [pixels][channels]; the box
 // is one staged piece: 32 pixels x piece_bytes.
-static int encode_rows_map(const void *base, int elem_bytes, int c_slice, int c_total, long long pixels,
-                           int piece_bytes, CUtensorMap *map)
+int encode_rows_map(const void *base, int elem_bytes, int c_slice, int c_total, long long pixels,
+                    int piece_bytes, CUtensorMap *map)
 {
     const cuuint64_t dims[2] = {(cuuint64_t)c_slice, (cuuint64_t)pixels};
     const cuuint64_t strides[1] = {(cuuint64_t)c_total * elem_bytes};
@@ -630,6 +854,8 @@ static int encode_rows_map(const void *base, int elem_bytes, int c_slice, int c_
     return ICONV_OK;
 }
 
+}  // namespace
+
 int umma_supported(const iconv_plan_t *p)
 {
     const iconv_desc &d = p->d;
@@ -643,6 +869,7 @@ int umma_supported(const iconv_plan_t *p)
     else if (d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && (d.skip_c_total % 16 || d.skip_c_offset % 16)) why = "8-bit skip channels must be multiples of 16";
     else if (d.kh > 16 || d.kw > 16 || d.pad > 16 || d.stride > 8) why = "filter, padding or stride beyond the im2col descriptor's range";
     else if ((long long)d.kh * d.kw * ((d.c_in + 127) / 128 * 128) >= (1ll << 24)) why = "reduction too long";
+    else if ((long long)d.n * p->h_out * p->w_out >= (1ll << 31) - 256) why = "more than 2^31 output pixels";
     if (why) {
         set_error("tensor-core path: %s", why);
         return ICONV_ERR_UNSUPPORTED;
@@ -669,25 +896,54 @@ int umma_setup(iconv_plan_t *p)
     const int n_tiles = (d.c_out + 255) / 256;
     p->block_n = ((d.c_out + n_tiles - 1) / n_tiles + 15) / 16 * 16;
     p->c_out_pad = p->block_n * n_tiles;
-    // epilogue split: the two warps of a TMEM lane quadrant take the two halves of the tile's
-    // columns; a staged piece is the widest power of two (up to 128 bytes) dividing both
-    p->half_n = (p->block_n / 2 + 15) / 16 * 16;
+    const int taps = d.kh * d.kw;
+    const int k_iters = taps * (p->c_in_pad / p->kc);
+    const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
+
+    // accumulator buffers: four when a tile has at most 128 columns, else two
+    p->nbuf = p->block_n <= 128 ? 4 : 2;
+
+    // shared-memory budget: pipeline stages (+ the resident filter bank) against the
+    // epilogue warps' staging.  Sixteen epilogue warps unless that leaves the pipeline short.
+    const int stage_a = BLOCK_M * p->kc;
+    const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
+    const long long bank = (long long)b_tile * k_iters * n_tiles;
+    const int fixed = (int)sizeof(Shared) + 2048;
+    p->resident_b = 0;
+    p->epi_warps = 0;
+    for (int ew = 16; ew >= 8 && !p->epi_warps; ew -= 8) {
+        const int avail = MAX_SMEM - fixed - ew * EPI_WARP_SMEM;
+        const int want = k_iters >= 4 ? 4 : (k_iters >= 2 ? 2 : 2);
+        if (bank <= RESIDENT_B_MAX && avail - (int)bank >= want * stage_a) {
+            p->resident_b = 1;
+            p->stages = (avail - (int)bank) / stage_a;
+            p->epi_warps = ew;
+        } else if (avail >= want * (stage_a + b_tile) || ew == 8) {
+            p->stages = avail / (stage_a + b_tile);
+            p->epi_warps = ew;
+        }
+    }
+    if (p->stages > MAX_STAGES) p->stages = MAX_STAGES;
+    if (p->stages < 2) { set_error("tensor-core path: tile does not fit shared memory"); return ICONV_ERR_UNSUPPORTED; }
+
+    // epilogue geometry: slots per TMEM lane quadrant, split between a tile's columns (cs)
+    // and tiles in flight (bi)
+    const int slots = p->epi_warps / 4;
+    p->cs = p->block_n > 128 ? 2 : 1;
+    p->bi = slots / p->cs;
+    if (p->bi > p->nbuf) p->bi = p->nbuf;
+    p->epi_warps = 4 * p->cs * p->bi;
+    p->half_n = p->cs == 2 ? (p->block_n / 2 + 15) / 16 * 16 : p->block_n;
     {
-        const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
-        const int w0 = p->half_n * esz, w1 = (p->block_n - p->half_n) * esz;
-        int pb = 128;
+        // staged piece: the widest power of two dividing every warp's row width, at most 64
+        // bytes of 8-bit outputs or 128 bytes of int32 (two pieces fit half the warp's staging)
+        const int w0 = p->half_n * esz, w1 = (p->block_n - (p->cs - 1) * p->half_n) * esz;
+        int pb = esz == 4 ? 128 : 64;
         while (pb > 16 && (w0 % pb || w1 % pb)) pb /= 2;
         p->piece_bytes = pb;
     }
-    const int stage_a = BLOCK_M * p->kc;
-    const int stage_b = (p->block_n * p->kc + 1023) / 1024 * 1024;
-    int stages = SMEM_BUDGET / (stage_a + stage_b);
-    if (stages > MAX_STAGES) stages = MAX_STAGES;
-    if (stages < 2) { set_error("tensor-core path: tile does not fit shared memory"); return ICONV_ERR_UNSUPPORTED; }
-    p->stages = stages;
 
     // repack weights [c_out][tap][c_in] -> [c_out_pad][tap][c_in_pad], zero filled
-    const int taps = d.kh * d.kw;
     const size_t k_pad = (size_t)taps * p->c_in_pad;
     std::vector<int8_t> packed((size_t)p->c_out_pad * k_pad, 0);
     for (int co = 0; co < d.c_out; ++co)
@@ -712,14 +968,33 @@ int umma_setup(iconv_plan_t *p)
     CUtensorMap probe;
     rc = encode_activation_map(p, (const uint8_t *)p->w_packed - d.in_c_offset, &probe);
     if (rc != ICONV_OK) return rc;
-    p->epi = choose_epilogue(d);
+
+    // epilogue variant and its per-channel constants: {c_a, mul, shift, h_i} x c_out_pad
+    std::vector<int32_t> c_a;
+    p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail);
+    std::vector<int32_t> par((size_t)4 * p->c_out_pad, 0);
+    for (int co = 0; co < p->c_out_pad; ++co) {
+        const int q = d.per_channel && co < d.c_out ? co : 0;
+        par[co] = c_a[co];
+        par[(size_t)p->c_out_pad + co] = d.out_dtype != ICONV_I32 ? d.mul[q] : 1;
+        par[(size_t)2 * p->c_out_pad + co] = d.out_dtype != ICONV_I32 ? d.shift[q] : 1;
+        par[(size_t)3 * p->c_out_pad + co] = d.out_dtype != ICONV_I32 ? d.h_i[q] : 0;
+    }
+    ICONV_CUDA_TRY(cudaMalloc((void **)&p->params_packed, par.size() * sizeof(int32_t)));
+    ICONV_CUDA_TRY(cudaMemcpy(p->params_packed, par.data(), par.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    p->q_mul = d.out_dtype != ICONV_I32 ? d.mul[0] : 1;
+    p->q_shift = d.out_dtype != ICONV_I32 ? d.shift[0] : 0;
+    p->q_h = d.out_dtype != ICONV_I32 ? d.h_i[0] : 0;
+
     static bool attr_set = false;
     if (!attr_set) {
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_NARROW_NOSKIP>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_NARROW_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_NARROW_SKIPWIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         attr_set = true;
     }
     return ICONV_OK;
@@ -746,10 +1021,19 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.taps = d.kh * d.kw;
     u.stages = p->stages;
     u.stage_a_bytes = BLOCK_M * p->kc;
-    u.stage_bytes = u.stage_a_bytes + (p->block_n * p->kc + 1023) / 1024 * 1024;
+    u.b_tile_bytes = (p->block_n * p->kc + 1023) / 1024 * 1024;
+    u.resident_b = p->resident_b;
+    u.stage_bytes = u.stage_a_bytes + (p->resident_b ? 0 : u.b_tile_bytes);
+    u.nbuf = p->nbuf;
+    u.lg_nbuf = p->nbuf == 4 ? 2 : 1;
     int cols = 32;
-    while (cols < 2 * p->block_n) cols *= 2;
+    while (cols < p->nbuf * p->block_n) cols *= 2;
     u.tmem_cols = cols;
+    u.epi_warps = p->epi_warps;
+    u.cs = p->cs;
+    u.bi = p->bi;
+    u.part_n = p->half_n;
+    u.piece_bytes = p->piece_bytes;
     // instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, N/8, M/16
     u.idesc = (2u << 4) | ((d.in_dtype == ICONV_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(p->block_n >> 3) << 17) |
               ((unsigned)(BLOCK_M >> 4) << 24);
@@ -757,36 +1041,57 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     // units), descriptor version 1, swizzle mode (128B = 2, 64B = 4, 32B = 6)
     const unsigned long long layout = p->kc == 128 ? 2ull : (p->kc == 64 ? 4ull : 6ull);
     u.desc_hi = ((unsigned long long)((8 * p->kc) >> 4) << 32) | (1ull << 46) | (layout << 61);
-    u.half_n = p->half_n;
-    u.piece_bytes = p->piece_bytes;
+    u.q_mul = p->q_mul;
+    u.q_shift = p->q_shift;
+    u.q_half = p->q_shift > 0 && p->q_shift <= 31 ? (int)(1u << (p->q_shift - 1)) : 0;
+    u.q_h = p->q_h;
+    u.skip_half = (d.skip_dtype >= 0 && d.skip_shift > 0 && d.skip_shift <= 31) ? (int)(1u << (d.skip_shift - 1)) : 0;
+    u.skip_xor = d.skip_dtype == ICONV_S8 ? 0x80808080u : 0u;
+    u.tail = p->tail;
+    u.c_a = p->params_packed;
+    u.c_mul = p->params_packed + p->c_out_pad;
+    u.c_shift = p->params_packed + 2 * (size_t)p->c_out_pad;
+    u.c_h = p->params_packed + 3 * (size_t)p->c_out_pad;
     const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
     CUtensorMap tmap_out, tmap_skip;
     rc = encode_rows_map((uint8_t *)a.out + (size_t)d.out_c_offset * esz, esz, d.c_out, d.out_c_total, u.m_total,
                          p->piece_bytes, &tmap_out);
     if (rc != ICONV_OK) return rc;
     tmap_skip = tmap_out;
-    if (p->epi == EPI_NARROW_SKIP8) {
+    if (p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8) {
         rc = encode_rows_map((const uint8_t *)a.skip + d.skip_c_offset, 1, d.c_out, d.skip_c_total, u.m_total,
                              p->piece_bytes, &tmap_skip);
         if (rc != ICONV_OK) return rc;
     }
+    find_divisor((unsigned)u.n_tiles, u.div_nt_mul, u.div_nt_shr);
+    find_divisor((unsigned)p->w_out, u.div_w_mul, u.div_w_shr);
+    find_divisor((unsigned)(p->h_out * p->w_out), u.div_hw_mul, u.div_hw_shr);
     u.status = device_status_ptr();
     if (!u.status) { set_error("device status word not available"); return ICONV_ERR_CUDA; }
 
-    int dev = 0, sms = 0;
-    ICONV_CUDA_TRY(cudaGetDevice(&dev));
-    ICONV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        ICONV_CUDA_TRY(cudaGetDevice(&dev));
+        ICONV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    }
     const long long tiles = (long long)u.m_tiles * u.n_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    const size_t smem = (size_t)u.stages * u.stage_bytes + sizeof(Shared) + 2048 + EPI_SMEM;
-    u.skip_half = (d.skip_dtype >= 0 && d.skip_shift > 0 && d.skip_shift <= 31) ? (int)(1u << (d.skip_shift - 1)) : 0;
+    const size_t smem = 1024 + (size_t)u.stages * u.stage_bytes +
+                        (p->resident_b ? (size_t)u.b_tile_bytes * u.taps * u.cchunks * u.n_tiles : 0) + sizeof(Shared) + 1024 +
+                        (size_t)p->epi_warps * EPI_WARP_SMEM;
+    if (smem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
+#define ICONV_LAUNCH(E) umma_conv_kernel<E><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u)
     switch (p->epi) {
-    case EPI_RAW: umma_conv_kernel<EPI_RAW><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u); break;
-    case EPI_NARROW_NOSKIP: umma_conv_kernel<EPI_NARROW_NOSKIP><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u); break;
-    case EPI_NARROW_SKIP8: umma_conv_kernel<EPI_NARROW_SKIP8><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u); break;
-    case EPI_NARROW_SKIPWIDE: umma_conv_kernel<EPI_NARROW_SKIPWIDE><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u); break;
-    default: umma_conv_kernel<EPI_WIDE><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u); break;
+    case EPI_RAW: ICONV_LAUNCH(EPI_RAW); break;
+    case EPI_FAST: ICONV_LAUNCH(EPI_FAST); break;
+    case EPI_FAST_SKIP8: ICONV_LAUNCH(EPI_FAST_SKIP8); break;
+    case EPI_SAFE: ICONV_LAUNCH(EPI_SAFE); break;
+    case EPI_SAFE_SKIP8: ICONV_LAUNCH(EPI_SAFE_SKIP8); break;
+    case EPI_SAFE_SKIP32: ICONV_LAUNCH(EPI_SAFE_SKIP32); break;
+    default: ICONV_LAUNCH(EPI_WIDE); break;
     }
+#undef ICONV_LAUNCH
     ICONV_CUDA_TRY(cudaGetLastError());
     return ICONV_OK;
 }

@@ -20,7 +20,12 @@ struct iconv_plan_s {
     CUtensorMap tmap_w;      // 2-D tiled map over the packed weights
     int block_n = 0, kc = 0, c_in_pad = 0, c_out_pad = 0, stages = 0, swizzle_bytes = 0;
     int epi = 0;             // epilogue variant of the tensor-core kernel
-    int half_n = 0, piece_bytes = 0;   // epilogue column split and staged piece width
+    int half_n = 0, piece_bytes = 0;   // columns per epilogue warp and staged piece width
+    int nbuf = 2;            // TMEM accumulator buffers
+    int resident_b = 0;      // 1: the packed filter bank stays in shared memory for the whole kernel
+    int epi_warps = 8, cs = 1, bi = 1;   // epilogue warps; column split per tile; tiles in flight
+    int tail = 1;            // 0: zero point and output range are provably no-ops
+    int q_mul = 1, q_shift = 0, q_h = 0; // per-layer Eq. 4 / BReLU scalars
     // stem path: repacked image (plan-owned scratch) and the plan of the GEMM that follows
     iconv_plan_s *inner = nullptr;
     void *workspace = nullptr;
