@@ -223,12 +223,14 @@ def main():
             fam_macs[fam] = fam_macs.get(fam, 0) + macs.get(name, 0)
             layer_ms[name] = layer_ms.get(name, 0.0) + dt / args.steps
     int8_peak, hbm_peak, peak_kind = measured_peaks()
+    issue_tops, issue_cycles = B.iconv_probe_mma_rate(256, 100000)     # outside every timed region
     umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
     roofline = {"kernel": "umma_conv_kernel", "bound": "tensor", "achieved": umma_tops, "peak": int8_peak,
                 "unit": "TOP/s", "frac": umma_tops / int8_peak, "traffic": None, "peak_kind": peak_kind + " 2 x bf16 sustained",
                 "launches": umma_launches, "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
                 "frac_of_nominal_4500": umma_tops / NOMINAL_INT8_TOPS,
+                "issue_rate_peak": issue_tops, "frac_of_issue_rate_peak": umma_tops / issue_tops,
                 "time_share": {k: v / sum(fam_ms.values()) for k, v in fam_ms.items()}}
 
     # ---- end to end: pinned host input in, logits out, every step ----

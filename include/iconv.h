@@ -175,6 +175,14 @@ ICONV_API int iconcat_plan(int32_t n_branches, const double *ratio_y, const doub
                  int32_t shift_min, int32_t *mul, int32_t *shift,
                  double *delta_scale, double *ratio_y_new, double *ratio_v_min);
 
+/* Measurement aid: how fast this GPU's tensor pipe retires tcgen05.mma kind::i8 (M = 128,
+ * N = block_n, K = 32, u8 x s8 -> s32, the instruction of the convolution kernel) when only the
+ * instruction stream limits it: operands stay in shared memory, one thread per SM issues `iters`
+ * dependent instructions.  Returns whole-GPU TOP/s (2 * MACs / event time of the launch) and the
+ * slowest SM's cycles per instruction.  Synchronous; allocates a few KB on the current device.
+ * The paper has no counterpart: its GPU had no tensor cores. */
+ICONV_API int iconv_probe_mma_rate(int32_t block_n, int32_t iters, double *tops, double *cycles_per_mma);
+
 /* Text of the calling thread's last error (never NULL; valid until its next failing call). */
 ICONV_API const char *iconv_last_error(void);
 

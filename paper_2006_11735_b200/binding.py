@@ -17,7 +17,8 @@ KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin"
 
 EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_forward", "iconv_check",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
-           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iconcat_plan", "iconv_last_error")
+           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iconcat_plan", "iconv_probe_mma_rate",
+           "iconv_last_error")
 
 
 class IconvError(RuntimeError):
@@ -63,6 +64,7 @@ def _load():
     lib.iq_brelu_params.argtypes = [dbl, dbl, i32, i32, P(i32), P(i32), P(i32), P(i32), P(dbl), P(dbl)]
     lib.iq_skip_sync.argtypes = [dbl, dbl, i32, P(i32), P(i32), P(dbl), P(dbl)]
     lib.iconcat_plan.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, P(dbl)]
+    lib.iconv_probe_mma_rate.argtypes = [i32, i32, P(dbl), P(dbl)]
     lib.iconv_last_error.restype = C.c_char_p
     for name in EXPORTS:
         if name != "iconv_last_error":
@@ -191,3 +193,10 @@ def iconcat_plan(ratio_y, ratio_v, shift_min: int = 16):
                             scale.ctypes.data, ry_new.ctypes.data, C.byref(rmin)))
     return dict(ratio_V_min=rmin.value, mul=mul.tolist(), shift=shift.tolist(), delta_scale=scale.tolist(),
                 ratio_Y_new=ry_new.tolist())
+
+
+def iconv_probe_mma_rate(block_n: int = 256, iters: int = 200000):
+    """(whole-GPU int8 TOP/s, cycles per instruction) of back-to-back tcgen05.mma kind::i8."""
+    tops, cyc = C.c_double(), C.c_double()
+    _check(lib.iconv_probe_mma_rate(block_n, iters, C.byref(tops), C.byref(cyc)))
+    return tops.value, cyc.value

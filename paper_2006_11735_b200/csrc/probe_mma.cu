@@ -1,0 +1,121 @@
+// Issue-rate probe of tcgen05.mma kind::i8: what the tensor pipe of this GPU sustains when
+// nothing but the instruction stream limits it (operands resident in shared memory, one
+// issuing thread per SM, every instruction accumulating into the same TMEM tile).  The
+// convolution kernel's achieved TOP/s is reported against this figure as well as against
+// the nominal one.
+#include <algorithm>
+#include <vector>
+
+#include "plan.h"
+
+namespace iconv {
+
+namespace {
+
+__device__ __forceinline__ uint32_t probe_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+struct ProbeResult {
+    long long cycles;
+    int timed_out;
+    int pad;
+};
+
+__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int iters, ProbeResult *res)
+{
+    extern __shared__ uint8_t probe_raw[];
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)probe_raw + 1023) & ~(uintptr_t)1023);   // A: 16 KB, B: 32 KB
+    __shared__ unsigned long long bar;
+    __shared__ uint32_t tmem_base;
+    for (int i = threadIdx.x; i < (16384 + 32768) / 4; i += blockDim.x) ((uint32_t *)tiles)[i] = 0x01010101u;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(probe_smem_u32(&bar)), "r"(1));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(probe_smem_u32(&tmem_base)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tb = tmem_base;
+    if (threadIdx.x == 0) {
+        // K-major tiles with 128-byte rows and the 128-byte swizzle, as the convolution kernel stages them
+        const unsigned long long hi = ((unsigned long long)((8 * 128) >> 4) << 32) | (1ull << 46) | (2ull << 61);
+        const unsigned long long da = hi | (unsigned long long)((probe_smem_u32(tiles) & 0x3FFFFu) >> 4) | (1ull << 16);
+        const unsigned long long db = hi | (unsigned long long)((probe_smem_u32(tiles + 16384) & 0x3FFFFu) >> 4) | (1ull << 16);
+        const uint32_t idesc = (2u << 4) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((128u >> 4) << 24);   // u8 x s8 -> s32
+        const long long t0 = clock64();
+        for (int i = 0; i < iters; ++i) {
+            const unsigned long long k = 2ull * (unsigned)(i & 3);    // walk the four 32-byte K slices of a row
+            asm volatile(
+                "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                ::"r"(tb), "l"(da + k), "l"(db + k), "r"(idesc), "r"(i) : "memory");
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(probe_smem_u32(&bar)) : "memory");
+        int timed_out = 1;
+        for (long long spin = 0; spin < 200000000ll; ++spin) {     // bounded wait for the last MMA
+            uint32_t ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(probe_smem_u32(&bar)), "r"(0) : "memory");
+            if (ok) { timed_out = 0; break; }
+        }
+        res[blockIdx.x].cycles = clock64() - t0;
+        res[blockIdx.x].timed_out = timed_out;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tb), "r"(256) : "memory");
+    }
+}
+
+}  // namespace
+
+}  // namespace iconv
+
+using namespace iconv;
+
+extern "C" int iconv_probe_mma_rate(int32_t block_n, int32_t iters, double *tops, double *cycles_per_mma)
+{
+    if (!tops || !cycles_per_mma || iters < 1 || iters > (1 << 22) || block_n < 16 || block_n > 256 || block_n % 16) {
+        set_error("iconv_probe_mma_rate: need 16 <= block_n <= 256 (a multiple of 16) and 1 <= iters <= 2^22");
+        return ICONV_ERR_ARG;
+    }
+    int dev = 0, sms = 0;
+    ICONV_CUDA_TRY(cudaGetDevice(&dev));
+    ICONV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const size_t smem = 16384 + 32768 + 1024;
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(mma_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ProbeResult *d_res = nullptr;
+    ICONV_CUDA_TRY(cudaMalloc((void **)&d_res, sizeof(ProbeResult) * sms));
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    float ms = 0.f;
+    cudaError_t err = cudaEventCreate(&e0);
+    if (err == cudaSuccess) err = cudaEventCreate(&e1);
+    for (int rep = 0; rep < 2 && err == cudaSuccess; ++rep) {      // the first launch warms up
+        if (err == cudaSuccess) err = cudaEventRecord(e0, 0);
+        mma_rate_kernel<<<sms, 128, smem, 0>>>(block_n, iters, d_res);
+        if (err == cudaSuccess) err = cudaGetLastError();
+        if (err == cudaSuccess) err = cudaEventRecord(e1, 0);
+        if (err == cudaSuccess) err = cudaEventSynchronize(e1);
+    }
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e0, e1);
+    std::vector<ProbeResult> h((size_t)sms);
+    if (err == cudaSuccess) err = cudaMemcpy(h.data(), d_res, sizeof(ProbeResult) * sms, cudaMemcpyDeviceToHost);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(d_res);
+    if (err != cudaSuccess) return cuda_fail(err, "iconv_probe_mma_rate");
+    long long worst = 0;
+    for (const ProbeResult &r : h) {
+        if (r.timed_out) { set_error("iconv_probe_mma_rate: a bounded wait ran out"); return ICONV_ERR_TIMEOUT; }
+        worst = std::max(worst, r.cycles);
+    }
+    *cycles_per_mma = (double)worst / iters;
+    *tops = 2.0 * (double)sms * iters * 128.0 * block_n * 32.0 / (ms * 1e-3) / 1e12;
+    return ICONV_OK;
+}

@@ -232,3 +232,11 @@ def test_stem_path_matches_oracle(shape, in_dtype):
     assert 0.05 < (want == 0).mean() < 0.95
     got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=2, pad=3, in_dtype=in_dtype)
     assert fam == B.KERNEL_STEM and np.array_equal(got, want)      # AUTO picks it too
+
+
+def test_mma_issue_rate_probe_reports_a_plausible_peak():
+    tops, cycles = B.iconv_probe_mma_rate(256, 20000)
+    assert 100.0 <= cycles <= 400.0          # 128 cycles per M128 N256 K32 instruction at the nominal rate
+    assert 1000.0 < tops < 10000.0
+    with pytest.raises(B.IconvError):
+        B.iconv_probe_mma_rate(100, 10)
