@@ -124,8 +124,8 @@ ICONV_API int iconv_forward(const iconv_plan_t *plan, const void *x, const void 
 
 /*
  * Device-side waits (mbarrier phases) are bounded.  A kernel whose wait runs out records
- * it in a per-device status word and returns early.  iconv_check synchronises the stream
- * and returns ICONV_ERR_TIMEOUT if any kernel recorded one since the last call,
+ * a code (1-7) in a per-device status word and returns early.  iconv_check synchronises the
+ * stream and returns ICONV_ERR_TIMEOUT if any kernel recorded a code since the last call,
  * ICONV_ERR_CUDA on a CUDA error, ICONV_OK otherwise.
  */
 ICONV_API int iconv_check(void *cuda_stream);
@@ -151,6 +151,47 @@ ICONV_API int ipool_max(const void *x, void *out, int32_t n, int32_t h, int32_t 
               int32_t k, int32_t stride, int32_t pad, void *cuda_stream);
 ICONV_API int ipool_avg_requant(const void *x, void *out, int32_t n, int32_t h, int32_t w, int32_t c,
                       int32_t mul, int32_t shift, int32_t max_int, void *cuda_stream);
+
+/*
+ * iconv_stem_forward_static -- the 7x7 stride-2 pad-3 first layer over a 3-channel image, for
+ * callers that may not allocate device memory.  (The paper has no counterpart; this exists for
+ * the way the library is embedded.)  Code that runs under a framework's memory pool, inside a
+ * latency-critical serving loop or in a process whose device memory is fully budgeted up front
+ * cannot call cudaMalloc, yet iconv_plan does (weights, constants and, for this layer, a
+ * repacked copy of the image).  This entry point needs no plan and calls no cudaMalloc, cudaFree
+ * or allocating library routine: its working memory -- the repacked image, the rearranged
+ * weights and the epilogue constants -- is a fixed array of ICONV_STEM_STATIC_BYTES inside the
+ * library's device image, which every GPU that loads the library holds until the process exits.
+ *
+ *   x        DEVICE uint8 (or int8) [n][h][w][3], 16-byte aligned
+ *   weights  DEVICE int8 [c_out][7][7][3]
+ *   bias     DEVICE int32 [c_out], |b| <= 2^30 (a larger one is replaced by 0 and recorded in the
+ *            device status word as code 8, which the next iconv_check reports)
+ *   out      DEVICE uint8 [n][h_out][w_out][out_c_total], 16-byte aligned; only the slice
+ *            [out_c_offset, out_c_offset + c_out) of each pixel is written
+ *
+ * The arithmetic is iconv_forward's with brelu = 1 and per-layer mul / shift / h_i; results are
+ * bit-identical to a planned forward of the same layer.  Returns ICONV_ERR_SHAPE with the sizes in
+ * iconv_last_error() when n * (h_out + 3) * w_out * 64 + 131072 exceeds ICONV_STEM_STATIC_BYTES
+ * (40 images of 224 x 224 fit), ICONV_ERR_ARG unless c_out is a multiple of 16 in [16, 256],
+ * 1 <= shift <= 31 and h_i * mul + 2^(shift-1) < 2^32.  Asynchronous on cuda_stream.
+ *
+ * The first call on each device looks up the array's device address (the GPU with that array
+ * must be current); make that first call outside any stream capture.  All calls on a device share
+ * the one array, which keeps whatever the last call left in it; each call rewrites every byte it
+ * later reads, so nothing has to be cleared, but two calls that overlap on the GPU (different
+ * streams, or different host threads) race on it: serialise them.
+ */
+#define ICONV_STEM_STATIC_BYTES (32u * 1024u * 1024u)
+typedef struct {
+    int32_t n, h, w, c_out;
+    int32_t in_dtype;                  /* ICONV_U8 | ICONV_S8 | ICONV_U8_RAW128 */
+    int32_t out_c_total, out_c_offset;
+    int32_t mul, shift, h_i;           /* Eq. 4 and the BReLU bound, one value for the layer */
+    int32_t out_lo, out_hi, out_zero;
+} istem_desc;
+ICONV_API int iconv_stem_forward_static(const istem_desc *desc, const void *x, const int8_t *weights, const int32_t *bias,
+                              void *out, void *cuda_stream);
 
 /* ---- host-side parameter arithmetic (no GPU involved) ------------------------------- */
 

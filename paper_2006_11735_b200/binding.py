@@ -18,7 +18,7 @@ KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin"
 EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_forward", "iconv_check",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
            "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iconcat_plan", "iconv_probe_mma_rate",
-           "iconv_last_error")
+           "iconv_stem_forward_static", "iconv_last_error")
 
 
 class IconvError(RuntimeError):
@@ -43,6 +43,15 @@ class iadd_desc(C.Structure):
         "brelu", "h_i", "mul", "shift", "out_zero", "out_lo", "out_hi")]
 
 
+class istem_desc(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in (
+        "n", "h", "w", "c_out", "in_dtype", "out_c_total", "out_c_offset", "mul", "shift", "h_i",
+        "out_lo", "out_hi", "out_zero")]
+
+
+STEM_STATIC_BYTES = 32 * 1024 * 1024
+
+
 def _load():
     if not os.path.exists(LIB_PATH):
         raise ImportError("%s is missing: build it with `python -m paper_2006_11735_b200.build` "
@@ -65,6 +74,7 @@ def _load():
     lib.iq_skip_sync.argtypes = [dbl, dbl, i32, P(i32), P(i32), P(dbl), P(dbl)]
     lib.iconcat_plan.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, P(dbl)]
     lib.iconv_probe_mma_rate.argtypes = [i32, i32, P(dbl), P(dbl)]
+    lib.iconv_stem_forward_static.argtypes = [P(istem_desc), vp, vp, vp, vp, vp]
     lib.iconv_last_error.restype = C.c_char_p
     for name in EXPORTS:
         if name != "iconv_last_error":
@@ -200,3 +210,13 @@ def iconv_probe_mma_rate(block_n: int = 256, iters: int = 200000):
     tops, cyc = C.c_double(), C.c_double()
     _check(lib.iconv_probe_mma_rate(block_n, iters, C.byref(tops), C.byref(cyc)))
     return tops.value, cyc.value
+
+
+def iconv_stem_forward_static(x_ptr, weights_ptr, bias_ptr, out_ptr, stream=0, *, n, h, w, c_out, in_dtype=U8_RAW128,
+                              out_c_total=None, out_c_offset=0, mul, shift, h_i, out_lo=0, out_hi=255, out_zero=0):
+    """The 7x7/2 first layer without any allocation: weights and bias are DEVICE addresses,
+    the scratch is the library's static device array (see ``include/iconv.h``)."""
+    d = istem_desc(n=n, h=h, w=w, c_out=c_out, in_dtype=in_dtype,
+                   out_c_total=c_out if out_c_total is None else out_c_total, out_c_offset=out_c_offset,
+                   mul=int(mul), shift=int(shift), h_i=int(h_i), out_lo=out_lo, out_hi=out_hi, out_zero=out_zero)
+    _check(lib.iconv_stem_forward_static(C.byref(d), x_ptr, weights_ptr, bias_ptr, out_ptr, stream))

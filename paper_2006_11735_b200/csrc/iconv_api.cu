@@ -252,7 +252,7 @@ extern "C" int iconv_check(void *cuda_stream)
     if (st != 0) {
         const int z = 0;
         ICONV_CUDA_TRY(cudaMemcpyToSymbol(g_device_status, &z, sizeof(int)));
-        set_error("a bounded device-side wait ran out (code %d)", st);
+        set_error("a kernel recorded device status code %d (1-7: a bounded wait ran out; 8: bias out of range)", st);
         return ICONV_ERR_TIMEOUT;
     }
     return ICONV_OK;

@@ -11,6 +11,7 @@
 //      T with weights rearranged the same way: out(oh, ow) = sum_R T[oh+R][ow] . W'[R].
 //
 // The sum is the same integers in another order, so the result is bit-identical.
+#include <cstring>
 #include <vector>
 
 #include "plan.h"
@@ -117,3 +118,173 @@ int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
 }
 
 }  // namespace iconv
+
+// ---------------------------------------------------------------- allocation-free variant
+//
+// The same two steps for callers that may not allocate device memory (see iconv.h): the
+// repacked image, the rearranged weights and the epilogue constants live in one file-scope
+// device array instead of plan-owned buffers, and the caller hands in weights and bias that
+// are already on the device.  In host code `g_stem_static` names a host-side stand-in of the
+// array, not its device address: the address every kernel and TMA descriptor receives is the
+// one cudaGetSymbolAddress returns, looked up once per device.
+namespace iconv {
+
+namespace {
+
+constexpr size_t STEM_STATIC_W_BYTES = 64 * 1024;       // rearranged weights: 256 channels x 4 x 64
+constexpr size_t STEM_STATIC_PAR_BYTES = 64 * 1024;     // {c_a, mul, shift, h_i} x 256 int32 (+ slack)
+constexpr size_t STEM_STATIC_T_OFFSET = STEM_STATIC_W_BYTES + STEM_STATIC_PAR_BYTES;
+
+static __device__ __align__(256) unsigned char g_stem_static[ICONV_STEM_STATIC_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+unsigned char *g_stem_static_ptr[MAX_DEVICES] = {nullptr};
+
+// Device address of the array on the current device (looked up on the first call per device).
+int stem_static_base(unsigned char **base)
+{
+    int dev = 0;
+    ICONV_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) { set_error("iconv_stem_forward_static: device index %d not supported", dev); return ICONV_ERR_UNSUPPORTED; }
+    if (!g_stem_static_ptr[dev]) {
+        unsigned char *ptr = nullptr;
+        ICONV_CUDA_TRY(cudaGetSymbolAddress((void **)&ptr, g_stem_static));
+        if (!ptr) { set_error("iconv_stem_forward_static: the scratch array has no device address"); return ICONV_ERR_CUDA; }
+        g_stem_static_ptr[dev] = ptr;
+    }
+    *base = g_stem_static_ptr[dev];
+    return ICONV_OK;
+}
+
+// Writes W'[co][R][S*16 + (dy*2+dx)*3 + c] = W[co][2R+dy-1][2S+dx-1][c] (0 where an index is
+// -1, in the padding lanes and in the padded channels) and the epilogue constants.  Every
+// byte the GEMM reads is written here, so the array's previous contents never matter.
+__global__ void __launch_bounds__(256)
+stem_static_prepare_kernel(const int8_t *__restrict__ w, const int32_t *__restrict__ bias, int8_t *__restrict__ w2,
+                           int32_t *__restrict__ par, int c_out, int c_out_pad, int mul, int shift, int h_i, int *status)
+{
+    const int total = c_out_pad * 256;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const int j = e & 63, R = (e >> 6) & 3, co = e >> 8;
+        const int S = j >> 4, k = j & 15;
+        int8_t v = 0;
+        if (co < c_out && k < 12) {
+            const int tap = k / 3, c = k - 3 * tap;
+            const int r = 2 * R + (tap >> 1) - 1, s = 2 * S + (tap & 1) - 1;
+            if (r >= 0 && s >= 0) v = w[((co * 7 + r) * 7 + s) * 3 + c];
+        }
+        w2[e] = v;
+        if (e < c_out_pad) {
+            int b = e < c_out ? bias[e] : 0;
+            if (b > (1 << 30) || b < -(1 << 30)) { atomicCAS(status, 0, 8); b = 0; }   // U + b must stay inside int32
+            par[e] = b;
+            par[c_out_pad + e] = mul;
+            par[2 * c_out_pad + e] = shift;
+            par[3 * c_out_pad + e] = h_i;
+        }
+    }
+}
+
+}  // namespace
+
+}  // namespace iconv
+
+using namespace iconv;
+
+extern "C" int iconv_stem_forward_static(const istem_desc *sd, const void *x, const int8_t *weights, const int32_t *bias,
+                                         void *out, void *cuda_stream)
+{
+    if (!sd) { set_error("iconv_stem_forward_static: null descriptor"); return ICONV_ERR_ARG; }
+    if (sd->n < 0 || sd->h < 1 || sd->w < 1 || sd->c_out < 16 || sd->c_out > 256 || sd->c_out % 16) {
+        set_error("iconv_stem_forward_static: need n >= 0, h, w >= 1 and c_out a multiple of 16 in [16, 256]");
+        return ICONV_ERR_ARG;
+    }
+    if (!(sd->in_dtype == ICONV_U8 || sd->in_dtype == ICONV_S8 || sd->in_dtype == ICONV_U8_RAW128)) {
+        set_error("iconv_stem_forward_static: in_dtype must be U8, S8 or U8_RAW128");
+        return ICONV_ERR_ARG;
+    }
+    if (sd->out_c_offset < 0 || sd->out_c_offset + sd->c_out > sd->out_c_total || sd->out_c_total % 16 || sd->out_c_offset % 16) {
+        set_error("iconv_stem_forward_static: output slice outside its tensor or not a multiple of 16 channels");
+        return ICONV_ERR_SHAPE;
+    }
+    if (sd->mul < 1 || sd->shift < 1 || sd->shift > 31 || sd->h_i < 0 || sd->out_lo > sd->out_hi || sd->out_lo < 0 || sd->out_hi > 255 ||
+        (unsigned long long)sd->h_i * (unsigned long long)sd->mul + (1ull << (sd->shift - 1)) >= (1ull << 32)) {
+        set_error("iconv_stem_forward_static: need mul >= 1, 1 <= shift <= 31, h_i * mul + 2^(shift-1) < 2^32, 0 <= out_lo <= out_hi <= 255");
+        return ICONV_ERR_ARG;
+    }
+    const int h_out = (sd->h + 6 - 7) / 2 + 1, w_out = (sd->w + 6 - 7) / 2 + 1;
+    const int hp = h_out + 3, wp = w_out;
+    const unsigned long long t_bytes = (unsigned long long)sd->n * hp * wp * 64ull;
+    if (STEM_STATIC_T_OFFSET + t_bytes > (unsigned long long)ICONV_STEM_STATIC_BYTES) {
+        set_error("iconv_stem_forward_static: %d images of %d x %d need %llu bytes of scratch, the static array holds %llu",
+                  sd->n, sd->h, sd->w, STEM_STATIC_T_OFFSET + t_bytes, (unsigned long long)ICONV_STEM_STATIC_BYTES);
+        return ICONV_ERR_SHAPE;
+    }
+    if (sd->n == 0) return ICONV_OK;
+    if (!x || !weights || !bias || !out) { set_error("iconv_stem_forward_static: null tensor pointer"); return ICONV_ERR_ARG; }
+    if (((uintptr_t)x % 16) || ((uintptr_t)out % 16)) { set_error("iconv_stem_forward_static: x and out must be 16-byte aligned"); return ICONV_ERR_ALIGN; }
+
+    unsigned char *base = nullptr;
+    int rc = stem_static_base(&base);
+    if (rc != ICONV_OK) return rc;
+    rc = umma_init_once();
+    if (rc != ICONV_OK) return rc;
+    int *status = device_status_ptr();
+    if (!status) { set_error("device status word not available"); return ICONV_ERR_CUDA; }
+    int8_t *w2 = (int8_t *)base;
+    int32_t *par = (int32_t *)(base + STEM_STATIC_W_BYTES);
+    uint8_t *T = base + STEM_STATIC_T_OFFSET;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    // a plan that lives on this call's stack and owns nothing: the GEMM over T
+    iconv_plan_s tmp;
+    iconv_desc &d = tmp.d;
+    memset(&d, 0, sizeof(d));
+    d.n = sd->n; d.h = hp; d.w = wp; d.c_in = 64; d.c_out = sd->c_out; d.kh = 4; d.kw = 1; d.stride = 1; d.pad = 0;
+    d.in_dtype = sd->in_dtype == ICONV_U8 ? ICONV_U8 : ICONV_S8; d.in_c_total = 64; d.in_c_offset = 0;
+    d.out_dtype = ICONV_U8; d.out_c_total = sd->out_c_total; d.out_c_offset = sd->out_c_offset;
+    d.brelu = 1; d.per_channel = 0; d.out_lo = sd->out_lo; d.out_hi = sd->out_hi; d.out_zero = sd->out_zero;
+    d.skip_dtype = -1; d.kernel = ICONV_KERNEL_UMMA;
+    tmp.h_out = h_out; tmp.w_out = w_out; tmp.kernel = ICONV_KERNEL_UMMA;
+    rc = umma_geometry(&tmp);
+    if (rc != ICONV_OK) return rc;
+    if ((size_t)tmp.c_out_pad * 256 > STEM_STATIC_W_BYTES || (size_t)tmp.c_out_pad * 16 > STEM_STATIC_PAR_BYTES) {
+        set_error("iconv_stem_forward_static: channel count beyond the static array's weight region");
+        return ICONV_ERR_SHAPE;
+    }
+    tmp.w_packed = w2;
+    rc = umma_encode_weight_map(&tmp);
+    if (rc == ICONV_OK) {
+        tmp.params_packed = par;
+        tmp.epi = umma_epilogue_safe();      // explicit clamps: no bound on the weights is known on the host
+        tmp.tail = 1;
+        tmp.q_mul = sd->mul; tmp.q_shift = sd->shift; tmp.q_h = sd->h_i;
+
+        stem_static_prepare_kernel<<<(tmp.c_out_pad * 256 + 255) / 256, 256, 0, stream>>>(weights, bias, w2, par, sd->c_out, tmp.c_out_pad,
+                                                                                    sd->mul, sd->shift, sd->h_i, status);
+        const long long total = (long long)sd->n * hp * wp * 4;
+        long long blocks = (total + 255) / 256;
+        if (blocks > 148ll * 32) blocks = 148ll * 32;
+        stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)x, T, sd->n, sd->h, sd->w, hp, wp,
+                                                                 sd->in_dtype == ICONV_U8_RAW128);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) rc = cuda_fail(e, "iconv_stem_forward_static launches");
+    }
+    if (rc == ICONV_OK) {
+        ConvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.x = T; a.skip = nullptr; a.out = out;
+        a.w = w2; a.bias = par; a.mul = par + tmp.c_out_pad; a.shift = par + 2 * tmp.c_out_pad; a.h_i = par + 3 * tmp.c_out_pad;
+        a.n = d.n; a.h = d.h; a.w_ = d.w; a.c_in = 64; a.c_out = d.c_out; a.kh = 4; a.kw = 1; a.stride = 1; a.pad = 0;
+        a.h_out = h_out; a.w_out = w_out;
+        a.in_dtype = d.in_dtype; a.in_c_total = 64; a.in_c_offset = 0;
+        a.out_dtype = ICONV_U8; a.out_c_total = d.out_c_total; a.out_c_offset = d.out_c_offset;
+        a.brelu = 1; a.per_channel = 0; a.out_lo = d.out_lo; a.out_hi = d.out_hi; a.out_zero = d.out_zero;
+        a.skip_dtype = -1; a.skip_mul = 1;
+        rc = launch_umma(&tmp, a, stream);
+    }
+    // the stack plan owns nothing: keep its destructor-free fields from being mistaken for allocations
+    tmp.w_packed = nullptr;
+    tmp.params_packed = nullptr;
+    return rc;
+}

@@ -877,12 +877,29 @@ int umma_supported(const iconv_plan_t *p)
     return ICONV_OK;
 }
 
-int umma_setup(iconv_plan_t *p)
+// Once per process: driver entry points and the kernels' shared-memory opt-in.  Allocates nothing.
+int umma_init_once()
+{
+    const int rc = load_driver_entry_points();
+    if (rc != ICONV_OK) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        attr_set = true;
+    }
+    return ICONV_OK;
+}
+
+// Tile, pipeline and epilogue geometry of a layer, from its descriptor alone (host only).
+int umma_geometry(iconv_plan_t *p)
 {
     const iconv_desc &d = p->d;
-    int rc = load_driver_entry_points();
-    if (rc != ICONV_OK) return rc;
-
     // channel chunk per pipeline stage: the padded reduction should be as short as possible,
     // ties go to the wider chunk (fewer, larger TMA transactions)
     int best_kc = 0, best_pad = 0;
@@ -943,15 +960,16 @@ int umma_setup(iconv_plan_t *p)
         p->piece_bytes = pb;
     }
 
-    // repack weights [c_out][tap][c_in] -> [c_out_pad][tap][c_in_pad], zero filled
-    const size_t k_pad = (size_t)taps * p->c_in_pad;
-    std::vector<int8_t> packed((size_t)p->c_out_pad * k_pad, 0);
-    for (int co = 0; co < d.c_out; ++co)
-        for (int t = 0; t < taps; ++t)
-            memcpy(&packed[(size_t)co * k_pad + (size_t)t * p->c_in_pad], d.weights + ((size_t)co * taps + t) * d.c_in, (size_t)d.c_in);
-    ICONV_CUDA_TRY(cudaMalloc((void **)&p->w_packed, packed.size()));
-    ICONV_CUDA_TRY(cudaMemcpy(p->w_packed, packed.data(), packed.size(), cudaMemcpyHostToDevice));
+    return ICONV_OK;
+}
 
+int umma_epilogue_safe() { return EPI_SAFE; }
+
+// 2-D tiled map over the packed weights p->w_packed, [c_out_pad][taps * c_in_pad].
+int umma_encode_weight_map(iconv_plan_t *p)
+{
+    const iconv_desc &d = p->d;
+    const size_t k_pad = (size_t)d.kh * d.kw * p->c_in_pad;
     const cuuint64_t dims[2] = {(cuuint64_t)k_pad, (cuuint64_t)p->c_out_pad};
     const cuuint64_t strides[1] = {(cuuint64_t)k_pad};
     const cuuint32_t box[2] = {(cuuint32_t)p->kc, (cuuint32_t)p->block_n};
@@ -963,6 +981,29 @@ int umma_setup(iconv_plan_t *p)
         set_error("cuTensorMapEncodeTiled failed with %d", (int)r);
         return ICONV_ERR_UNSUPPORTED;
     }
+    return ICONV_OK;
+}
+
+int umma_setup(iconv_plan_t *p)
+{
+    const iconv_desc &d = p->d;
+    int rc = umma_init_once();
+    if (rc != ICONV_OK) return rc;
+    rc = umma_geometry(p);
+    if (rc != ICONV_OK) return rc;
+
+    // repack weights [c_out][tap][c_in] -> [c_out_pad][tap][c_in_pad], zero filled
+    const int taps = d.kh * d.kw;
+    const size_t k_pad = (size_t)taps * p->c_in_pad;
+    std::vector<int8_t> packed((size_t)p->c_out_pad * k_pad, 0);
+    for (int co = 0; co < d.c_out; ++co)
+        for (int t = 0; t < taps; ++t)
+            memcpy(&packed[(size_t)co * k_pad + (size_t)t * p->c_in_pad], d.weights + ((size_t)co * taps + t) * d.c_in, (size_t)d.c_in);
+    ICONV_CUDA_TRY(cudaMalloc((void **)&p->w_packed, packed.size()));
+    ICONV_CUDA_TRY(cudaMemcpy(p->w_packed, packed.data(), packed.size(), cudaMemcpyHostToDevice));
+
+    rc = umma_encode_weight_map(p);
+    if (rc != ICONV_OK) return rc;
     // make sure the activation descriptor can be encoded for this geometry (the address is
     // only stored, never read, so the packed weights stand in for it)
     CUtensorMap probe;
@@ -986,17 +1027,6 @@ int umma_setup(iconv_plan_t *p)
     p->q_shift = d.out_dtype != ICONV_I32 ? d.shift[0] : 0;
     p->q_h = d.out_dtype != ICONV_I32 ? d.h_i[0] : 0;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        attr_set = true;
-    }
     return ICONV_OK;
 }
 

@@ -40,6 +40,10 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int umma_supported(const iconv_plan_t *p);   // ICONV_OK or the reason it is not
 int umma_setup(iconv_plan_t *p);
+int umma_init_once();                        // driver entry points, shared-memory opt-in; allocates nothing
+int umma_geometry(iconv_plan_t *p);           // host-only tile / pipeline / epilogue geometry
+int umma_encode_weight_map(iconv_plan_t *p);  // TMA map over p->w_packed
+int umma_epilogue_safe();                     // id of the explicit-clamp 32-bit epilogue variant
 int thin_supported(const iconv_plan_t *p);
 int stem_supported(const iconv_plan_t *p);
 int stem_setup(iconv_plan_t *p);
