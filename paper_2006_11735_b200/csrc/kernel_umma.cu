@@ -17,8 +17,9 @@
 //               channels per 16-byte shared-memory store and hand 32-row pieces to TMA
 //               stores aimed at the layer's channel offset.
 //
-// Persistent CTAs (one per SM) walk the tiles round-robin.  Warp 0 produces (TMA), warp 1
-// issues MMAs and owns the TMEM allocation, the others run the epilogue.  All mbarrier
+// Persistent CTAs (one per SM) walk the tiles round-robin.  Warps 0-2 produce (TMA; they take
+// the pipeline's k-iterations in turn), warp 3 issues MMAs and owns the TMEM allocation, the
+// others run the epilogue.  All mbarrier
 // waits are bounded: on expiry the CTA records a code in the device status word, drains
 // its copies in flight, frees its TMEM and returns.
 //
@@ -38,7 +39,10 @@ namespace {
 
 constexpr int BLOCK_M = 128;
 constexpr int EPI_WARPS_MAX = 16;
-constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS_MAX);   // TMA warp, MMA warp, epilogue warps
+constexpr int NUM_PRODUCERS = 3;          // TMA warps: one thread issues a load per 300-400 cycles, the unit takes three times that
+constexpr int MMA_WARP = NUM_PRODUCERS;
+constexpr int EPI_WARP0 = 4;              // first epilogue warp (a multiple of 4: warp % 4 is its TMEM lane quadrant)
+constexpr int NUM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS_MAX);
 constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces (+ the skip rows of one tile)
 constexpr int MAX_STAGES = 12;
 constexpr int MAX_TMEM_BUFS = 4;
@@ -62,7 +66,9 @@ struct UmmaArgs {
     long long m_total;
     int m_tiles, n_tiles;
     int block_n, kc, cchunks, taps;
-    int stages, stage_a_bytes, stage_bytes, b_tile_bytes, resident_b;
+    int stages, kg;                 // pipeline stages; k-iterations (slots) per stage
+    int slot_a_bytes, slot_bytes, stage_bytes, b_tile_bytes, resident_b;
+    int producers;                  // active TMA warps: min(NUM_PRODUCERS, stages * kg)
     int tmem_cols, nbuf, lg_nbuf;   // accumulator buffers (2 or 4)
     int epi_warps, cs, bi;          // epilogue warps, column split per tile, tiles in flight
     int part_n;                     // columns one epilogue warp handles per tile
@@ -189,15 +195,30 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, unsigned long long a_desc, unsigned long long b_desc,
-                                        uint32_t idesc, uint32_t accumulate)
+// tcgen05.mma kind::i8 with the descriptors given as 32-bit halves: the issuing thread's
+// scalar work per instruction is what bounds narrow tiles, so the per-slice address step is a
+// 32-bit add on the low half (start address in 16-byte units; it never carries out of its
+// 14-bit field because shared memory is smaller than 256 KB).
+__device__ __forceinline__ void umma_i8_split(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                              uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// KJ instructions over the KJ 32-byte K slices of one slot (+2 in 16-byte units per slice).
+template <int KJ>
+__device__ __forceinline__ void umma_slot(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                          uint32_t accumulate_first)
+{
+    umma_i8_split(d_tmem, a_lo, b_lo, desc_hi, idesc, accumulate_first);
+#pragma unroll
+    for (int j = 1; j < KJ; ++j) umma_i8_split(d_tmem, a_lo + 2u * j, b_lo + 2u * j, desc_hi, idesc, 1u);
 }
 // The mbarrier receives one arrival once every MMA issued so far by this thread is done.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
@@ -229,14 +250,6 @@ __device__ __forceinline__ unsigned pack4_sat(int v0, int v1, int v2, int v3)
         asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v1), "r"(v0), "r"(hi));
     }
     return d;
-}
-
-// Shared-memory matrix descriptor of a K-major, hardware-swizzled tile whose rows are one
-// swizzle span wide: start address, stride between 8-row groups, descriptor version 1
-// and the swizzle mode (the constant upper half comes from the host).
-__device__ __forceinline__ unsigned long long smem_desc(uint32_t addr, unsigned long long hi)
-{
-    return hi | (unsigned long long)((addr & 0x3FFFFu) >> 4) | (1ull << 16);
 }
 
 struct Shared {
@@ -423,7 +436,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < u.stages; ++s) {
-            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->full[s]), (uint32_t)u.kg);     // one arrival per slot
             mbar_init(smem_u32(&sh->empty[s]), 1);
         }
         for (int b = 0; b < u.nbuf; ++b) {
@@ -436,20 +449,27 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
+    if (warp == MMA_WARP) tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
 
-    int issued = 0;        // producer: k-iterations whose loads were issued
+    int last_stage = -1;   // producer: stage and phase of the last load this warp issued
+    uint32_t last_parity = 0;
     int b_issued = 0;      // producer: resident filter bank requested
     int skip_issued = 0;   // epilogue lane 0: skip prefetches issued
 
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        if (lane == 0 && (int)blockIdx.x < num_tiles) {
-            if (u.resident_b) {
+    if (warp < NUM_PRODUCERS) {
+        // ---------------------------------------------------------------- TMA producers
+        // Producer j of P issues the loads of k-iterations j, j + P, j + 2P, ... (counted across
+        // tiles).  A stage holds `kg` k-iterations (slots) behind one pair of barriers, so the MMA
+        // issuer pays its wait + commit round once per kg.  P never exceeds stages * kg: a parity
+        // wait cannot tell a barrier that is two phases behind from one that is done, and a
+        // producer that skips P iterations only knows the consumer's progress up to its own
+        // previous iteration.
+        if (lane == 0 && warp < u.producers && (int)blockIdx.x < num_tiles) {
+            if (u.resident_b && warp == 0) {
                 const uint32_t bf = smem_u32(&sh->b_full);
                 mbar_expect_tx(bf, (uint32_t)(u.block_n * u.kc * k_iters * u.n_tiles));
                 for (int nt = 0; nt < u.n_tiles; ++nt)
@@ -458,7 +478,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                     ki * u.kc, nt * u.block_n);
                 b_issued = 1;
             }
-            int it = 0, stage = 0;
+            int stage = 0, slot = 0, turn = warp;   // turn: iterations until this producer's next one
             uint32_t parity = 0;
             bool ok = true;
             const int hw = a.h_out * a.w_out;
@@ -472,29 +492,41 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const int p = (int)fast_div(rem, u.div_w_mul, u.div_w_shr);
                 const int q = (int)rem - p * a.w_out;
                 const int cw = q * a.stride - a.pad, ch = p * a.stride - a.pad;
-                int r = 0, s = 0, kx = 0;
+                int r = 0, s = 0, kx = 0, ki = 0;
                 for (int tap = 0; tap < u.taps && ok; ++tap) {
-                    for (int cc = 0; cc < u.cchunks; ++cc, ++it, kx += u.kc) {
-                        if (!mbar_wait(smem_u32(&sh->empty[stage]), parity ^ 1u, &sh->abort_flag)) {
-                            give_up(sh, u.status, 1);
-                            ok = false;
-                            break;
+                    for (int cc = 0; cc < u.cchunks; ++cc, ++ki, kx += u.kc) {
+                        const bool tile_end = ki == k_iters - 1;
+                        if (turn == 0) {
+                            if (!mbar_wait(smem_u32(&sh->empty[stage]), parity ^ 1u, &sh->abort_flag)) {
+                                give_up(sh, u.status, 1);
+                                ok = false;
+                                break;
+                            }
+                            const uint32_t full = smem_u32(&sh->full[stage]);
+                            const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes + (size_t)slot * u.slot_bytes);
+                            mbar_expect_tx(full, tx);
+                            tma_load_im2col_4d(sa, &tmap_x, full, cc * u.kc, cw, ch, img, (unsigned short)s,
+                                               (unsigned short)r);
+                            if (!u.resident_b) tma_load_2d(sa + u.slot_a_bytes, &tmap_w, full, kx, n_tile * u.block_n);
+                            // a tile's last stage may be short: stand in for its missing slots
+                            if (tile_end)
+                                for (int e = slot + 1; e < u.kg; ++e) mbar_arrive(full);
+                            last_stage = stage;
+                            last_parity = parity;
+                            turn = u.producers;
                         }
-                        const uint32_t full = smem_u32(&sh->full[stage]);
-                        const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes);
-                        mbar_expect_tx(full, tx);
-                        tma_load_im2col_4d(sa, &tmap_x, full, cc * u.kc, cw, ch, img, (unsigned short)s,
-                                           (unsigned short)r);
-                        if (!u.resident_b) tma_load_2d(sa + u.stage_a_bytes, &tmap_w, full, kx, n_tile * u.block_n);
-                        issued = it + 1;
-                        if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+                        --turn;
+                        if (++slot == u.kg || tile_end) {
+                            slot = 0;
+                            if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+                        }
                     }
                     if (++s == a.kw) { s = 0; ++r; }
                 }
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
+    } else if (warp == MMA_WARP) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0 && (int)blockIdx.x < num_tiles) {
             int t = 0, stage = 0;
@@ -504,7 +536,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 give_up(sh, u.status, 6);
                 ok = false;
             }
-            const int kj = u.kc >> 5;   // MMAs per stage: 32 bytes of K each
+            const int kj = u.kc >> 5;   // MMAs per k-iteration: 32 bytes of K each
+            const uint32_t desc_hi32 = (uint32_t)(u.desc_hi >> 32);
+            const uint32_t a_lo0 = ((smem_u32(tiles) & 0x3FFFFu) >> 4) | (1u << 16);
+            const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, slot_step = (uint32_t)u.slot_bytes >> 4;
+            const uint32_t slot_a_step = (uint32_t)u.slot_a_bytes >> 4;
+            const uint32_t b_step = (uint32_t)(u.resident_b ? u.b_tile_bytes : u.slot_bytes) >> 4;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & (u.nbuf - 1);
                 if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
@@ -516,28 +553,35 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 uint32_t sb = 0;
                 if (u.resident_b) {
                     const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
-                    sb = smem_u32(b_res + (size_t)((tile - m_tile * u.n_tiles) * k_iters) * u.b_tile_bytes);
+                    sb = ((smem_u32(b_res + (size_t)((tile - m_tile * u.n_tiles) * k_iters) * u.b_tile_bytes) & 0x3FFFFu) >> 4) | (1u << 16);
                 }
-                for (int ki = 0; ki < k_iters; ++ki) {
+                for (int ki = 0; ki < k_iters;) {
                     if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
                         give_up(sh, u.status, 3);
                         ok = false;
                         break;
                     }
-                    const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes);
-                    const unsigned long long da = smem_desc(sa, u.desc_hi);
-                    const unsigned long long db = smem_desc(u.resident_b ? sb : sa + u.stage_a_bytes, u.desc_hi);
-                    for (int j = 0; j < kj; ++j)   // +2 in 16-byte units per 32 bytes of K
-                        umma_i8(d_tmem, da + 2ull * j, db + 2ull * j, u.idesc, (uint32_t)((ki | j) != 0));
+                    // low descriptor halves: start address in 16-byte units, bit 16 = the (ignored) leading offset
+                    uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step;
+                    uint32_t b_lo = u.resident_b ? sb : a_lo + slot_a_step;
+                    const int in_stage = min(u.kg, k_iters - ki);
+                    for (int e = 0; e < in_stage; ++e, ++ki) {
+                        const uint32_t acc = (uint32_t)(ki != 0);
+                        if (kj == 4) umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        else if (kj == 2) umma_slot<2>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        else umma_slot<1>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        a_lo += slot_step;
+                        b_lo += b_step;
+                    }
+                    if (u.resident_b) sb = b_lo;
                     umma_commit(smem_u32(&sh->empty[stage]));   // frees the stage when these MMAs are done
                     if (++stage == u.stages) { stage = 0; parity ^= 1u; }
-                    sb += (uint32_t)u.b_tile_bytes;
                 }
                 if (ok) umma_commit(smem_u32(&sh->tmem_full[buf]));
             }
         }
         __syncwarp();
-    } else if (warp < 2 + u.epi_warps) {
+    } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps) {
         // ---------------------------------------------------------------- epilogue
         // warp % 4 fixes the TMEM lane quadrant (32 output pixels) a warp may read.  The warps
         // of a quadrant form `cs * bi` slots: `cs` slots split a tile's columns, `bi` groups
@@ -546,7 +590,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // outputs in its own two swizzled shared-memory pieces and writes them with its own
         // TMA stores (which also clip the ragged last tile and the channels beyond c_out), so
         // no cross-warp barrier exists that a warp which gave up could strand.
-        const int ew = warp - 2;
+        const int ew = warp - EPI_WARP0;
         const int quad = warp & 3;
         const int slot = ew >> 2;
         const int part = slot % u.cs;
@@ -680,24 +724,24 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // Something gave up: wait (bounded) for the copies and MMAs still in flight so that
         // nothing touches this CTA's shared memory or TMEM after it returns.
         volatile int never = 0;
-        if (warp == 0 && lane == 0) {
+        if (warp < NUM_PRODUCERS && lane == 0) {
             if (b_issued) mbar_wait(smem_u32(&sh->b_full), 0, &never);
-            for (int s = 0; s < u.stages; ++s) {
-                int last = -1;
-                for (int i = issued - 1; i >= 0 && i >= issued - u.stages; --i)
-                    if (i % u.stages == s) { last = i; break; }
-                if (last >= 0) mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((last / u.stages) & 1), &never);
-            }
+            // this warp's loads that can still be in flight: wait for the phase of the last one (it
+            // may lack another producer's arrival, hence the bound), then for longer than any load
+            // already handed to the TMA unit can take
+            if (last_stage >= 0) mbar_wait(smem_u32(&sh->full[last_stage]), last_parity, &never);
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000) {}
         }
-        if (warp == 1 && lane == 0) {
+        if (warp == MMA_WARP && lane == 0) {
             umma_commit(smem_u32(&sh->drain));
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }
-        if (warp >= 2 && warp < 2 + u.epi_warps && lane == 0 && skip_issued > 0)
-            mbar_wait(smem_u32(&sh->skip_full[warp - 2]), (uint32_t)((skip_issued - 1) & 1), &never);
+        if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps && lane == 0 && skip_issued > 0)
+            mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0]), (uint32_t)((skip_issued - 1) & 1), &never);
         __syncthreads();
     }
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)u.tmem_cols);
     }
@@ -926,18 +970,30 @@ int umma_geometry(iconv_plan_t *p)
     const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
     const long long bank = (long long)b_tile * k_iters * n_tiles;
     const int fixed = (int)sizeof(Shared) + 2048;
+    // Epilogue-heavy layers (one or two k-iterations per tile) get sixteen epilogue warps, the
+    // others eight and a deeper pipeline.  A stage groups kg k-iterations (at most 48 KB) as
+    // long as three stages still fit: the MMA issuer's wait + commit round costs about 400
+    // cycles whatever the stage holds.
     p->resident_b = 0;
     p->epi_warps = 0;
-    for (int ew = 16; ew >= 8 && !p->epi_warps; ew -= 8) {
+    p->kg = 1;
+    for (int ew = (k_iters <= 2 ? 16 : 8); ew >= 8 && !p->epi_warps; ew -= 8) {
         const int avail = MAX_SMEM - fixed - ew * EPI_WARP_SMEM;
-        const int want = k_iters >= 4 ? 4 : (k_iters >= 2 ? 2 : 2);
+        const int want = 2;
+        int room = 0, slot = 0;
         if (bank <= RESIDENT_B_MAX && avail - (int)bank >= want * stage_a) {
             p->resident_b = 1;
-            p->stages = (avail - (int)bank) / stage_a;
-            p->epi_warps = ew;
+            room = avail - (int)bank;
+            slot = stage_a;
         } else if (avail >= want * (stage_a + b_tile) || ew == 8) {
-            p->stages = avail / (stage_a + b_tile);
+            room = avail;
+            slot = stage_a + b_tile;
+        }
+        if (slot) {
             p->epi_warps = ew;
+            for (int kg = k_iters < 8 ? k_iters : 8; kg >= 1; --kg)
+                if (kg * slot <= 48 * 1024 && room / (kg * slot) >= 3) { p->kg = kg; break; }
+            p->stages = room / (p->kg * slot);
         }
     }
     if (p->stages > MAX_STAGES) p->stages = MAX_STAGES;
@@ -1050,10 +1106,13 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.cchunks = p->c_in_pad / p->kc;
     u.taps = d.kh * d.kw;
     u.stages = p->stages;
-    u.stage_a_bytes = BLOCK_M * p->kc;
+    u.kg = p->kg;
+    u.slot_a_bytes = BLOCK_M * p->kc;
     u.b_tile_bytes = (p->block_n * p->kc + 1023) / 1024 * 1024;
     u.resident_b = p->resident_b;
-    u.stage_bytes = u.stage_a_bytes + (p->resident_b ? 0 : u.b_tile_bytes);
+    u.slot_bytes = u.slot_a_bytes + (p->resident_b ? 0 : u.b_tile_bytes);
+    u.stage_bytes = u.kg * u.slot_bytes;
+    u.producers = p->stages * p->kg < NUM_PRODUCERS ? p->stages * p->kg : NUM_PRODUCERS;
     u.nbuf = p->nbuf;
     u.lg_nbuf = p->nbuf == 4 ? 2 : 1;
     int cols = 32;

@@ -21,6 +21,7 @@ struct iconv_plan_s {
     int block_n = 0, kc = 0, c_in_pad = 0, c_out_pad = 0, stages = 0, swizzle_bytes = 0;
     int epi = 0;             // epilogue variant of the tensor-core kernel
     int half_n = 0, piece_bytes = 0;   // columns per epilogue warp and staged piece width
+    int kg = 1;              // k-iterations grouped behind one pair of pipeline barriers
     int nbuf = 2;            // TMEM accumulator buffers
     int resident_b = 0;      // 1: the packed filter bank stays in shared memory for the whole kernel
     int epi_warps = 8, cs = 1, bi = 1;   // epilogue warps; column split per tile; tiles in flight
