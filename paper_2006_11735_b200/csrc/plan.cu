@@ -20,7 +20,7 @@ int choose_kernel(iconv_plan_t *p)
         const int rc = thin_supported(p);
         if (rc != ICONV_OK) return rc;
         p->kernel = ICONV_KERNEL_THIN;
-        return ICONV_OK;
+        return thin_setup(p);
     }
     if (want == ICONV_KERNEL_STEM) {
         const int rc = stem_supported(p);
@@ -32,7 +32,7 @@ int choose_kernel(iconv_plan_t *p)
     // the direct kernel for whatever is left.
     if (thin_supported(p) == ICONV_OK) {
         p->kernel = ICONV_KERNEL_THIN;
-        return ICONV_OK;
+        return thin_setup(p);
     }
     if (stem_supported(p) == ICONV_OK) {
         const int rc = stem_setup(p);

@@ -21,6 +21,7 @@ struct iconv_plan_s {
     int block_n = 0, kc = 0, c_in_pad = 0, c_out_pad = 0, stages = 0, swizzle_bytes = 0;
     int epi = 0;             // epilogue variant of the tensor-core kernel
     int half_n = 0, piece_bytes = 0;   // columns per epilogue warp and staged piece width
+    int thin_narrow = 0;     // thin kernels: BReLU + Eq. 4 provably fit 32 bits
     int kg = 1;              // k-iterations grouped behind one pair of pipeline barriers
     int nbuf = 2;            // TMEM accumulator buffers
     int resident_b = 0;      // 1: the packed filter bank stays in shared memory for the whole kernel
@@ -46,6 +47,7 @@ int umma_geometry(iconv_plan_t *p);           // host-only tile / pipeline / epi
 int umma_encode_weight_map(iconv_plan_t *p);  // TMA map over p->w_packed
 int umma_epilogue_safe();                     // id of the explicit-clamp 32-bit epilogue variant
 int thin_supported(const iconv_plan_t *p);
+int thin_setup(iconv_plan_t *p);
 int stem_supported(const iconv_plan_t *p);
 int stem_setup(iconv_plan_t *p);
 int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);

@@ -240,3 +240,58 @@ def test_mma_issue_rate_probe_reports_a_plausible_peak():
     assert 1000.0 < tops < 10000.0
     with pytest.raises(B.IconvError):
         B.iconv_probe_mma_rate(100, 10)
+
+
+THIN_SHAPES = [
+    # n, h, w, c_in, c_out, k, stride, pad
+    (2, 40, 48, 1, 64, 3, 1, 1),        # VDSR first layer
+    (2, 21, 37, 1, 64, 5, 1, 2),        # VRCNN first layer, ragged sizes
+    (1, 9, 11, 1, 16, 3, 2, 1),         # one channel group, stride 2
+    (3, 8, 8, 1, 128, 1, 1, 0),
+    (2, 40, 48, 64, 1, 3, 1, 1),        # VDSR last layer
+    (2, 19, 23, 48, 1, 3, 1, 1),        # VRCNN last layer: three lanes per pixel
+    (1, 7, 9, 16, 1, 5, 1, 2),
+    (2, 6, 6, 512, 1, 1, 1, 0),         # a whole warp per pixel
+]
+
+
+@pytest.mark.parametrize("shape", THIN_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("in_dtype", [B.U8, B.U8_RAW128, B.S8])
+def test_thin_kernels_match_oracle(shape, in_dtype):
+    n, h, w, c_in, c_out, k, stride, pad = shape
+    if c_out == 1 and in_dtype == B.U8_RAW128:
+        pytest.skip("raw-128 input is a first-layer format")
+    X, W, b, mul, shift, h_i = _layer(sum(shape) + 3, n, h, w, c_in, c_out, k, in_dtype)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, in_dtype=in_dtype, kernel=B.KERNEL_THIN)
+    want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, in_dtype=in_dtype)
+    assert fam == B.KERNEL_THIN
+    assert np.array_equal(got, want)
+    if c_out == 1:          # one channel, one bias: the zero share of a small sample is arbitrary
+        assert (want == 0).mean() < 0.95 and np.unique(want).size > 8
+    else:
+        assert 0.05 < (want == 0).mean() < 0.95
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, in_dtype=in_dtype)
+    assert fam == B.KERNEL_THIN and np.array_equal(got, want)        # AUTO picks it too
+
+
+def test_thin_kernels_variants():
+    # c_in = 1 into a channel offset of a wider tensor, per-channel parameters, wide (64-bit) Eq. 4
+    X, W, b, mul, shift, h_i = _layer(91, 2, 17, 13, 1, 32, 3, B.U8_RAW128, per_channel=True)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.U8_RAW128, out_c_total=64, out_c_offset=16)
+    want = oracle_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.U8_RAW128, out_c_total=64, out_c_offset=16)
+    assert fam == B.KERNEL_THIN and np.array_equal(got, want)
+    got, fam = gpu_conv(X, W, b, mul * 4096, shift + 12, h_i, pad=1, in_dtype=B.U8_RAW128)      # h_i * mul >= 2^32
+    want = oracle_conv(X, W, b, mul * 4096, shift + 12, h_i, pad=1, in_dtype=B.U8_RAW128)
+    assert fam == B.KERNEL_THIN and np.array_equal(got, want)
+    # c_out = 1 with the global residual: raw image skip, no BReLU, zero point 128 (the regression output)
+    X, W, b, mul, shift, h_i = _layer(92, 2, 18, 22, 64, 1, 3)
+    S = np.random.default_rng(5).integers(0, 256, size=(2, 18, 22, 1), dtype=np.uint8)
+    kw = dict(pad=1, brelu=False, out_zero=128, skip=S, skip_dtype=B.U8_RAW128, skip_mul=3000, skip_shift=2)
+    got, fam = gpu_conv(X, W, b, [20], [14], [0], **kw)
+    want = oracle_conv(X, W, b, [20], [14], [0], **kw)
+    assert fam == B.KERNEL_THIN and np.array_equal(got, want)
+    assert (want == 0).any() and (want == 255).any() and ((want > 0) & (want < 255)).mean() > 0.3
+    # c_out = 1, raw int32 output
+    got, fam = gpu_conv(X, W, b, [1], [0], [0], pad=1, out_dtype=B.I32, brelu=False)
+    want = oracle_conv(X, W, b, [1], [0], [0], pad=1, out_dtype=B.I32, brelu=False)
+    assert fam == B.KERNEL_THIN and np.array_equal(got, want)
