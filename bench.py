@@ -31,6 +31,12 @@ if ROOT not in sys.path:
 METRIC = "ResNet-50 int8 images/sec"
 UNIT = "images/s"
 WORKLOAD = "resnet50_b256_224x224x3"
+# the other full-size configurations can be timed the same way (--workload); the default and the
+# metric of record is the ResNet-50 one
+WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"),
+             "resnet152": ("ResNet-152 int8 images/sec", "resnet152_b128_224x224x3"),
+             "vdsr": ("VDSR int8 images/sec", "vdsr_16x256x256x1"),
+             "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1")}
 NOMINAL_INT8_TOPS = 4500.0      # NVIDIA's dense INT8 figure for B200 (context only)
 INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
 
@@ -152,6 +158,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--per-layer", action="store_true", help="print the per-layer table to stderr")
+    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--batch", type=int, default=0,
                     help="images per GPU; 0 = the full workload (256). Smaller batches are for profiler "
                          "captures only and are named in config.workload")
@@ -175,13 +182,17 @@ def main():
     dev = torch.device("cuda", local_rank)
     D.init("nccl")
 
-    net = N.resnet50(n=args.batch) if args.batch > 0 else N.resnet50()   # 256 images per GPU (weak scaling)
-    workload = WORKLOAD if net.n == 256 else "resnet50_b%d_224x224x3 (reduced batch: profiling only)" % net.n
-    params = load_params("resnet50")
+    metric, full_name = WORKLOADS[args.workload]
+    full = N.by_name(args.workload)
+    net = N.by_name(args.workload, n=args.batch) if args.batch > 0 else full   # the full batch per GPU (weak scaling)
+    workload = full_name if net.n == full.n else "%s with batch %d (reduced batch: profiling only)" % (full_name, net.n)
+    params = load_params(args.workload)
     g = Network(net, params, device=dev)
     x_host = torch.from_numpy(net_input(net)).pin_memory()
     x_dev = x_host.to(dev, non_blocking=True)
-    logits_host = torch.empty((net.n, 1, 1, 1000), dtype=torch.int32).pin_memory()
+    t_out = net.tensors[net.output]
+    logits_host = torch.empty((net.n, t_out.h, t_out.w, t_out.c),
+                              dtype=torch.int32 if t_out.dtype == "i32" else torch.uint8).pin_memory()
     stream = torch.cuda.current_stream(dev)
     kernels = g.kernels()
     macs = g.conv_macs()
@@ -211,7 +222,8 @@ def main():
     ms_local = e0.elapsed_time(e1)
     ms = D.max_over_ranks(ms_local, dev)
     B.iconv_check(stream.cuda_stream)
-    launches = len(g.steps) * args.steps
+    # the stem is two launches (repack + GEMM), every other step one
+    launches = (len(g.steps) + sum(1 for k in kernels.values() if k == "stem")) * args.steps
 
     # per-kernel-family time inside the timed region
     fam_ms, fam_macs, layer_ms = {}, {}, {}
@@ -255,7 +267,7 @@ def main():
                                                                       2.0 * m / max(t, 1e-9) / 1e9))
 
     cpu = None
-    if rank == 0 and size == 1 and not args.no_cpu_baseline:
+    if rank == 0 and size == 1 and not args.no_cpu_baseline and args.workload == "resnet50":
         n_s = 8
         v, dt = oracle_images_per_s(n_s)
         cpu = {"value": v, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
@@ -263,7 +275,7 @@ def main():
 
     if rank == 0:
         total_images = net.n * size * args.steps
-        line = {"metric": METRIC, "value": total_images / (ms * 1e-3), "unit": UNIT, "n_gpus": size,
+        line = {"metric": metric, "value": total_images / (ms * 1e-3), "unit": UNIT, "n_gpus": size,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
                 "config": {"workload": workload, "global_batch": net.n * size, "parallelism": "dp%d" % size,
@@ -271,7 +283,7 @@ def main():
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
                 "clocks": clocks,
                 "e2e": {"value": total_images / (ms_e2e * 1e-3), "unit": UNIT,
-                        "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(logits_host.numel() * 4)},
+                        "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(logits_host.numel() * logits_host.element_size())},
                 "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
         print(json.dumps(line))
     g.close()
