@@ -88,11 +88,22 @@ typedef struct {
     int32_t skip_c_total, skip_c_offset;
     int32_t skip_mul, skip_shift;      /* Y += [ (S - 128 if RAW128) * skip_mul / 2^skip_shift ] */
     int32_t kernel;                    /* iconv_kernel; AUTO unless a test forces a family */
+    /* Fused projection skip (Section 4.1, the skip that is itself a convolution of the block's
+     * quantised input): used when proj_weights != NULL.  Then the `skip` tensor of iconv_forward is
+     * the projection's INPUT, [n][proj_h][proj_w][proj_c_total] of skip_dtype (U8 or S8), and
+     *     S = sum x_p * W_p + proj_bias          (int32, never stored)
+     *     Y += [S * skip_mul / 2^skip_shift]
+     * exactly as if S had been written as an ICONV_I32 tensor by a separate layer and read back.
+     * The projection's output grid must equal this layer's (n, h_out, w_out).  skip_c_total and
+     * skip_c_offset are ignored.  Tensor-core kernel only; needs brelu = 1 and an 8-bit output. */
+    int32_t proj_h, proj_w, proj_c_in, proj_c_total, proj_c_offset, proj_k, proj_stride, proj_pad;
     const int8_t *weights;             /* host [c_out][kh][kw][c_in] */
     const int32_t *bias;               /* host [c_out] */
     const int32_t *mul;                /* host [1 or c_out], 1 <= mul < 2^31 (ignored for I32 out) */
     const int32_t *shift;              /* host [1 or c_out], 0 <= shift <= 40 */
     const int32_t *h_i;                /* host [1 or c_out], 0 <= h_i (ignored unless brelu) */
+    const int8_t *proj_weights;        /* host [c_out][proj_k][proj_k][proj_c_in], or NULL */
+    const int32_t *proj_bias;          /* host [c_out] (with proj_weights) */
 } iconv_desc;
 
 typedef struct iconv_plan_s iconv_plan_t;
@@ -116,7 +127,8 @@ ICONV_API int iconv_plan_kernel(const iconv_plan_t *plan);
  * x, skip, out: DEVICE pointers owned by the caller.  x holds n*h*w*in_c_total elements
  * of in_dtype; out holds n*h_out*w_out*out_c_total elements of out_dtype, of which only
  * the slice [out_c_offset, out_c_offset + c_out) of each pixel is written; skip (NULL when
- * skip_dtype < 0) holds n*h_out*w_out*skip_c_total elements.  Asynchronous on cuda_stream.
+ * skip_dtype < 0) holds n*h_out*w_out*skip_c_total elements (or, with a fused projection, the
+ * projection's input: n*proj_h*proj_w*proj_c_total elements).  Asynchronous on cuda_stream.
  * The plan is not modified: concurrent forwards on different streams are allowed.
  */
 ICONV_API int iconv_forward(const iconv_plan_t *plan, const void *x, const void *skip, void *out,

@@ -32,9 +32,10 @@ class iconv_desc(C.Structure):
         "n", "h", "w", "c_in", "c_out", "kh", "kw", "stride", "pad",
         "in_dtype", "in_c_total", "in_c_offset", "out_dtype", "out_c_total", "out_c_offset",
         "brelu", "per_channel", "out_lo", "out_hi", "out_zero",
-        "skip_dtype", "skip_c_total", "skip_c_offset", "skip_mul", "skip_shift", "kernel")] + [
+        "skip_dtype", "skip_c_total", "skip_c_offset", "skip_mul", "skip_shift", "kernel",
+        "proj_h", "proj_w", "proj_c_in", "proj_c_total", "proj_c_offset", "proj_k", "proj_stride", "proj_pad")] + [
         ("weights", C.c_void_p), ("bias", C.c_void_p), ("mul", C.c_void_p), ("shift", C.c_void_p),
-        ("h_i", C.c_void_p)]
+        ("h_i", C.c_void_p), ("proj_weights", C.c_void_p), ("proj_bias", C.c_void_p)]
 
 
 class iadd_desc(C.Structure):
@@ -101,8 +102,11 @@ def _i32(a):
 def iconv_plan(*, n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, in_dtype=U8, in_c_total=None, in_c_offset=0,
                out_dtype=U8, out_c_total=None, out_c_offset=0, brelu=1, out_lo=0, out_hi=255, out_zero=0,
                skip_dtype=-1, skip_c_total=0, skip_c_offset=0, skip_mul=1, skip_shift=0, kernel=KERNEL_AUTO,
-               weights, bias, mul=None, shift=None, h_i=None):
-    """Plan one layer; returns an opaque handle (int).  Arrays are host numpy arrays."""
+               weights, bias, mul=None, shift=None, h_i=None, proj=None):
+    """Plan one layer; returns an opaque handle (int).  Arrays are host numpy arrays.
+    proj: optional fused projection skip, a dict with ``weights`` [c_out][k][k][c_in], ``bias``,
+    ``h``, ``w``, ``c_total``, ``c_offset``, ``stride``, ``pad`` of the projection's input; the
+    forward's skip tensor is then that input and ``skip_dtype`` its storage type."""
     weights = np.ascontiguousarray(weights, dtype=np.int8)
     assert weights.shape == (c_out, kh, kw, c_in), weights.shape
     bias = _i32(bias)
@@ -121,6 +125,16 @@ def iconv_plan(*, n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, in_dtype=U8, in
         d.per_channel = int(mul.shape[0] == c_out and c_out > 1)
         d.mul, d.shift, d.h_i = mul.ctypes.data, shift.ctypes.data, h_i.ctypes.data
         keep += [mul, shift, h_i]
+    if proj is not None:
+        pw = np.ascontiguousarray(proj["weights"], dtype=np.int8)
+        pb = _i32(proj["bias"])
+        assert pw.shape[0] == c_out and pw.shape[1] == pw.shape[2] and pb.shape[0] == c_out
+        d.proj_h, d.proj_w, d.proj_c_in, d.proj_k = proj["h"], proj["w"], pw.shape[3], pw.shape[1]
+        d.proj_c_total = proj.get("c_total", pw.shape[3])
+        d.proj_c_offset = proj.get("c_offset", 0)
+        d.proj_stride, d.proj_pad = proj.get("stride", 1), proj.get("pad", 0)
+        d.proj_weights, d.proj_bias = pw.ctypes.data, pb.ctypes.data
+        keep += [pw, pb]
     plan = C.c_void_p()
     _check(lib.iconv_plan(C.byref(d), C.byref(plan)))
     return plan.value

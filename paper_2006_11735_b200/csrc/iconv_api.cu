@@ -77,7 +77,29 @@ static int validate(const iconv_desc &d, int &h_out, int &w_out)
         set_error("iconv_plan: channel slice outside its tensor");
         return ICONV_ERR_SHAPE;
     }
-    if (d.skip_dtype >= 0 && (d.skip_c_offset < 0 || d.skip_c_offset + d.c_out > d.skip_c_total)) {
+    const bool proj = d.proj_weights != nullptr;
+    if (proj) {
+        if (!d.proj_bias || !(d.skip_dtype == ICONV_U8 || d.skip_dtype == ICONV_S8) || d.proj_h < 1 || d.proj_w < 1 ||
+            d.proj_c_in < 1 || d.proj_k < 1 || d.proj_stride < 1 || d.proj_pad < 0) {
+            set_error("iconv_plan: a fused projection needs proj_bias, skip_dtype U8 or S8 and positive sizes");
+            return ICONV_ERR_ARG;
+        }
+        if (d.proj_c_offset < 0 || d.proj_c_offset + d.proj_c_in > d.proj_c_total) {
+            set_error("iconv_plan: projection input slice outside its tensor");
+            return ICONV_ERR_SHAPE;
+        }
+        if (d.proj_h + 2 * d.proj_pad < d.proj_k || d.proj_w + 2 * d.proj_pad < d.proj_k ||
+            (d.proj_h + 2 * d.proj_pad - d.proj_k) / d.proj_stride + 1 != h_out ||
+            (d.proj_w + 2 * d.proj_pad - d.proj_k) / d.proj_stride + 1 != w_out) {
+            set_error("iconv_plan: the projection's output grid differs from the layer's");
+            return ICONV_ERR_SHAPE;
+        }
+        if (!d.brelu || d.out_dtype == ICONV_I32) {
+            set_error("iconv_plan: a fused projection needs brelu = 1 and an 8-bit output");
+            return ICONV_ERR_UNSUPPORTED;
+        }
+    }
+    if (!proj && d.skip_dtype >= 0 && (d.skip_c_offset < 0 || d.skip_c_offset + d.c_out > d.skip_c_total)) {
         set_error("iconv_plan: skip slice outside its tensor");
         return ICONV_ERR_SHAPE;
     }
@@ -112,9 +134,29 @@ static int validate(const iconv_desc &d, int &h_out, int &w_out)
     // order, stays inside int32 when this bound does.
     const long long xmax = d.in_dtype == ICONV_U8 ? 255 : 128;
     long long skip_bound = 0;
-    if (d.skip_dtype >= 0 && dtype_is_8bit(d.skip_dtype)) {
+    if (!proj && d.skip_dtype >= 0 && dtype_is_8bit(d.skip_dtype)) {
         const long long smax = d.skip_dtype == ICONV_U8 ? 255 : 128;
         skip_bound = ((smax * d.skip_mul) >> d.skip_shift) + 1;
+    }
+    if (proj) {
+        // worst-case |S| over the channels from the projection's actual weights
+        const long long pmax = d.skip_dtype == ICONV_U8 ? 255 : 128;
+        const long long KP = (long long)d.proj_k * d.proj_k * d.proj_c_in;
+        long long worst = 0;
+        for (int co = 0; co < d.c_out; ++co) {
+            long long sw = 0;
+            const int8_t *wr = d.proj_weights + (long long)co * KP;
+            for (long long k = 0; k < KP; ++k) sw += wr[k] < 0 ? -(long long)wr[k] : wr[k];
+            long long b = d.proj_bias[co];
+            if (b < 0) b = -b;
+            if (sw * pmax + b >= (1ll << 31)) {
+                set_error("iconv_plan: worst-case |S| of projection channel %d does not fit int32", co);
+                return ICONV_ERR_OVERFLOW;
+            }
+            if (sw * pmax + b > worst) worst = sw * pmax + b;
+        }
+        if (worst > ((1ll << 62) / d.skip_mul)) { set_error("iconv_plan: rescaled projection skip overflows"); return ICONV_ERR_OVERFLOW; }
+        skip_bound = ((worst * d.skip_mul) >> d.skip_shift) + 1;
     }
     const long long K = (long long)d.kh * d.kw * d.c_in;
     for (int co = 0; co < d.c_out; ++co) {
@@ -196,6 +238,8 @@ extern "C" int iconv_plan(const iconv_desc *desc, iconv_plan_t **plan_out)
     p->d.weights = nullptr;
     p->d.bias = nullptr;
     p->d.mul = p->d.shift = p->d.h_i = nullptr;
+    p->d.proj_weights = nullptr;
+    p->d.proj_bias = nullptr;
     if (rc != ICONV_OK) {
         iconv_plan_destroy(p);
         return rc;

@@ -59,13 +59,17 @@ enum {
     EPI_FAST_SKIP8 = 3,  // ... with an 8-bit skip staged by TMA
     EPI_SAFE = 4,        // explicit BReLU clamp, 32-bit Eq. 4, optional zero point / range tail
     EPI_SAFE_SKIP8 = 5,  // ... with an 8-bit skip staged by TMA
-    EPI_SAFE_SKIP32 = 6  // ... with an int32 skip (projection), rescaled in 64 bits
+    EPI_SAFE_SKIP32 = 6, // ... with an int32 skip (projection), rescaled in 64 bits
+    EPI_PROJ = 7         // ... with the projection convolution fused: a second accumulator tile beside the first
 };
 
 struct UmmaArgs {
     long long m_total;
     int m_tiles, n_tiles;
     int block_n, kc, cchunks, taps;
+    // fused projection (segment 0 of the reduction; 0 iterations when absent)
+    int p_iters, p_taps, p_cchunks, p_kw, p_stride, p_pad, proj32;
+    int acc_cols;                   // TMEM columns per accumulator buffer: block_n, or 2 * block_n with a projection
     int stages, kg;                 // pipeline stages; k-iterations (slots) per stage
     int slot_a_bytes, slot_bytes, stage_bytes, b_tile_bytes, resident_b;
     int producers;                  // active TMA warps: min(NUM_PRODUCERS, stages * kg)
@@ -73,7 +77,7 @@ struct UmmaArgs {
     int epi_warps, cs, bi;          // epilogue warps, column split per tile, tiles in flight
     int part_n;                     // columns one epilogue warp handles per tile
     int piece_bytes;                // row width of one staged output piece (16 ... 128 bytes)
-    unsigned idesc;
+    unsigned idesc, idesc_p;        // instruction descriptors of the layer and of the projection (operand signedness)
     unsigned long long desc_hi;     // upper 32 bits of the shared-memory matrix descriptors
     // per-layer epilogue scalars (per-channel layers read the arrays instead)
     int q_mul, q_shift, q_half, q_h;
@@ -81,6 +85,7 @@ struct UmmaArgs {
     unsigned skip_xor;              // 0x80808080 turns int8 skip bytes into offset-binary
     int tail;                       // 1: out_zero / out_lo / out_hi are not provably no-ops
     const int32_t *c_a;             // [c_out_pad] per-channel additive constant of the variant
+    const int32_t *c_b;             // [c_out_pad] projection bias (64-bit form of EPI_PROJ)
     const int32_t *c_mul, *c_shift, *c_h;   // [c_out_pad] copies for per-channel layers
     int *status;
     // exact division of a tile index by n_tiles and of a pixel index by w_out and by
@@ -273,10 +278,45 @@ __device__ __forceinline__ void give_up(Shared *sh, int *status, int code)
 // One group of 16 consecutive output channels of one pixel: accumulators in, 16 output
 // values (8-bit variants) or 16 int32 (raw) out.  `sk` holds the 16 staged skip bytes.
 template <int EPI>
-__device__ __forceinline__ void epilogue16(const int *acc, int *V, int co0, long long m, bool row_ok, uint4 sk,
+__device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int *V, int co0, long long m, bool row_ok, uint4 sk,
                                            const ConvArgs &a, const UmmaArgs &u)
 {
     const int4 *ca4 = (const int4 *)(u.c_a + co0);
+    if (EPI == EPI_PROJ) {
+        // S = accp + b_p is the projection's int32 Y.  32-bit form (bounds proven at plan time):
+        // Y = U + ((accp * skip_mul + C) >> skip_shift), C = b_p * skip_mul + 2^(skip_shift-1) + (b << skip_shift);
+        // otherwise the rescale runs in 64 bits with the two biases apart.
+        const int4 *cb4 = (const int4 *)(u.c_b + co0);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int4 c = __ldg(ca4 + g);
+            const int cc[4] = {c.x, c.y, c.z, c.w};
+            int bp[4] = {0, 0, 0, 0};
+            if (!u.proj32) { const int4 b4 = __ldg(cb4 + g); bp[0] = b4.x; bp[1] = b4.y; bp[2] = b4.z; bp[3] = b4.w; }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                int h = u.q_h, mul = u.q_mul, shift = u.q_shift, half = u.q_half;
+                if (a.per_channel) {
+                    h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
+                    shift = __ldg(u.c_shift + co0 + 4 * g + e); half = (int)(1u << (shift - 1));
+                }
+                int y;
+                if (u.proj32) {
+                    y = acc[4 * g + e] + ((accp[4 * g + e] * a.skip_mul + cc[e]) >> a.skip_shift);
+                    y = max(min(y, h), 0);
+                } else {
+                    long long Y = (long long)acc[4 * g + e] + cc[e] +
+                                  round_shift64(((long long)accp[4 * g + e] + bp[e]) * a.skip_mul, a.skip_shift);
+                    Y = Y < 0 ? 0 : (Y > (long long)h ? (long long)h : Y);
+                    y = (int)Y;
+                }
+                int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
+                if (u.tail) v = min(max(v + a.out_zero, a.out_lo), a.out_hi);
+                V[4 * g + e] = v;
+            }
+        }
+        return;
+    }
     if (EPI == EPI_RAW) {
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
@@ -426,7 +466,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // tiles need the alignment of the widest swizzle pattern (8 rows x 128 bytes)
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *b_res = tiles + (size_t)u.stages * u.stage_bytes;                 // resident filter bank (may be empty)
-    const int k_iters = u.taps * u.cchunks;
+    const int k_iters = u.p_iters + u.taps * u.cchunks;
     Shared *sh = (Shared *)(b_res + (u.resident_b ? (size_t)u.b_tile_bytes * k_iters * u.n_tiles : 0));
     uint8_t *epi_smem = (uint8_t *)(((uintptr_t)(sh + 1) + 1023) & ~(uintptr_t)1023);
 
@@ -491,8 +531,40 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const unsigned rem = m0 - (unsigned)img * (unsigned)hw;
                 const int p = (int)fast_div(rem, u.div_w_mul, u.div_w_shr);
                 const int q = (int)rem - p * a.w_out;
+                int kx = 0, ki = 0;
+                // segment 0: the fused projection (its own input tensor, stride and padding)
+                {
+                    const int cwp = q * u.p_stride - u.p_pad, chp = p * u.p_stride - u.p_pad;
+                    int r = 0, s = 0;
+                    for (int tap = 0; tap < u.p_taps && ok; ++tap) {
+                        for (int cc = 0; cc < u.p_cchunks; ++cc, ++ki, kx += u.kc) {
+                            if (turn == 0) {
+                                if (!mbar_wait(smem_u32(&sh->empty[stage]), parity ^ 1u, &sh->abort_flag)) {
+                                    give_up(sh, u.status, 1);
+                                    ok = false;
+                                    break;
+                                }
+                                const uint32_t full = smem_u32(&sh->full[stage]);
+                                const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes + (size_t)slot * u.slot_bytes);
+                                mbar_expect_tx(full, tx);
+                                tma_load_im2col_4d(sa, &tmap_skip, full, cc * u.kc, cwp, chp, img, (unsigned short)s,
+                                                   (unsigned short)r);
+                                if (!u.resident_b) tma_load_2d(sa + u.slot_a_bytes, &tmap_w, full, kx, n_tile * u.block_n);
+                                last_stage = stage;
+                                last_parity = parity;
+                                turn = u.producers;
+                            }
+                            --turn;
+                            if (++slot == u.kg) {
+                                slot = 0;
+                                if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+                            }
+                        }
+                        if (++s == u.p_kw) { s = 0; ++r; }
+                    }
+                }
                 const int cw = q * a.stride - a.pad, ch = p * a.stride - a.pad;
-                int r = 0, s = 0, kx = 0, ki = 0;
+                int r = 0, s = 0;
                 for (int tap = 0; tap < u.taps && ok; ++tap) {
                     for (int cc = 0; cc < u.cchunks; ++cc, ++ki, kx += u.kc) {
                         const bool tile_end = ki == k_iters - 1;
@@ -549,7 +621,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * u.block_n);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * u.acc_cols);
                 uint32_t sb = 0;
                 if (u.resident_b) {
                     const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
@@ -566,10 +638,14 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     uint32_t b_lo = u.resident_b ? sb : a_lo + slot_a_step;
                     const int in_stage = min(u.kg, k_iters - ki);
                     for (int e = 0; e < in_stage; ++e, ++ki) {
-                        const uint32_t acc = (uint32_t)(ki != 0);
-                        if (kj == 4) umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                        else if (kj == 2) umma_slot<2>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                        else umma_slot<1>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        // the projection's iterations fill the second accumulator tile, the layer's own the first
+                        const uint32_t acc = (uint32_t)(ki != 0 && ki != u.p_iters);
+                        const bool in_proj = ki < u.p_iters;
+                        const uint32_t d = in_proj ? d_tmem + (uint32_t)u.block_n : d_tmem;
+                        const uint32_t id = in_proj ? u.idesc_p : u.idesc;
+                        if (kj == 4) umma_slot<4>(d, a_lo, b_lo, desc_hi32, id, acc);
+                        else if (kj == 2) umma_slot<2>(d, a_lo, b_lo, desc_hi32, id, acc);
+                        else umma_slot<1>(d, a_lo, b_lo, desc_hi32, id, acc);
                         a_lo += slot_step;
                         b_lo += b_step;
                     }
@@ -641,7 +717,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             const long long m = (long long)m_tile * BLOCK_M + quad * 32 + lane;
             const bool row_ok = m < u.m_total;
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.block_n + col_lo);
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.acc_cols + col_lo);
 
             for (int pc = 0; pc < ncols; pc += pcols, ++pieces) {
                 uint8_t *ob = obuf + (size_t)(pieces & 1) * piece_smem;
@@ -666,7 +742,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     for (int hf = 0; hf < 2; ++hf) {
                         if (hf == 1 && !two) break;
                         int V[16];
-                        epilogue16<EPI>(acc + 16 * hf, V, n0 + pc + cc + 16 * hf, m, row_ok, sk[hf], a, u);
+                        int accp[16];
+                        if (EPI == EPI_PROJ) {
+                            tmem_ld16(t_row + (uint32_t)(u.block_n + pc + cc + 16 * hf), accp);
+                            tmem_ld_wait();
+                        }
+                        epilogue16<EPI>(acc + 16 * hf, accp, V, n0 + pc + cc + 16 * hf, m, row_ok, sk[hf], a, u);
                         if (esz_rt == 4) {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) {
@@ -794,16 +875,16 @@ CUtensorMapSwizzle swizzle_of(int kc)
 
 // im2col-mode map over the activation slice: dims {c_in, w, h, n}; the box is KC channels
 // of 128 consecutive output pixels; base-pixel coordinates run over [-pad, dim + pad - k].
-int encode_activation_map(const iconv_plan_t *p, const void *x, CUtensorMap *map)
+int encode_im2col_map(const iconv_plan_t *p, const void *x, int c_in, int c_total, int c_offset, int h, int w, int kh, int kw,
+                      int stride, int pad, CUtensorMap *map)
 {
     const iconv_desc &d = p->d;
-    const cuuint64_t dims[4] = {(cuuint64_t)d.c_in, (cuuint64_t)d.w, (cuuint64_t)d.h, (cuuint64_t)d.n};
-    const cuuint64_t strides[3] = {(cuuint64_t)d.in_c_total, (cuuint64_t)d.in_c_total * d.w,
-                                   (cuuint64_t)d.in_c_total * d.w * d.h};
-    const int lower[2] = {-d.pad, -d.pad};
-    const int upper[2] = {d.pad - (d.kw - 1), d.pad - (d.kh - 1)};
-    const cuuint32_t estr[4] = {1, (cuuint32_t)d.stride, (cuuint32_t)d.stride, 1};
-    const CUresult r = g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, (void *)((const uint8_t *)x + d.in_c_offset),
+    const cuuint64_t dims[4] = {(cuuint64_t)c_in, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)d.n};
+    const cuuint64_t strides[3] = {(cuuint64_t)c_total, (cuuint64_t)c_total * w, (cuuint64_t)c_total * w * h};
+    const int lower[2] = {-pad, -pad};
+    const int upper[2] = {pad - (kw - 1), pad - (kh - 1)};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
+    const CUresult r = g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, (void *)((const uint8_t *)x + c_offset),
                                        dims, strides, lower, upper, (cuuint32_t)p->kc, (cuuint32_t)BLOCK_M, estr,
                                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p->kc),
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -814,7 +895,57 @@ int encode_activation_map(const iconv_plan_t *p, const void *x, CUtensorMap *map
     return ICONV_OK;
 }
 
+int encode_activation_map(const iconv_plan_t *p, const void *x, CUtensorMap *map)
+{
+    const iconv_desc &d = p->d;
+    return encode_im2col_map(p, x, d.c_in, d.in_c_total, d.in_c_offset, d.h, d.w, d.kh, d.kw, d.stride, d.pad, map);
+}
+
+int encode_projection_map(const iconv_plan_t *p, const void *x, CUtensorMap *map)
+{
+    const iconv_desc &d = p->d;
+    return encode_im2col_map(p, x, d.proj_c_in, d.proj_c_total, d.proj_c_offset, d.proj_h, d.proj_w, d.proj_k, d.proj_k,
+                             d.proj_stride, d.proj_pad, map);
+}
+
 long long labs64(long long v) { return v < 0 ? -v : v; }
+
+// Epilogue of a layer with a fused projection: explicit BReLU clamp and 32-bit Eq. 4 (as EPI_SAFE);
+// the skip rescale in 32 bits when |S|max * skip_mul + |C| < 2^31 for every channel, else in 64.
+// Fills c_a (C, or the layer's bias) and c_b (the projection's bias).  Returns < 0 when Eq. 4
+// itself does not fit 32 bits (the caller then plans the two convolutions apart).
+int choose_projection_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_a, std::vector<int32_t> &c_b, int &tail,
+                               int &proj32)
+{
+    c_a.assign((size_t)c_out_pad, 0);
+    c_b.assign((size_t)c_out_pad, 0);
+    const int np = d.per_channel ? d.c_out : 1;
+    bool tail_free = d.out_zero == 0 && d.out_lo <= 0;
+    for (int i = 0; i < np; ++i) {
+        if (d.shift[i] < 1 || d.shift[i] > 31) return -1;
+        const unsigned long long top = (unsigned long long)d.h_i[i] * (unsigned long long)d.mul[i] + (1ull << (d.shift[i] - 1));
+        if (top >= (1ull << 32)) return -1;
+        if ((long long)(top >> d.shift[i]) > d.out_hi) tail_free = false;
+    }
+    tail = tail_free ? 0 : 1;
+    const long long pmax = d.skip_dtype == ICONV_U8 ? 255 : 128;
+    const long long KP = (long long)d.proj_k * d.proj_k * d.proj_c_in;
+    const long long half = d.skip_shift ? (1ll << (d.skip_shift - 1)) : 0;
+    proj32 = d.skip_shift <= 30 ? 1 : 0;
+    for (int co = 0; co < d.c_out; ++co) {
+        long long sw = 0;
+        const int8_t *wr = d.proj_weights + (long long)co * KP;
+        for (long long k = 0; k < KP; ++k) sw += wr[k] < 0 ? -(long long)wr[k] : wr[k];
+        const long long C = (long long)d.proj_bias[co] * d.skip_mul + half + ((long long)d.bias[co] << d.skip_shift);
+        if (sw * pmax * d.skip_mul + labs64(C) >= (1ll << 31)) proj32 = 0;
+    }
+    for (int co = 0; co < d.c_out; ++co) {
+        c_b[co] = d.proj_bias[co];
+        c_a[co] = proj32 ? (int32_t)((long long)d.proj_bias[co] * d.skip_mul + half + ((long long)d.bias[co] << d.skip_shift))
+                         : d.bias[co];
+    }
+    return EPI_PROJ;
+}
 
 // Picks the cheapest epilogue whose 32-bit arithmetic is provably exact for this layer and
 // fills the per-channel additive constant of that variant (c_a, c_out_pad entries).
@@ -914,6 +1045,9 @@ int umma_supported(const iconv_plan_t *p)
     else if (d.kh > 16 || d.kw > 16 || d.pad > 16 || d.stride > 8) why = "filter, padding or stride beyond the im2col descriptor's range";
     else if ((long long)d.kh * d.kw * ((d.c_in + 127) / 128 * 128) >= (1ll << 24)) why = "reduction too long";
     else if ((long long)d.n * p->h_out * p->w_out >= (1ll << 31) - 256) why = "more than 2^31 output pixels";
+    else if (d.proj_weights && (d.proj_c_in % 16 || d.proj_c_total % 16 || d.proj_c_offset % 16)) why = "projection input channels must be multiples of 16";
+    else if (d.proj_weights && (d.proj_k > 16 || d.proj_pad > 16 || d.proj_stride > 8)) why = "projection filter, padding or stride beyond the im2col descriptor's range";
+    else if (d.proj_weights && d.out_dtype == ICONV_I32) why = "a fused projection needs an 8-bit output";
     if (why) {
         set_error("tensor-core path: %s", why);
         return ICONV_ERR_UNSUPPORTED;
@@ -935,6 +1069,7 @@ int umma_init_once()
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         attr_set = true;
     }
     return ICONV_OK;
@@ -946,23 +1081,28 @@ int umma_geometry(iconv_plan_t *p)
     const iconv_desc &d = p->d;
     // channel chunk per pipeline stage: the padded reduction should be as short as possible,
     // ties go to the wider chunk (fewer, larger TMA transactions)
+    const bool proj = d.proj_weights != nullptr;
     int best_kc = 0, best_pad = 0;
     for (int kc = 128; kc >= 32; kc /= 2) {
-        const int padded = (d.c_in + kc - 1) / kc * kc;
+        const int padded = (d.c_in + kc - 1) / kc * kc + (proj ? (d.proj_c_in + kc - 1) / kc * kc : 0);
         if (best_kc == 0 || padded < best_pad) { best_kc = kc; best_pad = padded; }
     }
     p->kc = best_kc;
-    p->c_in_pad = best_pad;
+    p->c_in_pad = (d.c_in + best_kc - 1) / best_kc * best_kc;
+    p->proj_c_in_pad = proj ? (d.proj_c_in + best_kc - 1) / best_kc * best_kc : 0;
     p->swizzle_bytes = best_kc;
-    const int n_tiles = (d.c_out + 255) / 256;
+    // a fused projection keeps two accumulator tiles per buffer: at most 128 columns each
+    const int n_max = proj ? 128 : 256;
+    const int n_tiles = (d.c_out + n_max - 1) / n_max;
     p->block_n = ((d.c_out + n_tiles - 1) / n_tiles + 15) / 16 * 16;
     p->c_out_pad = p->block_n * n_tiles;
     const int taps = d.kh * d.kw;
-    const int k_iters = taps * (p->c_in_pad / p->kc);
+    p->proj_iters = proj ? d.proj_k * d.proj_k * (p->proj_c_in_pad / p->kc) : 0;
+    const int k_iters = p->proj_iters + taps * (p->c_in_pad / p->kc);
     const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
 
-    // accumulator buffers: four when a tile has at most 128 columns, else two
-    p->nbuf = p->block_n <= 128 ? 4 : 2;
+    // accumulator buffers: four when a buffer has at most 128 columns, else two
+    p->nbuf = p->block_n * (proj ? 2 : 1) <= 128 ? 4 : 2;
 
     // shared-memory budget: pipeline stages (+ the resident filter bank) against the
     // epilogue warps' staging.  Sixteen epilogue warps unless that leaves the pipeline short.
@@ -1025,7 +1165,7 @@ int umma_epilogue_safe() { return EPI_SAFE; }
 int umma_encode_weight_map(iconv_plan_t *p)
 {
     const iconv_desc &d = p->d;
-    const size_t k_pad = (size_t)d.kh * d.kw * p->c_in_pad;
+    const size_t k_pad = (size_t)d.kh * d.kw * p->c_in_pad + (size_t)p->proj_iters * p->kc;
     const cuuint64_t dims[2] = {(cuuint64_t)k_pad, (cuuint64_t)p->c_out_pad};
     const cuuint64_t strides[1] = {(cuuint64_t)k_pad};
     const cuuint32_t box[2] = {(cuuint32_t)p->kc, (cuuint32_t)p->block_n};
@@ -1048,13 +1188,19 @@ int umma_setup(iconv_plan_t *p)
     rc = umma_geometry(p);
     if (rc != ICONV_OK) return rc;
 
-    // repack weights [c_out][tap][c_in] -> [c_out_pad][tap][c_in_pad], zero filled
-    const int taps = d.kh * d.kw;
-    const size_t k_pad = (size_t)taps * p->c_in_pad;
+    // repack weights [c_out][tap][c_in] -> [c_out_pad][tap][c_in_pad], zero filled; a fused
+    // projection's weights come first in every row
+    const int taps = d.kh * d.kw, ptaps = d.proj_weights ? d.proj_k * d.proj_k : 0;
+    const size_t kp_pad = (size_t)ptaps * p->proj_c_in_pad;
+    const size_t k_pad = kp_pad + (size_t)taps * p->c_in_pad;
     std::vector<int8_t> packed((size_t)p->c_out_pad * k_pad, 0);
-    for (int co = 0; co < d.c_out; ++co)
+    for (int co = 0; co < d.c_out; ++co) {
+        for (int t = 0; t < ptaps; ++t)
+            memcpy(&packed[(size_t)co * k_pad + (size_t)t * p->proj_c_in_pad], d.proj_weights + ((size_t)co * ptaps + t) * d.proj_c_in,
+                   (size_t)d.proj_c_in);
         for (int t = 0; t < taps; ++t)
-            memcpy(&packed[(size_t)co * k_pad + (size_t)t * p->c_in_pad], d.weights + ((size_t)co * taps + t) * d.c_in, (size_t)d.c_in);
+            memcpy(&packed[(size_t)co * k_pad + kp_pad + (size_t)t * p->c_in_pad], d.weights + ((size_t)co * taps + t) * d.c_in, (size_t)d.c_in);
+    }
     ICONV_CUDA_TRY(cudaMalloc((void **)&p->w_packed, packed.size()));
     ICONV_CUDA_TRY(cudaMemcpy(p->w_packed, packed.data(), packed.size(), cudaMemcpyHostToDevice));
 
@@ -1065,14 +1211,26 @@ int umma_setup(iconv_plan_t *p)
     CUtensorMap probe;
     rc = encode_activation_map(p, (const uint8_t *)p->w_packed - d.in_c_offset, &probe);
     if (rc != ICONV_OK) return rc;
+    if (d.proj_weights) {
+        rc = encode_projection_map(p, (const uint8_t *)p->w_packed - d.proj_c_offset, &probe);
+        if (rc != ICONV_OK) return rc;
+    }
 
-    // epilogue variant and its per-channel constants: {c_a, mul, shift, h_i} x c_out_pad
-    std::vector<int32_t> c_a;
-    p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail);
-    std::vector<int32_t> par((size_t)4 * p->c_out_pad, 0);
+    // epilogue variant and its per-channel constants: {c_a, mul, shift, h_i, c_b} x c_out_pad
+    std::vector<int32_t> c_a, c_b;
+    p->proj32 = 0;
+    if (d.proj_weights) {
+        p->epi = choose_projection_epilogue(d, p->c_out_pad, c_a, c_b, p->tail, p->proj32);
+        if (p->epi < 0) { set_error("tensor-core path: Eq. 4 of a layer with a fused projection must fit 32 bits"); return ICONV_ERR_UNSUPPORTED; }
+    } else {
+        p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail);
+        c_b.assign((size_t)p->c_out_pad, 0);
+    }
+    std::vector<int32_t> par((size_t)5 * p->c_out_pad, 0);
     for (int co = 0; co < p->c_out_pad; ++co) {
         const int q = d.per_channel && co < d.c_out ? co : 0;
         par[co] = c_a[co];
+        par[(size_t)4 * p->c_out_pad + co] = c_b[co];
         par[(size_t)p->c_out_pad + co] = d.out_dtype != ICONV_I32 ? d.mul[q] : 1;
         par[(size_t)2 * p->c_out_pad + co] = d.out_dtype != ICONV_I32 ? d.shift[q] : 1;
         par[(size_t)3 * p->c_out_pad + co] = d.out_dtype != ICONV_I32 ? d.h_i[q] : 0;
@@ -1105,6 +1263,13 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.kc = p->kc;
     u.cchunks = p->c_in_pad / p->kc;
     u.taps = d.kh * d.kw;
+    u.p_iters = p->proj_iters;
+    u.p_taps = p->proj_iters ? d.proj_k * d.proj_k : 0;
+    u.p_cchunks = p->proj_iters ? p->proj_c_in_pad / p->kc : 0;
+    u.p_kw = d.proj_k;
+    u.p_stride = d.proj_stride;
+    u.p_pad = d.proj_pad;
+    u.proj32 = p->proj32;
     u.stages = p->stages;
     u.kg = p->kg;
     u.slot_a_bytes = BLOCK_M * p->kc;
@@ -1116,7 +1281,8 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.nbuf = p->nbuf;
     u.lg_nbuf = p->nbuf == 4 ? 2 : 1;
     int cols = 32;
-    while (cols < p->nbuf * p->block_n) cols *= 2;
+    u.acc_cols = p->block_n * (p->proj_iters ? 2 : 1);
+    while (cols < p->nbuf * u.acc_cols) cols *= 2;
     u.tmem_cols = cols;
     u.epi_warps = p->epi_warps;
     u.cs = p->cs;
@@ -1126,6 +1292,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     // instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, N/8, M/16
     u.idesc = (2u << 4) | ((d.in_dtype == ICONV_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(p->block_n >> 3) << 17) |
               ((unsigned)(BLOCK_M >> 4) << 24);
+    u.idesc_p = (u.idesc & ~(7u << 7)) | ((d.skip_dtype == ICONV_S8 ? 1u : 0u) << 7);
     // matrix descriptor, upper half: stride between 8-row groups (8 * KC bytes, in 16-byte
     // units), descriptor version 1, swizzle mode (128B = 2, 64B = 4, 32B = 6)
     const unsigned long long layout = p->kc == 128 ? 2ull : (p->kc == 64 ? 4ull : 6ull);
@@ -1141,12 +1308,17 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.c_mul = p->params_packed + p->c_out_pad;
     u.c_shift = p->params_packed + 2 * (size_t)p->c_out_pad;
     u.c_h = p->params_packed + 3 * (size_t)p->c_out_pad;
+    u.c_b = p->params_packed + 4 * (size_t)p->c_out_pad;
     const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
     CUtensorMap tmap_out, tmap_skip;
     rc = encode_rows_map((uint8_t *)a.out + (size_t)d.out_c_offset * esz, esz, d.c_out, d.out_c_total, u.m_total,
                          p->piece_bytes, &tmap_out);
     if (rc != ICONV_OK) return rc;
     tmap_skip = tmap_out;
+    if (p->epi == EPI_PROJ) {
+        rc = encode_projection_map(p, a.skip, &tmap_skip);      // the slot of the skip map carries the projection's input
+        if (rc != ICONV_OK) return rc;
+    }
     if (p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8) {
         rc = encode_rows_map((const uint8_t *)a.skip + d.skip_c_offset, 1, d.c_out, d.skip_c_total, u.m_total,
                              p->piece_bytes, &tmap_skip);
@@ -1167,7 +1339,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     const long long tiles = (long long)u.m_tiles * u.n_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     const size_t smem = 1024 + (size_t)u.stages * u.stage_bytes +
-                        (p->resident_b ? (size_t)u.b_tile_bytes * u.taps * u.cchunks * u.n_tiles : 0) + sizeof(Shared) + 1024 +
+                        (p->resident_b ? (size_t)u.b_tile_bytes * (u.p_iters + u.taps * u.cchunks) * u.n_tiles : 0) + sizeof(Shared) + 1024 +
                         (size_t)p->epi_warps * EPI_WARP_SMEM;
     if (smem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
 #define ICONV_LAUNCH(E) umma_conv_kernel<E><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u)
@@ -1178,6 +1350,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     case EPI_SAFE: ICONV_LAUNCH(EPI_SAFE); break;
     case EPI_SAFE_SKIP8: ICONV_LAUNCH(EPI_SAFE_SKIP8); break;
     case EPI_SAFE_SKIP32: ICONV_LAUNCH(EPI_SAFE_SKIP32); break;
+    case EPI_PROJ: ICONV_LAUNCH(EPI_PROJ); break;
     default: ICONV_LAUNCH(EPI_WIDE); break;
     }
 #undef ICONV_LAUNCH

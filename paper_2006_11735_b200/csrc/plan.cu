@@ -6,6 +6,17 @@ namespace iconv {
 int choose_kernel(iconv_plan_t *p)
 {
     const int want = p->d.kernel;
+    if (p->d.proj_weights) {
+        // a fused projection skip exists on the tensor-core path only
+        if (want != ICONV_KERNEL_AUTO && want != ICONV_KERNEL_UMMA) {
+            set_error("iconv_plan: a fused projection needs the tensor-core kernel");
+            return ICONV_ERR_UNSUPPORTED;
+        }
+        const int rc = umma_supported(p);
+        if (rc != ICONV_OK) return rc;
+        p->kernel = ICONV_KERNEL_UMMA;
+        return umma_setup(p);
+    }
     if (want == ICONV_KERNEL_DIRECT || p->d.n == 0) {
         p->kernel = ICONV_KERNEL_DIRECT;
         return ICONV_OK;

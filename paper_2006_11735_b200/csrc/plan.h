@@ -21,6 +21,7 @@ struct iconv_plan_s {
     int block_n = 0, kc = 0, c_in_pad = 0, c_out_pad = 0, stages = 0, swizzle_bytes = 0;
     int epi = 0;             // epilogue variant of the tensor-core kernel
     int half_n = 0, piece_bytes = 0;   // columns per epilogue warp and staged piece width
+    int proj_c_in_pad = 0, proj_iters = 0, proj32 = 0;   // fused projection: padded channels, k-iterations, 32-bit rescale proven
     int thin_narrow = 0;     // thin kernels: BReLU + Eq. 4 provably fit 32 bits
     int kg = 1;              // k-iterations grouped behind one pair of pipeline barriers
     int nbuf = 2;            // TMEM accumulator buffers

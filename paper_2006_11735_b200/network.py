@@ -42,10 +42,22 @@ def net_input(net: Net, first: int = 0, count=None) -> np.ndarray:
 class Network:
     """Plans every layer once; ``forward`` enqueues the whole network on the current stream."""
 
-    def __init__(self, net: Net, params: dict, n=None, device="cuda:0", kernel=B.KERNEL_AUTO):
+    def __init__(self, net: Net, params: dict, n=None, device="cuda:0", kernel=B.KERNEL_AUTO, fuse_projection=True):
+        """fuse_projection: run a projection skip (a "raw" convolution whose int32 output only feeds
+        the next layer's skip) inside that layer's kernel; its int32 tensor is then never written."""
         self.net, self.n, self.device = net, net.n if n is None else n, torch.device(device)
         self.plans, self.steps, self.tensors = {}, [], {}
+        self.fused = {}          # name of a fused projection op -> name of the layer that absorbed it
+        self._pending = {}
         torch.cuda.set_device(self.device)
+        convs = {op.name: op for op in net.convs()}
+        fusable = {}             # skip tensor name -> projection op
+        if fuse_projection and kernel in (B.KERNEL_AUTO, B.KERNEL_UMMA):
+            for op in net.convs():
+                if op.role == "raw" and op.dst != net.output:
+                    users = [o for o in net.ops if getattr(o, "src", None) == op.dst or getattr(o, "skip", None) == op.dst]
+                    if len(users) == 1 and getattr(users[0], "skip", None) == op.dst and getattr(users[0], "src", None) != op.dst:
+                        fusable[op.dst] = op
         for name, t in net.tensors.items():
             self.tensors[name] = torch.zeros((self.n, t.h, t.w, t.c), dtype=_TORCH[t.dtype], device=self.device)
         for op in net.ops:
@@ -55,6 +67,8 @@ class Network:
             elif isinstance(op, AvgPool):
                 self.steps.append(("avg", op, params[op.name]))
             else:
+                if op.dst in fusable and self._try_fuse(op, fusable, params, kernel):
+                    continue
                 p = params[op.name]
                 w_f = gen.weights_f(net.seed, op.layer, op.c_out, op.k, op.k, op.c_in)
                 kw = dict(n=self.n, h=src.h, w=src.w, c_in=op.c_in, c_out=op.c_out, kh=op.k, kw=op.k,
@@ -62,7 +76,11 @@ class Network:
                           in_c_offset=op.in_c_offset, out_c_total=dst.c, out_c_offset=op.out_c_offset,
                           weights=B.iq_quantize_weights(w_f, p["delta"]),
                           bias=gen.bias_i32(net.seed, op.layer, op.c_out), kernel=kernel)
-                if op.skip:
+                fused = self._pending.pop(op.skip, None) if op.skip else None
+                if fused is not None:
+                    kw.update(skip_dtype=fused["skip_dtype"], skip_mul=p["skip_mul"], skip_shift=p["skip_shift"],
+                              proj=fused["proj"])
+                elif op.skip:
                     kw.update(skip_dtype=B.DTYPE_CODE[op.skip_dtype], skip_c_total=net.tensors[op.skip].c,
                               skip_mul=p["skip_mul"], skip_shift=p["skip_shift"])
                 if op.role == "raw":
@@ -70,8 +88,32 @@ class Network:
                 else:
                     kw.update(out_dtype=B.U8, brelu=p["brelu"], mul=p["mul"], shift=p["shift"], h_i=p["h_i"],
                               out_lo=p["out_lo"], out_hi=p["out_hi"], out_zero=p["out_zero"])
+                if fused is not None:
+                    try:
+                        self.plans[op.name] = B.iconv_plan(**kw)
+                    except B.IconvError as e:
+                        if e.status != B.ERR_UNSUPPORTED:
+                            raise
+                        raise RuntimeError("fused projection refused for %s: %s (build the network with "
+                                           "fuse_projection=False)" % (op.name, e))
+                    self.fused[fused["op"].name] = op.name
+                    self.tensors.pop(fused["op"].dst, None)        # the projection's int32 output is never written
+                    self.steps.append(("conv", op, fused["op"].src))
+                    continue
                 self.plans[op.name] = B.iconv_plan(**kw)
                 self.steps.append(("conv", op, None))
+
+    def _try_fuse(self, op, fusable, params, kernel) -> bool:
+        """Remember a projection op so that its consumer plans it as a fused skip."""
+        src = self.net.tensors[op.src]
+        if op.in_dtype != "u8" or op.c_in % 16 or src.c % 16 or op.in_c_offset % 16:
+            return False
+        p = params[op.name]
+        w_f = gen.weights_f(self.net.seed, op.layer, op.c_out, op.k, op.k, op.c_in)
+        self._pending[op.dst] = dict(op=op, skip_dtype=B.U8, proj=dict(
+            weights=B.iq_quantize_weights(w_f, p["delta"]), bias=gen.bias_i32(self.net.seed, op.layer, op.c_out),
+            h=src.h, w=src.w, c_total=src.c, c_offset=op.in_c_offset, stride=op.stride, pad=op.pad))
+        return True
 
     def kernels(self) -> dict:
         return {k: B.KERNEL_NAME[B.iconv_plan_kernel(p)] for k, p in self.plans.items()}
@@ -81,7 +123,8 @@ class Network:
         out = {}
         for op in self.net.convs():
             dst = self.net.tensors[op.dst]
-            out[op.name] = self.n * dst.h * dst.w * op.c_out * op.c_in * op.k * op.k
+            name = self.fused.get(op.name, op.name)          # a fused projection counts with the layer that runs it
+            out[name] = out.get(name, 0) + self.n * dst.h * dst.w * op.c_out * op.c_in * op.k * op.k
         return out
 
     def forward(self, x: torch.Tensor = None, marks: list = None) -> torch.Tensor:
@@ -100,8 +143,9 @@ class Network:
         for kind, op, p in self.steps:
             src = self.net.tensors[op.src]
             if kind == "conv":
+                skip_name = p if p is not None else op.skip       # a fused projection reads its own input
                 B.iconv_forward(self.plans[op.name], T[op.src].data_ptr(),
-                                T[op.skip].data_ptr() if op.skip else None, T[op.dst].data_ptr(), stream)
+                                T[skip_name].data_ptr() if skip_name else None, T[op.dst].data_ptr(), stream)
             elif kind == "max":
                 B.ipool_max(T[op.src].data_ptr(), T[op.dst].data_ptr(), self.n, src.h, src.w, src.c,
                             op.k, op.stride, op.pad, stream)

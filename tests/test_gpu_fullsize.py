@@ -29,6 +29,8 @@ def test_full_size_configuration_matches_oracle_on_sampled_images(name):
     for img in (0, net.n - 1):
         want = ON.forward(net, params, x[img:img + 1])
         for op in net.ops:
+            if op.name in g.fused:        # a fused projection's int32 tensor is never written
+                continue
             got = g.tensors[op.dst][img:img + 1].cpu().numpy()
             assert np.array_equal(got, want[op.dst]), "%s image %d layer %s: %d mismatches" % (
                 name, img, op.name, (got != want[op.dst]).sum())

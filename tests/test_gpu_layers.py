@@ -295,3 +295,40 @@ def test_thin_kernels_variants():
     got, fam = gpu_conv(X, W, b, [1], [0], [0], pad=1, out_dtype=B.I32, brelu=False)
     want = oracle_conv(X, W, b, [1], [0], [0], pad=1, out_dtype=B.I32, brelu=False)
     assert fam == B.KERNEL_THIN and np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("case", [
+    # n, h, w, c_prev, width, c_out, stride
+    (2, 12, 12, 64, 64, 256, 1),        # stage 1: both reductions 64 wide, two 128-column tiles
+    (2, 12, 10, 256, 128, 512, 2),      # strided projection over the block input
+    (1, 8, 8, 32, 16, 48, 1),           # narrow: four accumulator buffers, padded columns
+], ids=str)
+@pytest.mark.parametrize("skip_mul,skip_shift", [(766, 8), (20011, 14)], ids=["rescale32", "rescale64"])
+def test_fused_projection_equals_projection_layer_plus_int32_skip(case, skip_mul, skip_shift):
+    n, h, w, c_prev, width, c_out, stride = case
+    ho, wo = (h - 1) // stride + 1, (w - 1) // stride + 1
+    rng = np.random.default_rng(sum(case))
+    X0 = rng.integers(0, 256, size=(n, h, w, c_prev), dtype=np.uint8)            # block input: the projection's operand
+    Xb = rng.integers(0, 256, size=(n, ho, wo, width), dtype=np.uint8)           # output of the block's 3x3
+    _, Wp, bp, _, _, _ = _layer(3, 1, 1, 1, c_prev, c_out, 1)
+    _, W, b, mul, shift, h_i = _layer(4, 1, 1, 1, width, c_out, 1)
+    h_i = h_i * 6
+    # oracle: the projection as a layer of its own (int32 Y), then the closing layer with that int32 skip
+    S = oracle_conv(X0, Wp, bp, [1], [0], [0], stride=stride, out_dtype=B.I32, brelu=False)
+    want = oracle_conv(Xb, W, b, mul, shift, h_i, skip=S, skip_dtype=B.I32, skip_mul=skip_mul, skip_shift=skip_shift)
+    plan = B.iconv_plan(n=n, h=ho, w=wo, c_in=width, c_out=c_out, kh=1, kw=1, weights=W, bias=b, mul=mul, shift=shift, h_i=h_i,
+                        skip_dtype=B.U8, skip_mul=skip_mul, skip_shift=skip_shift,
+                        proj=dict(weights=Wp, bias=bp, h=h, w=w, stride=stride, pad=0))
+    try:
+        assert B.iconv_plan_kernel(plan) == B.KERNEL_UMMA
+        out = Fenced(want.shape, np.uint8)
+        xd, sd = dev(Xb), dev(X0)
+        st = torch.cuda.current_stream().cuda_stream
+        B.iconv_forward(plan, xd.data_ptr(), sd.data_ptr(), out.ptr, st)
+        B.iconv_check(st)
+        got = out.get()
+    finally:
+        B.iconv_plan_destroy(plan)
+    bad = np.argwhere(got != want)
+    assert bad.shape[0] == 0, "%d mismatches, first at %s" % (bad.shape[0], bad[0])
+    assert 0.02 < (want == 0).mean() < 0.98 and (want == 255).mean() < 0.9

@@ -21,15 +21,20 @@ SMALL = [
 
 
 @pytest.mark.parametrize("net", SMALL, ids=lambda n: n.name)
-@pytest.mark.parametrize("kernel", [B.KERNEL_DIRECT, B.KERNEL_AUTO], ids=["direct", "auto"])
-def test_every_layer_of_small_networks_matches_oracle(net, kernel):
+@pytest.mark.parametrize("kernel,fuse", [(B.KERNEL_DIRECT, False), (B.KERNEL_AUTO, False), (B.KERNEL_AUTO, True)],
+                         ids=["direct", "auto", "auto-fused-projection"])
+def test_every_layer_of_small_networks_matches_oracle(net, kernel, fuse):
     params = ON.calibrate(net)
     x = ON.net_input(net)
     want = ON.forward(net, params, x)
-    g = Network(net, params, kernel=kernel)
+    g = Network(net, params, kernel=kernel, fuse_projection=fuse)
     out = g.forward(torch.from_numpy(x).cuda())
     B.iconv_check(torch.cuda.current_stream().cuda_stream)
+    if fuse and net.name.startswith("resnet"):
+        assert len(g.fused) == 4          # one projection per stage, each absorbed by its block's closing layer
     for op in net.ops:
+        if op.name in g.fused:            # its int32 tensor never exists; the absorbing layer's output is checked
+            continue
         got = g.tensors[op.dst].cpu().numpy()
         assert np.array_equal(got, want[op.dst]), "%s: %d mismatches" % (op.name, (got != want[op.dst]).sum())
     assert np.array_equal(out.cpu().numpy(), want[net.output])
