@@ -195,6 +195,7 @@ def main():
                               dtype=torch.int32 if t_out.dtype == "i32" else torch.uint8).pin_memory()
     stream = torch.cuda.current_stream(dev)
     kernels = g.kernels()
+    described = g.describe()
     macs = g.conv_macs()
 
     for _ in range(args.warmup):
@@ -263,8 +264,8 @@ def main():
         for op in net.ops:
             m = macs.get(op.name, 0)
             t = layer_ms.get(op.name, 0.0)
-            sys.stderr.write("%-14s %-6s %8.4f ms %8.1f TOP/s\n" % (op.name, kernels.get(op.name, "pool"), t,
-                                                                      2.0 * m / max(t, 1e-9) / 1e9))
+            sys.stderr.write("%-14s %-6s %8.4f ms %8.1f TOP/s  %s\n" % (op.name, kernels.get(op.name, "pool"), t,
+                                                                          2.0 * m / max(t, 1e-9) / 1e9, described.get(op.name, "")))
 
     cpu = None
     if rank == 0 and size == 1 and not args.no_cpu_baseline and args.workload == "resnet50":

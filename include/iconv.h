@@ -67,9 +67,12 @@ typedef enum {
     ICONV_KERNEL_DIRECT = 1,   /* CUDA-core direct convolution, any shape */
     ICONV_KERNEL_UMMA = 2,     /* tcgen05.mma kind::i8 implicit GEMM, TMA im2col staging */
     ICONV_KERNEL_THIN = 3,     /* bandwidth-bound layers: c_in <= 4 or c_out == 1 */
-    ICONV_KERNEL_STEM = 4      /* 7x7/2 layer over a 3-channel image: space-to-depth repack into
+    ICONV_KERNEL_STEM = 4,     /* 7x7/2 layer over a 3-channel image: space-to-depth repack into
                                   plan-owned scratch, then the tensor-core kernel.  Forwards of
                                   one such plan must not overlap on the GPU (they share the scratch). */
+    ICONV_KERNEL_UMMA_IM2COL = 5  /* the tensor-core kernel with im2col staging even where the plan
+                                  would load one input patch per tile (stride-1 filters); reported
+                                  as ICONV_KERNEL_UMMA by iconv_plan_kernel */
 } iconv_kernel;
 
 /*
@@ -121,6 +124,11 @@ ICONV_API int iconv_plan_destroy(iconv_plan_t *plan);
 
 /* Which kernel family the plan selected (an iconv_kernel), or a negative status. */
 ICONV_API int iconv_plan_kernel(const iconv_plan_t *plan);
+
+/* One line of text on what the plan decided (kernel family, tile and pipeline geometry, epilogue
+ * variant), for logs and tests: at most `size` bytes including the terminating zero are written
+ * to the HOST buffer `text`. */
+ICONV_API int iconv_plan_describe(const iconv_plan_t *plan, char *text, size_t size);
 
 /*
  * iconv_forward -- one layer forward (Section 3.1 / Eq. 4 / Eq. 5 as listed at the top).

@@ -11,11 +11,11 @@ LIB_PATH = os.path.join(_HERE, "libiconv_b200.so")
 
 OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_OVERFLOW, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
 U8, S8, I32, U8_RAW128 = 0, 1, 2, 3
-KERNEL_AUTO, KERNEL_DIRECT, KERNEL_UMMA, KERNEL_THIN, KERNEL_STEM = 0, 1, 2, 3, 4
+KERNEL_AUTO, KERNEL_DIRECT, KERNEL_UMMA, KERNEL_THIN, KERNEL_STEM, KERNEL_UMMA_IM2COL = 0, 1, 2, 3, 4, 5
 DTYPE_CODE = {"u8": U8, "s8": S8, "i32": I32, "u8_raw128": U8_RAW128}
 KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin", KERNEL_STEM: "stem"}
 
-EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_forward", "iconv_check",
+EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_plan_describe", "iconv_forward", "iconv_check",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
            "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iconcat_plan", "iconv_probe_mma_rate",
            "iconv_stem_forward_static", "iconv_last_error")
@@ -63,6 +63,7 @@ def _load():
     lib.iconv_plan.argtypes = [P(iconv_desc), P(vp)]
     lib.iconv_plan_destroy.argtypes = [vp]
     lib.iconv_plan_kernel.argtypes = [vp]
+    lib.iconv_plan_describe.argtypes = [vp, C.c_char_p, C.c_size_t]
     lib.iconv_forward.argtypes = [vp, vp, vp, vp, vp]
     lib.iconv_check.argtypes = [vp]
     lib.iadd_requant.argtypes = [P(iadd_desc), vp, vp, vp, vp]
@@ -149,6 +150,12 @@ def iconv_plan_kernel(plan) -> int:
     if rc < 0:
         _check(rc)
     return rc
+
+
+def iconv_plan_describe(plan) -> str:
+    buf = C.create_string_buffer(256)
+    _check(lib.iconv_plan_describe(plan, buf, 256))
+    return buf.value.decode()
 
 
 def iconv_forward(plan, x_ptr, skip_ptr, out_ptr, stream=0):

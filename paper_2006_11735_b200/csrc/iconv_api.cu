@@ -58,7 +58,7 @@ static int validate(const iconv_desc &d, int &h_out, int &w_out)
         set_error("iconv_plan: bad skip_dtype");
         return ICONV_ERR_ARG;
     }
-    if (d.kernel < ICONV_KERNEL_AUTO || d.kernel > ICONV_KERNEL_STEM) {
+    if (d.kernel < ICONV_KERNEL_AUTO || d.kernel > ICONV_KERNEL_UMMA_IM2COL) {
         set_error("iconv_plan: bad kernel selector");
         return ICONV_ERR_ARG;
     }
@@ -255,6 +255,25 @@ extern "C" int iconv_plan_kernel(const iconv_plan_t *plan)
         return ICONV_ERR_ARG;
     }
     return plan->kernel;
+}
+
+extern "C" int iconv_plan_describe(const iconv_plan_t *p, char *text, size_t size)
+{
+    if (!p || !text || size == 0) {
+        set_error("iconv_plan_describe: null argument");
+        return ICONV_ERR_ARG;
+    }
+    static const char *fam[] = {"auto", "direct", "umma", "thin", "stem", "umma"};
+    if (p->kernel == ICONV_KERNEL_UMMA)
+        snprintf(text, size, "umma %s block_n=%d kc=%d stages=%d kg=%d resident_b=%d epi_warps=%d cs=%d bi=%d nbuf=%d epi=%d proj_iters=%d",
+                 p->window ? (p->win_full_width ? "window(rows)" : "window(strips)") : "im2col", p->block_n, p->kc,
+                 p->window ? p->win_stages : p->stages, p->kg, p->window ? 1 : p->resident_b, p->epi_warps, p->cs, p->bi, p->nbuf, p->epi,
+                 p->proj_iters);
+    else if (p->kernel == ICONV_KERNEL_STEM && p->inner)
+        snprintf(text, size, "stem -> umma block_n=%d kc=%d stages=%d kg=%d", p->inner->block_n, p->inner->kc, p->inner->stages, p->inner->kg);
+    else
+        snprintf(text, size, "%s", fam[p->kernel >= 0 && p->kernel <= 5 ? p->kernel : 0]);
+    return ICONV_OK;
 }
 
 extern "C" int iconv_forward(const iconv_plan_t *p, const void *x, const void *skip, void *out, void *cuda_stream)

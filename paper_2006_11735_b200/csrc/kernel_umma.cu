@@ -88,6 +88,9 @@ struct UmmaArgs {
     const int32_t *c_b;             // [c_out_pad] projection bias (64-bit form of EPI_PROJ)
     const int32_t *c_mul, *c_shift, *c_h;   // [c_out_pad] copies for per-channel layers
     int *status;
+    // window mode (stride-1 filters: one patch load per tile, every tap a shifted view of it)
+    int win_vw, win_bw, win_bh, win_full_width, win_tpi;    // virtual row width, patch width / height, mode, tiles per image
+    unsigned div_tpi_mul, div_tpi_shr, div_vw_mul, div_vw_shr;
     // exact division of a tile index by n_tiles and of a pixel index by w_out and by
     // h_out * w_out without a divide instruction: q = umulhi(x, mul) >> shr  (x < 2^31)
     unsigned div_nt_mul, div_nt_shr, div_w_mul, div_w_shr, div_hw_mul, div_hw_shr;
@@ -177,6 +180,14 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
         "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
         " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_tile_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h, int n)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n)
         : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
@@ -278,10 +289,9 @@ __device__ __forceinline__ void give_up(Shared *sh, int *status, int code)
 // One group of 16 consecutive output channels of one pixel: accumulators in, 16 output
 // values (8-bit variants) or 16 int32 (raw) out.  `sk` holds the 16 staged skip bytes.
 template <int EPI>
-__device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int *V, int co0, long long m, bool row_ok, uint4 sk,
-                                           const ConvArgs &a, const UmmaArgs &u)
+__device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int *V, const int4 *ca4, int co0, long long m, bool row_ok,
+                                           uint4 sk, const ConvArgs &a, const UmmaArgs &u)
 {
-    const int4 *ca4 = (const int4 *)(u.c_a + co0);
     if (EPI == EPI_PROJ) {
         // S = accp + b_p is the projection's int32 Y.  32-bit form (bounds proven at plan time):
         // Y = U + ((accp * skip_mul + C) >> skip_shift), C = b_p * skip_mul + 2^(skip_shift-1) + (b << skip_shift);
@@ -289,7 +299,7 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
         const int4 *cb4 = (const int4 *)(u.c_b + co0);
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int4 c = __ldg(ca4 + g);
+            const int4 c = ca4[g];
             const int cc[4] = {c.x, c.y, c.z, c.w};
             int bp[4] = {0, 0, 0, 0};
             if (!u.proj32) { const int4 b4 = __ldg(cb4 + g); bp[0] = b4.x; bp[1] = b4.y; bp[2] = b4.z; bp[3] = b4.w; }
@@ -320,7 +330,7 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
     if (EPI == EPI_RAW) {
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int4 c = __ldg(ca4 + g);
+            const int4 c = ca4[g];
             V[4 * g] = acc[4 * g] + c.x; V[4 * g + 1] = acc[4 * g + 1] + c.y;
             V[4 * g + 2] = acc[4 * g + 2] + c.z; V[4 * g + 3] = acc[4 * g + 3] + c.w;
         }
@@ -331,7 +341,7 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
         // u8 saturation that follows stands for both BReLU clamps (proven at plan time)
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int4 c = __ldg(ca4 + g);
+            const int4 c = ca4[g];
             V[4 * g] = (acc[4 * g] * u.q_mul + c.x) >> u.q_shift;
             V[4 * g + 1] = (acc[4 * g + 1] * u.q_mul + c.y) >> u.q_shift;
             V[4 * g + 2] = (acc[4 * g + 2] * u.q_mul + c.z) >> u.q_shift;
@@ -346,7 +356,7 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
         const unsigned w4[4] = {sk.x ^ u.skip_xor, sk.y ^ u.skip_xor, sk.z ^ u.skip_xor, sk.w ^ u.skip_xor};
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int4 c = __ldg(ca4 + g);
+            const int4 c = ca4[g];
             const int cc[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -379,7 +389,7 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
         }
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int4 c = __ldg(ca4 + g);
+            const int4 c = ca4[g];
             const int cc[4] = {c.x, c.y, c.z, c.w};
             const int ss[4] = {s32[g].x, s32[g].y, s32[g].z, s32[g].w};
 #pragma unroll
@@ -421,7 +431,7 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
         const unsigned w4[4] = {sk8.x, sk8.y, sk8.z, sk8.w};
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int4 c = __ldg(ca4 + g);
+            const int4 c = ca4[g];
             const int cc[4] = {c.x, c.y, c.z, c.w};
             const int ss[4] = {s32[g].x, s32[g].y, s32[g].z, s32[g].w};
 #pragma unroll
@@ -726,32 +736,40 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                 }
-                for (int cc = 0; cc < pcols; cc += 32) {
-                    int acc[32];
-                    const bool two = cc + 16 < pcols;
-                    tmem_ld16(t_row + (uint32_t)(pc + cc), acc);
-                    if (two) tmem_ld16(t_row + (uint32_t)(pc + cc + 16), acc + 16);
-                    uint4 sk[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                    if (SKIP8) {
-                        const uint8_t *sp = sbuf + (size_t)(pc / pcols) * piece_smem + row_off;
-                        sk[0] = *(const uint4 *)(sp + (((unsigned)(cc >> 4) ^ row_swz) << 4));
-                        if (two) sk[1] = *(const uint4 *)(sp + (((unsigned)((cc >> 4) + 1) ^ row_swz) << 4));
-                    }
-                    tmem_ld_wait();
+                // 16 columns at a time, the TMEM load of the next group in flight while this one is
+                // worked on; each group's constants and skip bytes are fetched before the wait
+                const int ngroups = pcols >> 4;
+                // (the variants that hold a second accumulator or 64-bit temporaries do not prefetch:
+                // they would spill)
+                constexpr bool PIPE = EPI != EPI_PROJ && EPI != EPI_SAFE_SKIP32 && EPI != EPI_WIDE;
+                int accA[16], accB[16], accpA[16];
+                if (PIPE) tmem_ld16(t_row + (uint32_t)pc, accA);
+                for (int gi = 0; gi < ngroups; gi += 2) {
 #pragma unroll
                     for (int hf = 0; hf < 2; ++hf) {
-                        if (hf == 1 && !two) break;
-                        int V[16];
-                        int accp[16];
-                        if (EPI == EPI_PROJ) {
-                            tmem_ld16(t_row + (uint32_t)(u.block_n + pc + cc + 16 * hf), accp);
-                            tmem_ld_wait();
+                        const int gcur = gi + hf;
+                        if (gcur >= ngroups) break;
+                        const int cc = gcur << 4;
+                        const int co0 = n0 + pc + cc;
+                        if (!PIPE) {
+                            tmem_ld16(t_row + (uint32_t)(pc + cc), accA);
+                            if (EPI == EPI_PROJ) tmem_ld16(t_row + (uint32_t)(u.block_n + pc + cc), accpA);
                         }
-                        epilogue16<EPI>(acc + 16 * hf, accp, V, n0 + pc + cc + 16 * hf, m, row_ok, sk[hf], a, u);
+                        int4 ca[4];
+                        const int4 *cap = (const int4 *)(u.c_a + co0);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + g);
+                        uint4 sk = make_uint4(0, 0, 0, 0);
+                        if (SKIP8)
+                            sk = *(const uint4 *)(sbuf + (size_t)(pc / pcols) * piece_smem + row_off + (((unsigned)gcur ^ row_swz) << 4));
+                        tmem_ld_wait();
+                        if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)(pc + cc + 16), hf ? accA : accB);
+                        int V[16];
+                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, a, u);
                         if (esz_rt == 4) {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) {
-                                const unsigned chunk = (unsigned)(((cc + 16 * hf) >> 2) + g);     // 4 columns = 16 bytes
+                                const unsigned chunk = (unsigned)((cc >> 2) + g);     // 4 columns = 16 bytes
                                 *(int4 *)(ob + row_off + ((chunk ^ row_swz) << 4)) = make_int4(V[4 * g], V[4 * g + 1], V[4 * g + 2], V[4 * g + 3]);
                             }
                         } else {
@@ -763,8 +781,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                 o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
                                 o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
                             }
-                            const unsigned chunk = (unsigned)((cc >> 4) + hf);
-                            *(uint4 *)(ob + row_off + ((chunk ^ row_swz) << 4)) = o;
+                            *(uint4 *)(ob + row_off + (((unsigned)gcur ^ row_swz) << 4)) = o;
                         }
                     }
                 }
@@ -820,6 +837,218 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps && lane == 0 && skip_issued > 0)
             mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0]), (uint32_t)((skip_issued - 1) & 1), &never);
+        __syncthreads();
+    }
+    if (warp == MMA_WARP) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)u.tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------- window mode
+// Stride-1 filters wider than one tap re-read every input pixel kh * kw times in the im2col
+// form, and what a CTA can pull through the TMA unit is about its share of the HBM rate.  Here a
+// tile's whole input patch (its rows plus the halo, the full padded width or a 128 + kw - 1
+// wide strip of it) arrives with ONE tiled load, zero-filled outside the image, as consecutive
+// pixel rows of KC bytes.  Output pixels are numbered along "virtual rows" of win_vw pixels
+// (the padded width, or the width rounded up to 128), 128 consecutive numbers per tile, so that
+// for tap (r, s) the A operand is simply the 128 patch rows starting r * win_bw + s further on:
+// a descriptor whose start address moves by whole rows (the swizzle is a function of the
+// absolute shared-memory address, so any start row reads what TMA wrote).  Virtual pixels
+// beyond the real width are computed and dropped.  The filter bank is resident, the epilogue
+// stores straight from registers (a tile is not a contiguous run of real pixels).
+template <int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                   const __grid_constant__ ConvArgs a, const __grid_constant__ UmmaArgs u)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *b_res = tiles + (size_t)u.stages * u.stage_bytes;
+    Shared *sh = (Shared *)(b_res + (size_t)u.b_tile_bytes * u.taps);
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = u.m_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < u.stages; ++s) {
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
+        }
+        for (int b = 0; b < u.nbuf; ++b) {
+            mbar_init(smem_u32(&sh->tmem_full[b]), 1);
+            mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)(4 * u.cs));
+        }
+        mbar_init(smem_u32(&sh->b_full), 1);
+        mbar_init(smem_u32(&sh->drain), 1);
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == MMA_WARP) tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    int last_stage = -1, b_issued = 0;
+    uint32_t last_parity = 0;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0 && (int)blockIdx.x < num_tiles) {
+            const uint32_t bf = smem_u32(&sh->b_full);
+            mbar_expect_tx(bf, (uint32_t)(u.block_n * u.kc * u.taps));
+            for (int tap = 0; tap < u.taps; ++tap)
+                tma_load_2d(smem_u32(b_res + (size_t)tap * u.b_tile_bytes), &tmap_w, bf, tap * u.kc, 0);
+            b_issued = 1;
+            int stage = 0;
+            uint32_t parity = 0;
+            const uint32_t tx = (uint32_t)(u.kc * u.win_bw * u.win_bh);
+            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+                const int img = (int)fast_div((unsigned)tile, u.div_tpi_mul, u.div_tpi_shr);
+                const unsigned i0 = (unsigned)(tile - img * u.win_tpi) * BLOCK_M;
+                const int y0 = (int)fast_div(i0, u.div_vw_mul, u.div_vw_shr);
+                const int c0 = (int)i0 - y0 * u.win_vw;
+                if (!mbar_wait(smem_u32(&sh->empty[stage]), parity ^ 1u, &sh->abort_flag)) {
+                    give_up(sh, u.status, 1);
+                    break;
+                }
+                const uint32_t full = smem_u32(&sh->full[stage]);
+                mbar_expect_tx(full, tx);
+                tma_load_tile_4d(smem_u32(tiles + (size_t)stage * u.stage_bytes), &tmap_x, full, 0,
+                                 (u.win_full_width ? 0 : c0) - a.pad, y0 - a.pad, img);
+                last_stage = stage;
+                last_parity = parity;
+                if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == MMA_WARP) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0 && (int)blockIdx.x < num_tiles) {
+            int t = 0, stage = 0;
+            uint32_t parity = 0;
+            bool ok = mbar_wait(smem_u32(&sh->b_full), 0, &sh->abort_flag);
+            if (!ok) give_up(sh, u.status, 6);
+            const int kj = u.kc >> 5;
+            const uint32_t desc_hi32 = (uint32_t)(u.desc_hi >> 32);
+            const uint32_t a_lo0 = ((smem_u32(tiles) & 0x3FFFFu) >> 4) | (1u << 16);
+            const uint32_t b_lo0 = ((smem_u32(b_res) & 0x3FFFFu) >> 4) | (1u << 16);
+            const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, row_step = (uint32_t)u.kc >> 4;
+            const uint32_t b_step = (uint32_t)u.b_tile_bytes >> 4;
+            const uint32_t line_step = (uint32_t)u.win_bw * row_step;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+                const int buf = t & (u.nbuf - 1);
+                uint32_t off0 = 0;
+                if (u.win_full_width) {
+                    const int img = (int)fast_div((unsigned)tile, u.div_tpi_mul, u.div_tpi_shr);
+                    const unsigned i0 = (unsigned)(tile - img * u.win_tpi) * BLOCK_M;
+                    off0 = i0 - fast_div(i0, u.div_vw_mul, u.div_vw_shr) * (unsigned)u.win_vw;
+                }
+                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
+                    give_up(sh, u.status, 2);
+                    break;
+                }
+                tc_fence_after();
+                if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
+                    give_up(sh, u.status, 3);
+                    break;
+                }
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * u.block_n);
+                uint32_t a_line = a_lo0 + (uint32_t)stage * stage_step + off0 * row_step;
+                uint32_t b_lo = b_lo0;
+                uint32_t acc = 0;
+                for (int r = 0; r < a.kh; ++r) {
+                    uint32_t a_lo = a_line;
+                    for (int sx = 0; sx < a.kw; ++sx) {
+                        if (kj == 4) umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        else if (kj == 2) umma_slot<2>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        else umma_slot<1>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                        acc = 1;
+                        a_lo += row_step;
+                        b_lo += b_step;
+                    }
+                    a_line += line_step;
+                }
+                umma_commit(smem_u32(&sh->empty[stage]));
+                umma_commit(smem_u32(&sh->tmem_full[buf]));
+                if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps) {
+        // ---------------------------------------------------------------- epilogue
+        const int ew = warp - EPI_WARP0;
+        const int quad = warp & 3;
+        const int slot = ew >> 2;
+        const int part = slot % u.cs;
+        const int turn = slot / u.cs;
+        const int col_lo = part * u.part_n;
+        const int ncols = min(u.block_n - col_lo, u.part_n);
+        const int tile_step = u.bi * (int)gridDim.x;
+        for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles; t += u.bi, tile += tile_step) {
+            const int buf = t & (u.nbuf - 1);
+            const int img = (int)fast_div((unsigned)tile, u.div_tpi_mul, u.div_tpi_shr);
+            const unsigned i = (unsigned)(tile - img * u.win_tpi) * BLOCK_M + (unsigned)(quad * 32 + lane);   // this lane's virtual pixel
+            const int y = (int)fast_div(i, u.div_vw_mul, u.div_vw_shr);
+            const int xq = (int)i - y * u.win_vw;
+            const bool valid = xq < a.w_out && y < a.h_out;
+            uint8_t *orow = (uint8_t *)a.out + (((long long)img * a.h_out + y) * a.w_out + xq) * a.out_c_total + a.out_c_offset;
+            if (!mbar_wait_warp(smem_u32(&sh->tmem_full[buf]), (uint32_t)((t >> u.lg_nbuf) & 1), &sh->abort_flag, lane)) {
+                give_up(sh, u.status, 4);
+                break;
+            }
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.block_n + col_lo);
+            const int ngroups = ncols >> 4;
+            int accA[16], accB[16];
+            tmem_ld16(t_row, accA);
+            for (int gi = 0; gi < ngroups; gi += 2) {
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int gcur = gi + hf;
+                    if (gcur >= ngroups) break;
+                    const int co0 = col_lo + (gcur << 4);
+                    int4 ca[4];
+                    const int4 *cap = (const int4 *)(u.c_a + co0);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + g);
+                    tmem_ld_wait();
+                    if (gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
+                    int V[16];
+                    epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), a, u);
+                    uint4 o;
+                    if (EPI == EPI_FAST || a.out_dtype == ICONV_U8) {
+                        o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
+                        o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
+                    } else {
+                        o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
+                        o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
+                    }
+                    if (valid && co0 < a.c_out) *(uint4 *)(orow + co0) = o;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (sh->abort_flag) {
+        volatile int never = 0;
+        if (warp == 0 && lane == 0) {
+            if (b_issued) mbar_wait(smem_u32(&sh->b_full), 0, &never);
+            if (last_stage >= 0) mbar_wait(smem_u32(&sh->full[last_stage]), last_parity, &never);
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000) {}
+        }
+        if (warp == MMA_WARP && lane == 0) {
+            umma_commit(smem_u32(&sh->drain));
+            mbar_wait(smem_u32(&sh->drain), 0, &never);
+        }
         __syncthreads();
     }
     if (warp == MMA_WARP) {
@@ -899,6 +1128,25 @@ int encode_activation_map(const iconv_plan_t *p, const void *x, CUtensorMap *map
 {
     const iconv_desc &d = p->d;
     return encode_im2col_map(p, x, d.c_in, d.in_c_total, d.in_c_offset, d.h, d.w, d.kh, d.kw, d.stride, d.pad, map);
+}
+
+// Tiled 4-D map over the activation slice for window mode: dims {c_in, w, h, n}, box
+// {KC, win_bw, win_bh, 1}; coordinates outside the image read as zero.
+int encode_patch_map(const iconv_plan_t *p, const void *x, CUtensorMap *map)
+{
+    const iconv_desc &d = p->d;
+    const cuuint64_t dims[4] = {(cuuint64_t)d.c_in, (cuuint64_t)d.w, (cuuint64_t)d.h, (cuuint64_t)d.n};
+    const cuuint64_t strides[3] = {(cuuint64_t)d.in_c_total, (cuuint64_t)d.in_c_total * d.w, (cuuint64_t)d.in_c_total * d.w * d.h};
+    const cuuint32_t box[4] = {(cuuint32_t)p->kc, (cuuint32_t)p->win_bw, (cuuint32_t)p->win_bh, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, (void *)((const uint8_t *)x + d.in_c_offset), dims, strides, box,
+                                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p->kc), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (patch map) failed with %d", (int)r);
+        return ICONV_ERR_UNSUPPORTED;
+    }
+    return ICONV_OK;
 }
 
 int encode_projection_map(const iconv_plan_t *p, const void *x, CUtensorMap *map)
@@ -1142,15 +1390,18 @@ int umma_geometry(iconv_plan_t *p)
     // epilogue geometry: slots per TMEM lane quadrant, split between a tile's columns (cs)
     // and tiles in flight (bi)
     const int slots = p->epi_warps / 4;
-    p->cs = p->block_n > 128 ? 2 : 1;
-    p->bi = slots / p->cs;
-    if (p->bi > p->nbuf) p->bi = p->nbuf;
+    p->bi = slots < p->nbuf ? slots : p->nbuf;
+    p->cs = slots / p->bi;
+    while (p->cs > 1 && p->block_n < 32 * p->cs) p->cs /= 2;     // at least 32 columns per warp
+    if (p->block_n > 128 && p->cs < 2) { p->cs = 2; p->bi = slots / 2 ? slots / 2 : 1; if (p->bi > p->nbuf) p->bi = p->nbuf; }
     p->epi_warps = 4 * p->cs * p->bi;
-    p->half_n = p->cs == 2 ? (p->block_n / 2 + 15) / 16 * 16 : p->block_n;
+    p->half_n = p->cs > 1 ? (p->block_n / p->cs + 15) / 16 * 16 : p->block_n;
     {
         // staged piece: the widest power of two dividing every warp's row width, at most 64
         // bytes of 8-bit outputs or 128 bytes of int32 (two pieces fit half the warp's staging)
-        const int w0 = p->half_n * esz, w1 = (p->block_n - (p->cs - 1) * p->half_n) * esz;
+        int last = p->block_n - (p->cs - 1) * p->half_n;
+        while (last <= 0) { --p->cs; p->epi_warps = 4 * p->cs * p->bi; p->half_n = p->cs > 1 ? (p->block_n / p->cs + 15) / 16 * 16 : p->block_n; last = p->block_n - (p->cs - 1) * p->half_n; }
+        const int w0 = p->half_n * esz, w1 = last * esz;
         int pb = esz == 4 ? 128 : 64;
         while (pb > 16 && (w0 % pb || w1 % pb)) pb /= 2;
         p->piece_bytes = pb;
@@ -1160,6 +1411,50 @@ int umma_geometry(iconv_plan_t *p)
 }
 
 int umma_epilogue_safe() { return EPI_SAFE; }
+
+// Window mode for this layer?  Fills the plan's win_* fields when it applies: stride 1, a filter
+// wider than one tap, one channel chunk, one N tile, no skip, an 8-bit output whose epilogue is
+// one of the 32-bit forms, the filter bank and at least two patches in shared memory, and
+// tiles that are mostly real pixels.
+void window_plan(iconv_plan_t *p)
+{
+    const iconv_desc &d = p->d;
+    p->window = 0;
+    if (d.kernel == ICONV_KERNEL_UMMA_IM2COL) return;
+    if (d.stride != 1 || d.kh * d.kw < 2 || d.proj_weights || d.skip_dtype >= 0 || d.out_dtype == ICONV_I32) return;
+    if (p->c_in_pad != p->kc || p->c_out_pad != p->block_n) return;
+    if (p->epi != EPI_FAST && p->epi != EPI_SAFE) return;
+    const int taps = d.kh * d.kw;
+    const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
+    const long long bank = (long long)b_tile * taps;
+    const int wp = p->w_out + d.kw - 1;
+    int vw, bw, bh, full_width;
+    if (p->w_out >= 128) {                      // strips of 128 pixels inside one row
+        vw = (p->w_out + 127) / 128 * 128; bw = 128 + d.kw - 1; bh = d.kh; full_width = 0;
+    } else {                                    // the padded width, tiles run across rows
+        vw = wp; bw = wp; bh = (wp - 1 + 127) / wp + d.kh; full_width = 1;
+    }
+    if (bw > 256 || bh > 256) return;
+    const long long patch = ((long long)(bh * bw + d.kw) * p->kc + 1023) / 1024 * 1024;
+    if (patch > 64 * 1024) return;
+    const long long room = MAX_SMEM - 1024 - (long long)sizeof(Shared) - bank;
+    if (room < 2 * patch) return;
+    const long long tpi = ((long long)p->h_out * vw + BLOCK_M - 1) / BLOCK_M;
+    if ((long long)p->h_out * p->w_out * 10 < tpi * BLOCK_M * 6) return;          // under 60 % real pixels
+    if (tpi * d.n >= (1ll << 31) / BLOCK_M) return;
+    p->window = 1;
+    p->win_vw = vw; p->win_bw = bw; p->win_bh = bh; p->win_full_width = full_width; p->win_tpi = (int)tpi;
+    p->win_patch_bytes = (int)patch;
+    p->win_stages = (int)(room / patch < 6 ? room / patch : 6);
+    // sixteen epilogue warps: no staging memory is needed here
+    const int slots = 4;
+    p->bi = slots < p->nbuf ? slots : p->nbuf;
+    p->cs = slots / p->bi;
+    while (p->cs > 1 && p->block_n < 32 * p->cs) p->cs /= 2;
+    p->half_n = p->cs > 1 ? (p->block_n / p->cs + 15) / 16 * 16 : p->block_n;
+    while (p->cs > 1 && p->block_n - (p->cs - 1) * p->half_n <= 0) { --p->cs; p->half_n = p->cs > 1 ? (p->block_n / p->cs + 15) / 16 * 16 : p->block_n; }
+    p->epi_warps = 4 * p->cs * p->bi;
+}
 
 // 2-D tiled map over the packed weights p->w_packed, [c_out_pad][taps * c_in_pad].
 int umma_encode_weight_map(iconv_plan_t *p)
@@ -1241,6 +1536,17 @@ int umma_setup(iconv_plan_t *p)
     p->q_shift = d.out_dtype != ICONV_I32 ? d.shift[0] : 0;
     p->q_h = d.out_dtype != ICONV_I32 ? d.h_i[0] : 0;
 
+    window_plan(p);
+    if (p->window) {
+        static bool win_attr_set = false;
+        if (!win_attr_set) {
+            ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+            ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+            win_attr_set = true;
+        }
+        CUtensorMap probe2;     // the tiled patch map must be encodable as well
+        if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
+    }
     return ICONV_OK;
 }
 
@@ -1252,10 +1558,13 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         return ICONV_ERR_ALIGN;
     }
     CUtensorMap tmap_x;
-    int rc = encode_activation_map(p, a.x, &tmap_x);
+    int rc = p->window ? encode_patch_map(p, a.x, &tmap_x) : encode_activation_map(p, a.x, &tmap_x);
     if (rc != ICONV_OK) return rc;
 
     UmmaArgs u;
+    u.win_vw = p->win_vw; u.win_bw = p->win_bw; u.win_bh = p->win_bh; u.win_full_width = p->win_full_width; u.win_tpi = p->win_tpi;
+    find_divisor((unsigned)(p->win_tpi > 0 ? p->win_tpi : 1), u.div_tpi_mul, u.div_tpi_shr);
+    find_divisor((unsigned)(p->win_vw > 0 ? p->win_vw : 1), u.div_vw_mul, u.div_vw_shr);
     u.m_total = (long long)d.n * p->h_out * p->w_out;
     u.m_tiles = (int)((u.m_total + BLOCK_M - 1) / BLOCK_M);
     u.n_tiles = p->c_out_pad / p->block_n;
@@ -1335,6 +1644,18 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         int dev = 0;
         ICONV_CUDA_TRY(cudaGetDevice(&dev));
         ICONV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    }
+    if (p->window) {
+        u.m_tiles = p->win_tpi * d.n;
+        u.stages = p->win_stages;
+        u.stage_bytes = p->win_patch_bytes;
+        const unsigned wgrid = (unsigned)(u.m_tiles < sms ? u.m_tiles : sms);
+        const size_t wsmem = 1024 + (size_t)u.stages * u.stage_bytes + (size_t)u.b_tile_bytes * u.taps + sizeof(Shared);
+        if (wsmem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
+        if (p->epi == EPI_FAST) umma_window_kernel<EPI_FAST><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
+        else umma_window_kernel<EPI_SAFE><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        return ICONV_OK;
     }
     const long long tiles = (long long)u.m_tiles * u.n_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);

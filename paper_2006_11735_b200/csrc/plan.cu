@@ -8,7 +8,7 @@ int choose_kernel(iconv_plan_t *p)
     const int want = p->d.kernel;
     if (p->d.proj_weights) {
         // a fused projection skip exists on the tensor-core path only
-        if (want != ICONV_KERNEL_AUTO && want != ICONV_KERNEL_UMMA) {
+        if (want != ICONV_KERNEL_AUTO && want != ICONV_KERNEL_UMMA && want != ICONV_KERNEL_UMMA_IM2COL) {
             set_error("iconv_plan: a fused projection needs the tensor-core kernel");
             return ICONV_ERR_UNSUPPORTED;
         }
@@ -21,7 +21,7 @@ int choose_kernel(iconv_plan_t *p)
         p->kernel = ICONV_KERNEL_DIRECT;
         return ICONV_OK;
     }
-    if (want == ICONV_KERNEL_UMMA) {
+    if (want == ICONV_KERNEL_UMMA || want == ICONV_KERNEL_UMMA_IM2COL) {
         const int rc = umma_supported(p);
         if (rc != ICONV_OK) return rc;
         p->kernel = ICONV_KERNEL_UMMA;

@@ -118,6 +118,9 @@ class Network:
     def kernels(self) -> dict:
         return {k: B.KERNEL_NAME[B.iconv_plan_kernel(p)] for k, p in self.plans.items()}
 
+    def describe(self) -> dict:
+        return {k: B.iconv_plan_describe(p) for k, p in self.plans.items()}
+
     def conv_macs(self) -> dict:
         """True multiply-accumulates per forward of every convolution (M * N * K)."""
         out = {}

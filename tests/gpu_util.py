@@ -35,7 +35,7 @@ class Fenced:
 def gpu_conv(X, W, b, mul, shift, h_i, *, stride=1, pad=0, in_dtype=B.U8, in_c_offset=0, c_in=None,
              out_dtype=B.U8, out_c_total=None, out_c_offset=0, brelu=True, out_lo=0, out_hi=255, out_zero=0,
              skip=None, skip_dtype=-1, skip_c_offset=0, skip_mul=1, skip_shift=0, kernel=B.KERNEL_AUTO,
-             fill=0x5A):
+             fill=0x5A, describe=None):
     n, h, w, in_c_total = X.shape
     c_out, kh, kw, wc = W.shape
     c_in = wc if c_in is None else c_in
@@ -49,6 +49,8 @@ def gpu_conv(X, W, b, mul, shift, h_i, *, stride=1, pad=0, in_dtype=B.U8, in_c_o
                         skip_mul=skip_mul, skip_shift=skip_shift, kernel=kernel,
                         weights=W, bias=b, mul=mul, shift=shift, h_i=h_i)
     try:
+        if describe is not None:
+            describe.append(B.iconv_plan_describe(plan))
         xd = dev(X)
         sd = dev(skip) if skip is not None else None
         out = Fenced((n, ho, wo, out_c_total), _NP[out_dtype], fill)

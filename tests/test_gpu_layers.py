@@ -188,16 +188,36 @@ UMMA_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("shape", UMMA_SHAPES, ids=lambda s: "x".join(map(str, s)))
-def test_tensor_core_kernel_matches_oracle(shape):
+WINDOW_SHAPES = [
+    # stride-1 filters the plan runs in window mode (one patch load per tile); n, h, w, c_in, c_out, k, stride, pad
+    (2, 5, 256, 64, 64, 3, 1, 1),       # VDSR rows: two 128-pixel strips per row
+    (1, 6, 260, 64, 32, 3, 1, 1),       # ragged third strip
+    (1, 9, 250, 64, 16, 5, 1, 2),       # VRCNN 5x5 branch, 16 output channels
+    (2, 30, 26, 48, 16, 3, 1, 1),       # 48 channels in a 64-byte row
+    (3, 28, 28, 128, 128, 3, 1, 1),     # 128-byte rows, tiles across rows, ragged last tile per image
+    (2, 20, 17, 32, 64, 3, 1, 0),       # no padding: the output is narrower than the input
+    (1, 40, 33, 16, 256, 3, 1, 1),      # two column halves per tile
+    (2, 12, 50, 64, 48, 5, 1, 4),       # padding wider than the filter needs
+]
+
+
+@pytest.mark.parametrize("shape", UMMA_SHAPES + WINDOW_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("kernel", [B.KERNEL_UMMA, B.KERNEL_UMMA_IM2COL], ids=["plan", "im2col"])
+def test_tensor_core_kernel_matches_oracle(shape, kernel):
     n, h, w, c_in, c_out, k, stride, pad = shape
     X, W, b, mul, shift, h_i = _layer(sum(shape) + 1, n, h, w, c_in, c_out, k)
     if c_out % 16:
         got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, out_dtype=B.I32, brelu=False,
-                            kernel=B.KERNEL_UMMA)
+                            kernel=kernel)
         want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, out_dtype=B.I32, brelu=False)
     else:
-        got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, kernel=B.KERNEL_UMMA)
+        text = []
+        got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, kernel=kernel, describe=text)
+        # the shapes listed for window mode must really run in it when the plan is free to choose
+        if kernel == B.KERNEL_UMMA_IM2COL:
+            assert "im2col" in text[0], text[0]
+        elif shape in WINDOW_SHAPES:
+            assert "window" in text[0], text[0]
         want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad)
         assert 0.05 < (want == 0).mean() < 0.95
     assert fam == B.KERNEL_UMMA
@@ -206,10 +226,17 @@ def test_tensor_core_kernel_matches_oracle(shape):
         bad.shape[0], bad[0], got[tuple(bad[0])], want[tuple(bad[0])])
 
 
-def test_tensor_core_kernel_signed_activations_and_large_batch_tail():
+@pytest.mark.parametrize("kernel", [B.KERNEL_UMMA, B.KERNEL_UMMA_IM2COL], ids=["plan", "im2col"])
+def test_tensor_core_kernel_signed_activations_and_large_batch_tail(kernel):
     X, W, b, mul, shift, h_i = _layer(77, 7, 19, 17, 64, 64, 3, in_dtype=B.S8)
-    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.S8, kernel=B.KERNEL_UMMA)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.S8, kernel=kernel)
     want = oracle_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.S8)
+    assert fam == B.KERNEL_UMMA and np.array_equal(got, want)
+    # window mode with the explicit-clamp epilogue (a signed output with a zero point) inside a wider tensor
+    X, W, b, mul, shift, h_i = _layer(79, 2, 21, 23, 64, 32, 3)
+    kw = dict(pad=1, out_dtype=B.S8, out_lo=-100, out_hi=100, out_zero=-90, out_c_total=64, out_c_offset=32)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, kernel=kernel, **kw)
+    want = oracle_conv(X, W, b, mul, shift, h_i, **kw)
     assert fam == B.KERNEL_UMMA and np.array_equal(got, want)
 
 
