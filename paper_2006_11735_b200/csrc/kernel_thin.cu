@@ -37,17 +37,25 @@ struct ThinArgs {
     int w4;            // thin_in: packed words per output channel
     int narrow;        // thin_in: 1 when BReLU + Eq. 4 provably fit 32 bits for every channel
     int lpp;           // thin_out: lanes per pixel (c_in / 16)
+    // x / w_out and x / (h_out * w_out) as umulhi(x, mul) >> shr (x < 2^31; mul == 0: divisor 1)
+    unsigned div_w_mul, div_w_shr, div_hw_mul, div_hw_shr;
 };
 
+__device__ __forceinline__ unsigned thin_div(unsigned x, unsigned mul, unsigned shr) { return mul ? (__umulhi(x, mul) >> shr) : x; }
+
 // SIGNED: the packed input bytes are int8 (stored int8, or raw uint8 turned into raw - 128 by
-// flipping bit 7); otherwise uint8.
-template <bool SIGNED>
+// flipping bit 7); otherwise uint8.  KH, KW: the filter size when known at compile time (0:
+// read from the arguments).  FAST: per-layer parameters and a proven 32-bit Eq. 4 (then the
+// thread keeps its 16 biases in registers: it serves the same channel group for every pixel).
+template <bool SIGNED, int KH, int KW, bool FAST>
 __global__ void __launch_bounds__(THIN_IN_THREADS) thin_in_kernel(const __grid_constant__ ConvArgs a, const __grid_constant__ ThinArgs t)
 {
     extern __shared__ int ws[];                       // [w4][c_out + c_out / 16]: word j of channel co at j * pitch + co + co / 16
     const int pitch = a.c_out + a.c_out / 16;         // one pad word per 16 channels: the groups of a pixel hit distinct banks
-    const int K = a.kh * a.kw;
-    for (int e = threadIdx.x; e < t.w4 * a.c_out; e += blockDim.x) {
+    const int kh = KH ? KH : a.kh, kw = KW ? KW : a.kw;
+    const int K = kh * kw;
+    const int w4 = KH ? (KH * KW + 3) / 4 : t.w4;
+    for (int e = threadIdx.x; e < w4 * a.c_out; e += blockDim.x) {
         const int co = e % a.c_out, j = e / a.c_out;
         unsigned word = 0;
         for (int b = 0; b < 4; ++b) {
@@ -60,27 +68,55 @@ __global__ void __launch_bounds__(THIN_IN_THREADS) thin_in_kernel(const __grid_c
 
     const int g = threadIdx.x % t.groups;              // this thread's 16-channel group
     const int ppb = blockDim.x / t.groups;             // pixels per block and pass
-    const long long m_total = (long long)a.n * a.h_out * a.w_out;
+    const unsigned m_total = (unsigned)((long long)a.n * a.h_out * a.w_out);
+    const unsigned hw = (unsigned)(a.h_out * a.w_out);
     const unsigned flip = a.in_dtype == ICONV_U8_RAW128 ? 0x80u : 0u;
     const uint8_t *x = (const uint8_t *)a.x;
-    for (long long m = (long long)blockIdx.x * ppb + threadIdx.x / t.groups; m < m_total; m += (long long)gridDim.x * ppb) {
-        const int ow = (int)(m % a.w_out);
-        const int oh = (int)((m / a.w_out) % a.h_out);
-        const long long img = m / ((long long)a.w_out * a.h_out);
+    const int *wg = ws + g * 17;                       // word j of this group's channel c at wg[j * pitch + c]
+    int b16[16];
+    int q_mul = 0, q_shift = 1, q_h = 0;
+    unsigned q_half = 0;
+    if (FAST) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) b16[c] = __ldg(a.bias + g * 16 + c);
+        q_mul = __ldg(a.mul); q_shift = __ldg(a.shift); q_h = __ldg(a.h_i); q_half = 1u << (q_shift - 1);
+    }
+    for (unsigned m = blockIdx.x * ppb + threadIdx.x / t.groups; m < m_total; m += gridDim.x * ppb) {
+        const unsigned img = thin_div(m, t.div_hw_mul, t.div_hw_shr);
+        const unsigned rem = m - img * hw;
+        const int oh = (int)thin_div(rem, t.div_w_mul, t.div_w_shr);
+        const int ow = (int)rem - oh * a.w_out;
+        const uint8_t *ximg = x + (size_t)img * a.h * a.w_;
         unsigned xw[THIN_MAX_W4];
 #pragma unroll
         for (int j = 0; j < THIN_MAX_W4; ++j) xw[j] = 0;
-        int k = 0;
-        for (int r = 0; r < a.kh; ++r) {
-            const int ih = oh * a.stride - a.pad + r;
-            for (int s = 0; s < a.kw; ++s, ++k) {
-                const int iw = ow * a.stride - a.pad + s;
-                unsigned v = 0;                        // zero padding, after the re-normalisation
-                if (ih >= 0 && ih < a.h && iw >= 0 && iw < a.w_) v = (unsigned)__ldg(x + (img * a.h + ih) * a.w_ + iw) ^ flip;
-                const unsigned sh = (unsigned)(k & 3) * 8u;
+        if (KH) {
 #pragma unroll
-                for (int j = 0; j < THIN_MAX_W4; ++j)
-                    if (j == (k >> 2)) xw[j] |= v << sh;
+            for (int r = 0; r < (KH ? KH : 1); ++r) {
+                const int ih = oh * a.stride - a.pad + r;
+                const bool row_in = ih >= 0 && ih < a.h;
+#pragma unroll
+                for (int s = 0; s < (KW ? KW : 1); ++s) {
+                    const int k = r * KW + s;
+                    const int iw = ow * a.stride - a.pad + s;
+                    unsigned v = 0;                    // zero padding, after the re-normalisation
+                    if (row_in && iw >= 0 && iw < a.w_) v = (unsigned)__ldg(ximg + ih * a.w_ + iw) ^ flip;
+                    xw[k >> 2] |= v << ((k & 3) * 8);
+                }
+            }
+        } else {
+            int k = 0;
+            for (int r = 0; r < kh; ++r) {
+                const int ih = oh * a.stride - a.pad + r;
+                for (int s = 0; s < kw; ++s, ++k) {
+                    const int iw = ow * a.stride - a.pad + s;
+                    unsigned v = 0;
+                    if (ih >= 0 && ih < a.h && iw >= 0 && iw < a.w_) v = (unsigned)__ldg(ximg + ih * a.w_ + iw) ^ flip;
+                    const unsigned sh = (unsigned)(k & 3) * 8u;
+#pragma unroll
+                    for (int j = 0; j < THIN_MAX_W4; ++j)
+                        if (j == (k >> 2)) xw[j] |= v << sh;
+                }
             }
         }
         unsigned packed[4];
@@ -93,62 +129,100 @@ __global__ void __launch_bounds__(THIN_IN_THREADS) thin_in_kernel(const __grid_c
                 int U = 0;
 #pragma unroll
                 for (int j = 0; j < THIN_MAX_W4; ++j)
-                    if (j < t.w4) {
-                        const int wv = ws[j * pitch + co + g];
+                    if (j < w4) {
+                        const int wv = wg[j * pitch + c];
                         U = SIGNED ? dp4a_ss((int)xw[j], wv, U) : dp4a_us(xw[j], wv, U);
                     }
-                const int pc = a.per_channel ? co : 0;
-                if (t.narrow) {
-                    int y = U + __ldg(a.bias + co);
-                    const int shift = __ldg(a.shift + pc);
-                    y = max(min(y, __ldg(a.h_i + pc)), 0);
-                    const int v = (int)(((unsigned)y * (unsigned)__ldg(a.mul + pc) + (1u << (shift - 1))) >> shift);
+                if (FAST) {
+                    const int y = max(min(U + b16[c], q_h), 0);
+                    const int v = (int)(((unsigned)y * (unsigned)q_mul + q_half) >> q_shift);
                     V[e] = min(max(v + a.out_zero, a.out_lo), a.out_hi);
                 } else {
-                    V[e] = requant_tail((long long)U + __ldg(a.bias + co), a.brelu, __ldg(a.h_i + pc), __ldg(a.mul + pc),
-                                        __ldg(a.shift + pc), a.out_zero, a.out_lo, a.out_hi);
+                    const int pc = a.per_channel ? co : 0;
+                    if (t.narrow) {
+                        int y = U + __ldg(a.bias + co);
+                        const int shift = __ldg(a.shift + pc);
+                        y = max(min(y, __ldg(a.h_i + pc)), 0);
+                        const int v = (int)(((unsigned)y * (unsigned)__ldg(a.mul + pc) + (1u << (shift - 1))) >> shift);
+                        V[e] = min(max(v + a.out_zero, a.out_lo), a.out_hi);
+                    } else {
+                        V[e] = requant_tail((long long)U + __ldg(a.bias + co), a.brelu, __ldg(a.h_i + pc), __ldg(a.mul + pc),
+                                            __ldg(a.shift + pc), a.out_zero, a.out_lo, a.out_hi);
+                    }
                 }
             }
             packed[q] = (V[0] & 0xff) | ((V[1] & 0xff) << 8) | ((V[2] & 0xff) << 16) | ((unsigned)(V[3] & 0xff) << 24);
         }
-        *(uint4 *)((uint8_t *)a.out + m * a.out_c_total + a.out_c_offset + g * 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        *(uint4 *)((uint8_t *)a.out + (size_t)m * a.out_c_total + a.out_c_offset + g * 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
     }
 }
 
-template <bool SIGNED>
+// K3: a 3x3 filter, whose nine 16-byte weight slices the lane keeps in registers.
+template <bool SIGNED, bool K3>
 __global__ void __launch_bounds__(256) thin_out_kernel(const __grid_constant__ ConvArgs a, const __grid_constant__ ThinArgs t)
 {
     const int lane = threadIdx.x & 31;
     const int ppw = 32 / t.lpp;                        // pixels per warp and pass
     const int lp = lane / t.lpp, part = lane - lp * t.lpp;
     const bool active = lp < ppw;
-    const long long m_total = (long long)a.n * a.h_out * a.w_out;
-    const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
-    const long long warp_id = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const unsigned m_total = (unsigned)((long long)a.n * a.h_out * a.w_out);
+    const unsigned hw = (unsigned)(a.h_out * a.w_out);
+    const unsigned warps = gridDim.x * (blockDim.x >> 5);
+    const unsigned warp_id = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const uint8_t *x = (const uint8_t *)a.x + a.in_c_offset + part * 16;
     const int8_t *w = a.w + part * 16;
-    for (long long m0 = warp_id * ppw; m0 < m_total; m0 += warps * ppw) {      // the same trip count for every lane of a warp
-        const long long m = m0 + lp;
+    int4 wr[9];
+    if (K3) {
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) wr[tap] = __ldg((const int4 *)(w + tap * a.c_in));
+    }
+    const int bias = __ldg(a.bias);
+    for (unsigned m0 = warp_id * ppw; m0 < m_total; m0 += warps * ppw) {      // the same trip count for every lane of a warp
+        const unsigned m = m0 + lp;
         const bool live = active && m < m_total;
         int U = 0;
         if (live) {
-            const int ow = (int)(m % a.w_out);
-            const int oh = (int)((m / a.w_out) % a.h_out);
-            const long long img = m / ((long long)a.w_out * a.h_out);
-            for (int r = 0; r < a.kh; ++r) {
-                const int ih = oh * a.stride - a.pad + r;
-                if (ih < 0 || ih >= a.h) continue;
-                for (int s = 0; s < a.kw; ++s) {
-                    const int iw = ow * a.stride - a.pad + s;
-                    if (iw < 0 || iw >= a.w_) continue;
-                    const uint4 xv = __ldg((const uint4 *)(x + ((img * a.h + ih) * a.w_ + iw) * a.in_c_total));
-                    const int4 wv = __ldg((const int4 *)(w + (r * a.kw + s) * a.c_in));
-                    if (SIGNED) {
-                        U = dp4a_ss((int)xv.x, wv.x, U); U = dp4a_ss((int)xv.y, wv.y, U);
-                        U = dp4a_ss((int)xv.z, wv.z, U); U = dp4a_ss((int)xv.w, wv.w, U);
-                    } else {
-                        U = dp4a_us(xv.x, wv.x, U); U = dp4a_us(xv.y, wv.y, U);
-                        U = dp4a_us(xv.z, wv.z, U); U = dp4a_us(xv.w, wv.w, U);
+            const unsigned img = thin_div(m, t.div_hw_mul, t.div_hw_shr);
+            const unsigned rem = m - img * hw;
+            const int oh = (int)thin_div(rem, t.div_w_mul, t.div_w_shr);
+            const int ow = (int)rem - oh * a.w_out;
+            const uint8_t *ximg = x + (size_t)img * a.h * a.w_ * a.in_c_total;
+            if (K3) {
+#pragma unroll
+                for (int r = 0; r < 3; ++r) {
+                    const int ih = oh * a.stride - a.pad + r;
+                    if (ih < 0 || ih >= a.h) continue;
+#pragma unroll
+                    for (int s = 0; s < 3; ++s) {
+                        const int iw = ow * a.stride - a.pad + s;
+                        if (iw < 0 || iw >= a.w_) continue;
+                        const uint4 xv = __ldg((const uint4 *)(ximg + (size_t)(ih * a.w_ + iw) * a.in_c_total));
+                        const int4 wv = wr[r * 3 + s];
+                        if (SIGNED) {
+                            U = dp4a_ss((int)xv.x, wv.x, U); U = dp4a_ss((int)xv.y, wv.y, U);
+                            U = dp4a_ss((int)xv.z, wv.z, U); U = dp4a_ss((int)xv.w, wv.w, U);
+                        } else {
+                            U = dp4a_us(xv.x, wv.x, U); U = dp4a_us(xv.y, wv.y, U);
+                            U = dp4a_us(xv.z, wv.z, U); U = dp4a_us(xv.w, wv.w, U);
+                        }
+                    }
+                }
+            } else {
+                for (int r = 0; r < a.kh; ++r) {
+                    const int ih = oh * a.stride - a.pad + r;
+                    if (ih < 0 || ih >= a.h) continue;
+                    for (int s = 0; s < a.kw; ++s) {
+                        const int iw = ow * a.stride - a.pad + s;
+                        if (iw < 0 || iw >= a.w_) continue;
+                        const uint4 xv = __ldg((const uint4 *)(ximg + (size_t)(ih * a.w_ + iw) * a.in_c_total));
+                        const int4 wv = __ldg((const int4 *)(w + (r * a.kw + s) * a.c_in));
+                        if (SIGNED) {
+                            U = dp4a_ss((int)xv.x, wv.x, U); U = dp4a_ss((int)xv.y, wv.y, U);
+                            U = dp4a_ss((int)xv.z, wv.z, U); U = dp4a_ss((int)xv.w, wv.w, U);
+                        } else {
+                            U = dp4a_us(xv.x, wv.x, U); U = dp4a_us(xv.y, wv.y, U);
+                            U = dp4a_us(xv.z, wv.z, U); U = dp4a_us(xv.w, wv.w, U);
+                        }
                     }
                 }
             }
@@ -156,10 +230,10 @@ __global__ void __launch_bounds__(256) thin_out_kernel(const __grid_constant__ C
         int total = U;
         for (int k = 1; k < t.lpp; ++k) total += __shfl_down_sync(0xffffffffu, U, k);
         if (live && part == 0) {
-            long long Y = (long long)total + __ldg(a.bias);
+            long long Y = (long long)total + bias;
             if (a.skip_dtype >= 0)
-                Y += round_shift64((long long)load_skip(a.skip, m * a.skip_c_total + a.skip_c_offset, a.skip_dtype) * a.skip_mul, a.skip_shift);
-            const long long oi = m * a.out_c_total + a.out_c_offset;
+                Y += round_shift64((long long)load_skip(a.skip, (long long)m * a.skip_c_total + a.skip_c_offset, a.skip_dtype) * a.skip_mul, a.skip_shift);
+            const long long oi = (long long)m * a.out_c_total + a.out_c_offset;
             if (a.out_dtype == ICONV_I32) {
                 ((int32_t *)a.out)[oi] = (int32_t)Y;
             } else {
@@ -169,6 +243,15 @@ __global__ void __launch_bounds__(256) thin_out_kernel(const __grid_constant__ C
             }
         }
     }
+}
+
+void thin_divisor(unsigned d, unsigned &mul, unsigned &shr)
+{
+    if (d <= 1) { mul = 0; shr = 0; return; }
+    unsigned lg = 0;
+    while ((1ull << lg) < d) ++lg;
+    mul = (unsigned)(((1ull << (31 + lg)) + d - 1) / d);
+    shr = lg - 1;
 }
 
 bool is_thin_in(const iconv_desc &d)
@@ -227,20 +310,35 @@ int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     t.narrow = p->thin_narrow;
     t.lpp = d.c_in / 16;
     const bool is_signed = d.in_dtype != ICONV_U8;
+    if (m_total >= (1ll << 31) - 65536) { set_error("thin kernels: more than 2^31 output pixels"); return ICONV_ERR_UNSUPPORTED; }
+    thin_divisor((unsigned)p->w_out, t.div_w_mul, t.div_w_shr);
+    thin_divisor((unsigned)(p->h_out * p->w_out), t.div_hw_mul, t.div_hw_shr);
     if (is_thin_in(d)) {
         const int ppb = THIN_IN_THREADS / t.groups;
         long long blocks = (m_total + ppb - 1) / ppb;
         if (blocks > 148ll * 16) blocks = 148ll * 16;
         const size_t smem = (size_t)t.w4 * (d.c_out + d.c_out / 16) * sizeof(int);
-        if (is_signed) thin_in_kernel<true><<<(unsigned)blocks, THIN_IN_THREADS, smem, stream>>>(a, t);
-        else thin_in_kernel<false><<<(unsigned)blocks, THIN_IN_THREADS, smem, stream>>>(a, t);
+        const bool fast = p->thin_narrow && !d.per_channel;
+        const int k = d.kh == d.kw ? d.kh : 0;
+#define ICONV_THIN_IN(S, KH, KW, F) thin_in_kernel<S, KH, KW, F><<<(unsigned)blocks, THIN_IN_THREADS, smem, stream>>>(a, t)
+#define ICONV_THIN_IN_K(S, F)                                    \
+    do {                                                         \
+        if (k == 3) ICONV_THIN_IN(S, 3, 3, F);                   \
+        else if (k == 5) ICONV_THIN_IN(S, 5, 5, F);              \
+        else ICONV_THIN_IN(S, 0, 0, F);                          \
+    } while (0)
+        if (is_signed) { if (fast) ICONV_THIN_IN_K(true, true); else ICONV_THIN_IN_K(true, false); }
+        else { if (fast) ICONV_THIN_IN_K(false, true); else ICONV_THIN_IN_K(false, false); }
+#undef ICONV_THIN_IN_K
+#undef ICONV_THIN_IN
     } else {
         if (t.lpp > 32) { set_error("thin kernels: c_in too wide"); return ICONV_ERR_UNSUPPORTED; }
         const int ppw = 32 / t.lpp;
         long long blocks = (m_total + 8ll * ppw - 1) / (8ll * ppw);
         if (blocks > 148ll * 16) blocks = 148ll * 16;
-        if (is_signed) thin_out_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(a, t);
-        else thin_out_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(a, t);
+        const bool k3 = d.kh == 3 && d.kw == 3;
+        if (is_signed) { if (k3) thin_out_kernel<true, true><<<(unsigned)blocks, 256, 0, stream>>>(a, t); else thin_out_kernel<true, false><<<(unsigned)blocks, 256, 0, stream>>>(a, t); }
+        else { if (k3) thin_out_kernel<false, true><<<(unsigned)blocks, 256, 0, stream>>>(a, t); else thin_out_kernel<false, false><<<(unsigned)blocks, 256, 0, stream>>>(a, t); }
     }
     ICONV_CUDA_TRY(cudaGetLastError());
     return ICONV_OK;
