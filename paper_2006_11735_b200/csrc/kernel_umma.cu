@@ -139,6 +139,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
         if (mbar_test_wait(bar, parity)) return true;
+        if (i >= 4) __nanosleep(20);      // a thread that polls flat out slows the MMA issuer's own shared-memory traffic
         if ((i & 1023u) == 0) {
             if (*abort_flag) return false;
             const long long now = clock64();
@@ -235,6 +236,21 @@ __device__ __forceinline__ void umma_slot(uint32_t d_tmem, uint32_t a_lo, uint32
     umma_i8_split(d_tmem, a_lo, b_lo, desc_hi, idesc, accumulate_first);
 #pragma unroll
     for (int j = 1; j < KJ; ++j) umma_i8_split(d_tmem, a_lo + 2u * j, b_lo + 2u * j, desc_hi, idesc, 1u);
+}
+// All slots of one pipeline stage (im2col kernel): slot e of the stage is k-iteration ki + e.  A
+// fused projection's iterations (ki < p_iters) go to the second accumulator tile.
+template <int KJ>
+__device__ __forceinline__ void umma_stage(uint32_t d_tmem, uint32_t block_n, uint32_t a_lo, uint32_t b_lo, uint32_t slot_step,
+                                           uint32_t b_step, uint32_t desc_hi, uint32_t idesc, uint32_t idesc_p, int ki, int in_stage,
+                                           int p_iters)
+{
+    for (int e = 0; e < in_stage; ++e, ++ki) {
+        const bool in_proj = ki < p_iters;
+        umma_slot<KJ>(in_proj ? d_tmem + block_n : d_tmem, a_lo, b_lo, desc_hi, in_proj ? idesc_p : idesc,
+                      (uint32_t)(ki != 0 && ki != p_iters));
+        a_lo += slot_step;
+        b_lo += b_step;
+    }
 }
 // The mbarrier receives one arrival once every MMA issued so far by this thread is done.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
@@ -647,19 +663,11 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step;
                     uint32_t b_lo = u.resident_b ? sb : a_lo + slot_a_step;
                     const int in_stage = min(u.kg, k_iters - ki);
-                    for (int e = 0; e < in_stage; ++e, ++ki) {
-                        // the projection's iterations fill the second accumulator tile, the layer's own the first
-                        const uint32_t acc = (uint32_t)(ki != 0 && ki != u.p_iters);
-                        const bool in_proj = ki < u.p_iters;
-                        const uint32_t d = in_proj ? d_tmem + (uint32_t)u.block_n : d_tmem;
-                        const uint32_t id = in_proj ? u.idesc_p : u.idesc;
-                        if (kj == 4) umma_slot<4>(d, a_lo, b_lo, desc_hi32, id, acc);
-                        else if (kj == 2) umma_slot<2>(d, a_lo, b_lo, desc_hi32, id, acc);
-                        else umma_slot<1>(d, a_lo, b_lo, desc_hi32, id, acc);
-                        a_lo += slot_step;
-                        b_lo += b_step;
-                    }
-                    if (u.resident_b) sb = b_lo;
+                    if (kj == 4) umma_stage<4>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, u.p_iters);
+                    else if (kj == 2) umma_stage<2>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, u.p_iters);
+                    else umma_stage<1>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, u.p_iters);
+                    ki += in_stage;
+                    if (u.resident_b) sb = b_lo + (uint32_t)in_stage * b_step;
                     umma_commit(smem_u32(&sh->empty[stage]));   // frees the stage when these MMAs are done
                     if (++stage == u.stages) { stage = 0; parity ^= 1u; }
                 }
@@ -857,7 +865,10 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 // absolute shared-memory address, so any start row reads what TMA wrote).  Virtual pixels
 // beyond the real width are computed and dropped.  The filter bank is resident, the epilogue
 // stores straight from registers (a tile is not a contiguous run of real pixels).
-template <int EPI>
+// KH, KW, KJ: filter size and MMAs per tap when known at compile time (0: read from the
+// arguments).  The issuing thread runs alone: every branch it takes costs it a resolution
+// latency nothing hides, so the common filters get straight-line issue code.
+template <int EPI, int KH, int KW, int KJ>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                    const __grid_constant__ ConvArgs a, const __grid_constant__ UmmaArgs u)
@@ -957,18 +968,29 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * u.block_n);
                 uint32_t a_line = a_lo0 + (uint32_t)stage * stage_step + off0 * row_step;
                 uint32_t b_lo = b_lo0;
-                uint32_t acc = 0;
-                for (int r = 0; r < a.kh; ++r) {
-                    uint32_t a_lo = a_line;
-                    for (int sx = 0; sx < a.kw; ++sx) {
-                        if (kj == 4) umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                        else if (kj == 2) umma_slot<2>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                        else umma_slot<1>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                        acc = 1;
-                        a_lo += row_step;
-                        b_lo += b_step;
+                if (KH) {
+#pragma unroll
+                    for (int r = 0; r < (KH ? KH : 1); ++r) {
+#pragma unroll
+                        for (int sx = 0; sx < (KW ? KW : 1); ++sx)
+                            umma_slot<KJ ? KJ : 1>(d_tmem, a_line + (uint32_t)sx * row_step, b_lo + (uint32_t)(r * KW + sx) * b_step, desc_hi32,
+                                                   u.idesc, (uint32_t)((r | sx) != 0));
+                        a_line += line_step;
                     }
-                    a_line += line_step;
+                } else {
+                    uint32_t acc = 0;
+                    for (int r = 0; r < a.kh; ++r) {
+                        uint32_t a_lo = a_line;
+                        for (int sx = 0; sx < a.kw; ++sx) {
+                            if (kj == 4) umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                            else if (kj == 2) umma_slot<2>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                            else umma_slot<1>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                            acc = 1;
+                            a_lo += row_step;
+                            b_lo += b_step;
+                        }
+                        a_line += line_step;
+                    }
                 }
                 umma_commit(smem_u32(&sh->empty[stage]));
                 umma_commit(smem_u32(&sh->tmem_full[buf]));
@@ -1540,8 +1562,14 @@ int umma_setup(iconv_plan_t *p)
     if (p->window) {
         static bool win_attr_set = false;
         if (!win_attr_set) {
-            ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-            ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+#define ICONV_WIN_ATTR(E)                                                                                                          \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 5, 5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM))
+            ICONV_WIN_ATTR(EPI_FAST);
+            ICONV_WIN_ATTR(EPI_SAFE);
+#undef ICONV_WIN_ATTR
             win_attr_set = true;
         }
         CUtensorMap probe2;     // the tiled patch map must be encodable as well
@@ -1652,8 +1680,17 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         const unsigned wgrid = (unsigned)(u.m_tiles < sms ? u.m_tiles : sms);
         const size_t wsmem = 1024 + (size_t)u.stages * u.stage_bytes + (size_t)u.b_tile_bytes * u.taps + sizeof(Shared);
         if (wsmem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
-        if (p->epi == EPI_FAST) umma_window_kernel<EPI_FAST><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
-        else umma_window_kernel<EPI_SAFE><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
+        const int kj = p->kc >> 5;
+#define ICONV_WIN(E)                                                                                                                \
+    do {                                                                                                                            \
+        if (d.kh == 3 && d.kw == 3 && kj == 2) umma_window_kernel<E, 3, 3, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);      \
+        else if (d.kh == 3 && d.kw == 3 && kj == 4) umma_window_kernel<E, 3, 3, 4><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
+        else if (d.kh == 5 && d.kw == 5 && kj == 2) umma_window_kernel<E, 5, 5, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
+        else umma_window_kernel<E, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);                        \
+    } while (0)
+        if (p->epi == EPI_FAST) ICONV_WIN(EPI_FAST);
+        else ICONV_WIN(EPI_SAFE);
+#undef ICONV_WIN
         ICONV_CUDA_TRY(cudaGetLastError());
         return ICONV_OK;
     }
