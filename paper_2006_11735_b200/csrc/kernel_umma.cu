@@ -302,181 +302,161 @@ __device__ __forceinline__ void give_up(Shared *sh, int *status, int code)
     atomicCAS(status, 0, code);
 }
 
-// One group of 16 consecutive output channels of one pixel: accumulators in, 16 output
-// values (8-bit variants) or 16 int32 (raw) out.  `sk` holds the 16 staged skip bytes.
-template <int EPI>
-__device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int *V, const int4 *ca4, int co0, long long m, bool row_ok,
-                                           uint4 sk, const ConvArgs &a, const UmmaArgs &u)
+// The scalars the epilogue needs, copied once per thread into registers (read through the kernel
+// parameters inside the unrolled element loops they cost an indexed constant load each).
+struct EpiScalars {
+    int q_mul, q_shift, q_half, q_h;
+    int skip_mul, skip_shift;
+    unsigned skip_xor;
+    int out_zero, out_lo, out_hi, tail;
+    int per_channel, proj32, brelu, skip_dtype, out_dtype, c_out;
+};
+
+__device__ __forceinline__ EpiScalars epi_scalars(const ConvArgs &a, const UmmaArgs &u)
 {
-    if (EPI == EPI_PROJ) {
-        // S = accp + b_p is the projection's int32 Y.  32-bit form (bounds proven at plan time):
-        // Y = U + ((accp * skip_mul + C) >> skip_shift), C = b_p * skip_mul + 2^(skip_shift-1) + (b << skip_shift);
-        // otherwise the rescale runs in 64 bits with the two biases apart.
-        const int4 *cb4 = (const int4 *)(u.c_b + co0);
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int4 c = ca4[g];
-            const int cc[4] = {c.x, c.y, c.z, c.w};
-            int bp[4] = {0, 0, 0, 0};
-            if (!u.proj32) { const int4 b4 = __ldg(cb4 + g); bp[0] = b4.x; bp[1] = b4.y; bp[2] = b4.z; bp[3] = b4.w; }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                int h = u.q_h, mul = u.q_mul, shift = u.q_shift, half = u.q_half;
-                if (a.per_channel) {
-                    h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
-                    shift = __ldg(u.c_shift + co0 + 4 * g + e); half = (int)(1u << (shift - 1));
-                }
-                int y;
-                if (u.proj32) {
-                    y = acc[4 * g + e] + ((accp[4 * g + e] * a.skip_mul + cc[e]) >> a.skip_shift);
-                    y = max(min(y, h), 0);
-                } else {
-                    long long Y = (long long)acc[4 * g + e] + cc[e] +
-                                  round_shift64(((long long)accp[4 * g + e] + bp[e]) * a.skip_mul, a.skip_shift);
-                    Y = Y < 0 ? 0 : (Y > (long long)h ? (long long)h : Y);
-                    y = (int)Y;
-                }
-                int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
-                if (u.tail) v = min(max(v + a.out_zero, a.out_lo), a.out_hi);
-                V[4 * g + e] = v;
-            }
-        }
-        return;
+    EpiScalars e;
+    e.q_mul = u.q_mul; e.q_shift = u.q_shift; e.q_half = u.q_half; e.q_h = u.q_h;
+    e.skip_mul = a.skip_mul; e.skip_shift = a.skip_shift; e.skip_xor = u.skip_xor;
+    e.out_zero = a.out_zero; e.out_lo = a.out_lo; e.out_hi = a.out_hi; e.tail = u.tail;
+    e.per_channel = a.per_channel; e.proj32 = u.proj32; e.brelu = a.brelu; e.skip_dtype = a.skip_dtype;
+    e.out_dtype = a.out_dtype; e.c_out = a.c_out;
+    return e;
+}
+
+// BReLU clamp + 32-bit Eq. 4 (+ zero point / range when they are not provable no-ops)
+__device__ __forceinline__ int requant32(int y, int h, int mul, int half, int shift, const EpiScalars &s)
+{
+    y = max(min(y, h), 0);
+    int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
+    if (s.tail) v = min(max(v + s.out_zero, s.out_lo), s.out_hi);
+    return v;
+}
+
+// Eq. 4 parameters of output channel co: the layer's scalars, or (PC) the channel's own.
+template <bool PC>
+__device__ __forceinline__ void chan_params(const EpiScalars &s, const UmmaArgs &u, int co, int &h, int &mul, int &half, int &shift)
+{
+    if (PC) {
+        h = __ldg(u.c_h + co); mul = __ldg(u.c_mul + co); shift = __ldg(u.c_shift + co); half = (int)(1u << (shift - 1));
+    } else {
+        h = s.q_h; mul = s.q_mul; shift = s.q_shift; half = s.q_half;
     }
+}
+
+// One group of 16 consecutive output channels of one pixel: accumulators in, 16 output
+// values (8-bit variants) or 16 int32 (raw) out.  ca4: the variant's per-channel additive
+// constants of the group; `sk`: the 16 staged skip bytes; accp: the projection's accumulators.
+// PC: per-channel mul / shift / h_i.
+template <int EPI, bool PC>
+__device__ __forceinline__ void epilogue16_pc(const int *acc, const int *accp, int *V, const int4 *ca4, int co0, long long m, bool row_ok,
+                                              uint4 sk, const EpiScalars &s, const ConvArgs &a, const UmmaArgs &u)
+{
+    int ca[16];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) { ca[4 * g] = ca4[g].x; ca[4 * g + 1] = ca4[g].y; ca[4 * g + 2] = ca4[g].z; ca[4 * g + 3] = ca4[g].w; }
+    int h, mul, half, shift;
+
     if (EPI == EPI_RAW) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int4 c = ca4[g];
-            V[4 * g] = acc[4 * g] + c.x; V[4 * g + 1] = acc[4 * g + 1] + c.y;
-            V[4 * g + 2] = acc[4 * g + 2] + c.z; V[4 * g + 3] = acc[4 * g + 3] + c.w;
-        }
+        for (int k = 0; k < 16; ++k) V[k] = acc[k] + ca[k];
         return;
     }
     if (EPI == EPI_FAST) {
         // (U + b) * mul + half = U * mul + C with C = b * mul + half; the shift is arithmetic and the
         // u8 saturation that follows stands for both BReLU clamps (proven at plan time)
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int4 c = ca4[g];
-            V[4 * g] = (acc[4 * g] * u.q_mul + c.x) >> u.q_shift;
-            V[4 * g + 1] = (acc[4 * g + 1] * u.q_mul + c.y) >> u.q_shift;
-            V[4 * g + 2] = (acc[4 * g + 2] * u.q_mul + c.z) >> u.q_shift;
-            V[4 * g + 3] = (acc[4 * g + 3] * u.q_mul + c.w) >> u.q_shift;
-        }
+        for (int k = 0; k < 16; ++k) V[k] = (acc[k] * s.q_mul + ca[k]) >> s.q_shift;
         return;
     }
     if (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8) {
-        // Y = U + ((s * skip_mul + C) >> skip_shift) with C = (b << skip_shift) + skip_half - z * skip_mul,
-        // where s is the stored byte as an unsigned number and z its zero (0, or 128 for raw-128 and
+        // Y = U + ((sv * skip_mul + C) >> skip_shift) with C = (b << skip_shift) + skip_half - z * skip_mul,
+        // where sv is the stored byte as an unsigned number and z its zero (0, or 128 for raw-128 and
         // offset-binary int8): the bias rides inside the rounding shift, which is exact.
-        const unsigned w4[4] = {sk.x ^ u.skip_xor, sk.y ^ u.skip_xor, sk.z ^ u.skip_xor, sk.w ^ u.skip_xor};
+        const unsigned w4[4] = {sk.x ^ s.skip_xor, sk.y ^ s.skip_xor, sk.z ^ s.skip_xor, sk.w ^ s.skip_xor};
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int4 c = ca4[g];
-            const int cc[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int sv = (int)__byte_perm(w4[g], 0, 0x4440 + e);
-                int y = acc[4 * g + e] + ((sv * a.skip_mul + cc[e]) >> a.skip_shift);
-                if (EPI == EPI_FAST_SKIP8) {
-                    V[4 * g + e] = (y * u.q_mul + u.q_half) >> u.q_shift;
-                } else {
-                    int h = u.q_h, mul = u.q_mul, shift = u.q_shift, half = u.q_half;
-                    if (a.per_channel) {
-                        h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
-                        shift = __ldg(u.c_shift + co0 + 4 * g + e); half = (int)(1u << (shift - 1));
-                    }
-                    y = max(min(y, h), 0);
-                    int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
-                    if (u.tail) v = min(max(v + a.out_zero, a.out_lo), a.out_hi);
-                    V[4 * g + e] = v;
-                }
-            }
-        }
-        return;
-    }
-    if (EPI == EPI_SAFE || EPI == EPI_SAFE_SKIP32) {
-        int4 s32[4] = {make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0)};
-        if (EPI == EPI_SAFE_SKIP32 && row_ok) {
-            const int4 *sp = (const int4 *)((const int32_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0);
-#pragma unroll
-            for (int g = 0; g < 4; ++g)
-                s32[g] = (co0 + 4 * g < a.c_out) ? __ldg(sp + g) : make_int4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int4 c = ca4[g];
-            const int cc[4] = {c.x, c.y, c.z, c.w};
-            const int ss[4] = {s32[g].x, s32[g].y, s32[g].z, s32[g].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                int h = u.q_h, mul = u.q_mul, shift = u.q_shift, half = u.q_half;
-                if (a.per_channel) {
-                    h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
-                    shift = __ldg(u.c_shift + co0 + 4 * g + e); half = (int)(1u << (shift - 1));
-                }
-                int y;
-                if (EPI == EPI_SAFE_SKIP32) {
-                    long long Y = (long long)acc[4 * g + e] + cc[e] + round_shift64((long long)ss[e] * a.skip_mul, a.skip_shift);
-                    Y = Y < 0 ? 0 : (Y > (long long)h ? (long long)h : Y);
-                    y = (int)Y;
-                } else {
-                    y = max(min(acc[4 * g + e] + cc[e], h), 0);
-                }
-                int v = (int)(((unsigned)y * (unsigned)mul + (unsigned)half) >> shift);
-                if (u.tail) v = min(max(v + a.out_zero, a.out_lo), a.out_hi);
-                V[4 * g + e] = v;
-            }
-        }
-        return;
-    }
-    // EPI_WIDE: everything at run time, 64-bit products, skip read straight from global memory
-    {
-        uint4 sk8 = make_uint4(0, 0, 0, 0);
-        int4 s32[4] = {make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0)};
-        if (a.skip_dtype >= 0 && row_ok && co0 < a.c_out) {
-            if (a.skip_dtype == ICONV_I32) {
-                const int4 *sp = (const int4 *)((const int32_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0);
-#pragma unroll
-                for (int g = 0; g < 4; ++g)
-                    s32[g] = (co0 + 4 * g < a.c_out) ? __ldg(sp + g) : make_int4(0, 0, 0, 0);
+        for (int k = 0; k < 16; ++k) {
+            const int sv = (int)__byte_perm(w4[k >> 2], 0, 0x4440 + (k & 3));
+            const int y = acc[k] + ((sv * s.skip_mul + ca[k]) >> s.skip_shift);
+            if (EPI == EPI_FAST_SKIP8) {
+                V[k] = (y * s.q_mul + s.q_half) >> s.q_shift;
             } else {
-                sk8 = __ldg((const uint4 *)((const uint8_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0));
+                chan_params<PC>(s, u, co0 + k, h, mul, half, shift);
+                V[k] = requant32(y, h, mul, half, shift, s);
             }
         }
-        const unsigned w4[4] = {sk8.x, sk8.y, sk8.z, sk8.w};
+        return;
+    }
+    if (EPI == EPI_PROJ) {
+        // S = accp + b_p is the projection's int32 Y.  32-bit form (bounds proven at plan time):
+        // Y = U + ((accp * skip_mul + C) >> skip_shift), C = b_p * skip_mul + 2^(skip_shift-1) + (b << skip_shift);
+        // otherwise the rescale runs in 64 bits with the two biases apart.
+        if (s.proj32) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int4 c = ca4[g];
-            const int cc[4] = {c.x, c.y, c.z, c.w};
-            const int ss[4] = {s32[g].x, s32[g].y, s32[g].z, s32[g].w};
+            for (int k = 0; k < 16; ++k) {
+                chan_params<PC>(s, u, co0 + k, h, mul, half, shift);
+                V[k] = requant32(acc[k] + ((accp[k] * s.skip_mul + ca[k]) >> s.skip_shift), h, mul, half, shift, s);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                chan_params<PC>(s, u, co0 + k, h, mul, half, shift);
+                long long Y = (long long)acc[k] + ca[k] +
+                              round_shift64(((long long)accp[k] + __ldg(u.c_b + co0 + k)) * s.skip_mul, s.skip_shift);
+                Y = Y < 0 ? 0 : (Y > (long long)h ? (long long)h : Y);
+                V[k] = requant32((int)Y, h, mul, half, shift, s);
+            }
+        }
+        return;
+    }
+    if (EPI == EPI_SAFE) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            chan_params<PC>(s, u, co0 + k, h, mul, half, shift);
+            V[k] = requant32(acc[k] + ca[k], h, mul, half, shift, s);
+        }
+        return;
+    }
+    // EPI_SAFE_SKIP32 and EPI_WIDE read the skip straight from global memory
+    const bool have = s.skip_dtype >= 0 && row_ok && co0 < s.c_out;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        int ss[4] = {0, 0, 0, 0};
+        if (have && s.skip_dtype == ICONV_I32 && co0 + 4 * g < s.c_out) {
+            const int4 t = __ldg((const int4 *)((const int32_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0) + g);
+            ss[0] = t.x; ss[1] = t.y; ss[2] = t.z; ss[3] = t.w;
+        } else if (have && s.skip_dtype != ICONV_I32) {
+            const unsigned w = __ldg((const unsigned *)((const uint8_t *)a.skip + m * a.skip_c_total + a.skip_c_offset + co0) + g);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                long long Y = (long long)acc[4 * g + e] + cc[e];
-                if (a.skip_dtype >= 0) {
-                    int sv;
-                    if (a.skip_dtype == ICONV_I32) {
-                        sv = ss[e];
-                    } else {
-                        const unsigned byte = (w4[g] >> (8 * e)) & 0xffu;
-                        sv = a.skip_dtype == ICONV_S8 ? (int)(int8_t)byte
-                                                      : (int)byte - (a.skip_dtype == ICONV_U8_RAW128 ? 128 : 0);
-                    }
-                    Y += round_shift64((long long)sv * a.skip_mul, a.skip_shift);
-                }
-                if (a.out_dtype == ICONV_I32) {
-                    V[4 * g + e] = (int)Y;
-                } else {
-                    int h = u.q_h, mul = u.q_mul, shift = u.q_shift;
-                    if (a.per_channel) {
-                        h = __ldg(u.c_h + co0 + 4 * g + e); mul = __ldg(u.c_mul + co0 + 4 * g + e);
-                        shift = __ldg(u.c_shift + co0 + 4 * g + e);
-                    }
-                    V[4 * g + e] = requant_tail(Y, a.brelu, h, mul, shift, a.out_zero, a.out_lo, a.out_hi);
-                }
+                const unsigned byte = (w >> (8 * e)) & 0xffu;
+                ss[e] = s.skip_dtype == ICONV_S8 ? (int)(int8_t)byte : (int)byte - (s.skip_dtype == ICONV_U8_RAW128 ? 128 : 0);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int k = 4 * g + e;
+            chan_params<PC>(s, u, co0 + k, h, mul, half, shift);
+            long long Y = (long long)acc[k] + ca[k];
+            if (s.skip_dtype >= 0) Y += round_shift64((long long)ss[e] * s.skip_mul, s.skip_shift);
+            if (EPI == EPI_SAFE_SKIP32) {
+                Y = Y < 0 ? 0 : (Y > (long long)h ? (long long)h : Y);
+                V[k] = requant32((int)Y, h, mul, half, shift, s);
+            } else {
+                V[k] = s.out_dtype == ICONV_I32 ? (int)Y : requant_tail(Y, s.brelu, h, mul, shift, s.out_zero, s.out_lo, s.out_hi);
             }
         }
     }
+}
+
+template <int EPI>
+__device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int *V, const int4 *ca4, int co0, long long m, bool row_ok,
+                                           uint4 sk, const EpiScalars &s, const ConvArgs &a, const UmmaArgs &u)
+{
+    // the fast forms are planned for per-layer parameters only
+    if (EPI != EPI_RAW && EPI != EPI_FAST && EPI != EPI_FAST_SKIP8 && s.per_channel)
+        epilogue16_pc<EPI, true>(acc, accp, V, ca4, co0, m, row_ok, sk, s, a, u);
+    else
+        epilogue16_pc<EPI, false>(acc, accp, V, ca4, co0, m, row_ok, sk, s, a, u);
 }
 
 }  // namespace
@@ -703,6 +683,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const unsigned row_off = (unsigned)lane * (unsigned)pb;
         const unsigned row_swz = pb >= 32 ? (((unsigned)lane >> swz_shift) & (unsigned)(pb / 16 - 1)) : 0u;
         const int tile_step = u.bi * (int)gridDim.x;
+        const EpiScalars es = epi_scalars(a, u);
         int mine = 0, pieces = 0;
         bool ok = true;
 
@@ -773,7 +754,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         tmem_ld_wait();
                         if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)(pc + cc + 16), hf ? accA : accB);
                         int V[16];
-                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, a, u);
+                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, es, a, u);
                         if (esz_rt == 4) {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) {
@@ -1008,6 +989,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         const int col_lo = part * u.part_n;
         const int ncols = min(u.block_n - col_lo, u.part_n);
         const int tile_step = u.bi * (int)gridDim.x;
+        const EpiScalars es = epi_scalars(a, u);
         for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles; t += u.bi, tile += tile_step) {
             const int buf = t & (u.nbuf - 1);
             const int img = (int)fast_div((unsigned)tile, u.div_tpi_mul, u.div_tpi_shr);
@@ -1038,7 +1020,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     tmem_ld_wait();
                     if (gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
                     int V[16];
-                    epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), a, u);
+                    epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), es, a, u);
                     uint4 o;
                     if (EPI == EPI_FAST || a.out_dtype == ICONV_U8) {
                         o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
