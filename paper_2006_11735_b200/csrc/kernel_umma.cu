@@ -1362,14 +1362,16 @@ int umma_geometry(iconv_plan_t *p)
     const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
     const long long bank = (long long)b_tile * k_iters * n_tiles;
     const int fixed = (int)sizeof(Shared) + 2048;
-    // Epilogue-heavy layers (one or two k-iterations per tile) get sixteen epilogue warps, the
-    // others eight and a deeper pipeline.  A stage groups kg k-iterations (at most 48 KB) as
-    // long as three stages still fit: the MMA issuer's wait + commit round costs about 400
-    // cycles whatever the stage holds.
+    // Epilogue-heavy layers (many output columns per k-iteration, more with a skip to rescale) get
+    // sixteen epilogue warps, the others eight and a deeper pipeline.  A stage groups kg
+    // k-iterations (at most 48 KB) as long as three stages still fit (two for a tile that is a
+    // single stage): the MMA issuer's wait + commit round costs about 400 cycles whatever the
+    // stage holds.
     p->resident_b = 0;
     p->epi_warps = 0;
     p->kg = 1;
-    for (int ew = (k_iters <= 2 ? 16 : 8); ew >= 8 && !p->epi_warps; ew -= 8) {
+    const int weight = p->block_n * (proj ? 7 : (d.skip_dtype >= 0 ? 5 : 2)) / (2 * k_iters);
+    for (int ew = (weight >= 100 ? 16 : 8); ew >= 8 && !p->epi_warps; ew -= 8) {
         const int avail = MAX_SMEM - fixed - ew * EPI_WARP_SMEM;
         const int want = 2;
         int room = 0, slot = 0;
