@@ -192,8 +192,8 @@ ICONV_API int ipool_avg_requant(const void *x, void *out, int32_t n, int32_t h, 
  *
  * The arithmetic is iconv_forward's with brelu = 1 and per-layer mul / shift / h_i; results are
  * bit-identical to a planned forward of the same layer.  Returns ICONV_ERR_SHAPE with the sizes in
- * iconv_last_error() when n * (h_out + 3) * w_out * 64 + 131072 exceeds ICONV_STEM_STATIC_BYTES
- * (40 images of 224 x 224 fit), ICONV_ERR_ARG unless c_out is a multiple of 16 in [16, 256],
+ * iconv_last_error() when n * (h_out + 3) * (w_out + 3) * 16 + 196608 exceeds ICONV_STEM_STATIC_BYTES
+ * (157 images of 224 x 224 fit), ICONV_ERR_ARG unless c_out is a multiple of 16 in [16, 256],
  * 1 <= shift <= 31 and h_i * mul + 2^(shift-1) < 2^32.  Asynchronous on cuda_stream.
  *
  * The first call on each device looks up the array's device address (the GPU with that array

@@ -2,13 +2,13 @@
 // the ResNet-shaped networks).  Three channels are far too narrow for TMA (16-byte rows at
 // least) and K = 147 is awkward for the tensor cores, so the layer runs in two steps:
 //
-//   1. a repack kernel rewrites the image as T[n][Y][X][64]: a 2x2 space-to-depth (which
-//      turns the stride-2 7x7 filter into a stride-1 4x4 filter over 12 channels, padded to
-//      16) with the four filter columns of every output position laid side by side, and
-//      the re-normalisation (raw - 128, Section 3.4.1) and the zero padding applied on the
-//      way:   T[n][Y][X][S*16 + (dy*2+dx)*3 + c] = in[n][2(Y-2)+dy][2(X+S-2)+dx][c]
-//   2. the tensor-core kernel runs a kh=4, kw=1, c_in=64, stride-1, unpadded convolution on
-//      T with weights rearranged the same way: out(oh, ow) = sum_R T[oh+R][ow] . W'[R].
+//   1. a repack kernel rewrites the image as T[n][Y][X][16]: a 2x2 space-to-depth, which
+//      turns the stride-2 7x7 filter into a stride-1 4x4 filter over 12 channels (padded to
+//      16), with the re-normalisation (raw - 128, Section 3.4.1) and the zero padding applied
+//      on the way:   T[n][Y][X][(dy*2+dx)*3 + c] = in[n][2(Y-2)+dy][2(X-2)+dx][c]
+//   2. the tensor-core kernel runs a 4x4, 16-channel, stride-1, unpadded convolution on T
+//      (in window mode: one patch of T per tile) with weights rearranged the same way:
+//      out(oh, ow) = sum_{R,S} T[oh+R][ow+S] . W'[R][S],  W'[R][S][(dy*2+dx)*3+c] = W[2R+dy-1][2S+dx-1][c].
 //
 // The sum is the same integers in another order, so the result is bit-identical.
 #include <cstring>
@@ -20,16 +20,14 @@ namespace iconv {
 
 namespace {
 
-// One thread writes 16 bytes: position (n, Y, X) and filter column S of T.
+// One thread writes the 16 bytes of one position (n, Y, X) of T.
 __global__ void __launch_bounds__(256)
 stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int n, int h, int w, int hp, int wp,
                    int raw128)
 {
-    const long long total = (long long)n * hp * wp * 4;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
-         e += (long long)gridDim.x * blockDim.x) {
-        const int S = (int)(e & 3);
-        const long long pos = e >> 2;
+    const long long total = (long long)n * hp * wp;
+    for (long long pos = (long long)blockIdx.x * blockDim.x + threadIdx.x; pos < total;
+         pos += (long long)gridDim.x * blockDim.x) {
         const int X = (int)(pos % wp);
         const int Y = (int)((pos / wp) % hp);
         const int img = (int)(pos / ((long long)wp * hp));
@@ -39,7 +37,7 @@ stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int 
             const int ih = 2 * (Y - 2) + dy;
 #pragma unroll
             for (int dx = 0; dx < 2; ++dx) {
-                const int iw = 2 * (X + S - 2) + dx;
+                const int iw = 2 * (X - 2) + dx;
                 if (ih < 0 || ih >= h || iw < 0 || iw >= w) continue;    // zero padding
                 const uint8_t *p = in + (((long long)img * h + ih) * w + iw) * 3;
 #pragma unroll
@@ -51,7 +49,7 @@ stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int 
                 }
             }
         }
-        *(uint4 *)(T + pos * 64 + S * 16) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+        *(uint4 *)(T + pos * 16) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
     }
 }
 
@@ -70,9 +68,9 @@ int stem_supported(const iconv_plan_t *p)
 int stem_setup(iconv_plan_t *p)
 {
     const iconv_desc &d = p->d;
-    const int hp = p->h_out + 3, wp = p->w_out;
-    // W'[co][R][0][S*16 + (dy*2+dx)*3 + c] = W[co][2R+dy-1][2S+dx-1][c]  (0 where an index is -1)
-    std::vector<int8_t> w2((size_t)d.c_out * 4 * 64, 0);
+    const int hp = p->h_out + 3, wp = p->w_out + 3;
+    // W'[co][R][S][(dy*2+dx)*3 + c] = W[co][2R+dy-1][2S+dx-1][c]  (0 where an index is -1)
+    std::vector<int8_t> w2((size_t)d.c_out * 16 * 16, 0);
     for (int co = 0; co < d.c_out; ++co)
         for (int R = 0; R < 4; ++R)
             for (int S = 0; S < 4; ++S)
@@ -81,17 +79,17 @@ int stem_setup(iconv_plan_t *p)
                         const int r = 2 * R + dy - 1, s = 2 * S + dx - 1;
                         if (r < 0 || s < 0) continue;
                         for (int c = 0; c < 3; ++c)
-                            w2[((size_t)co * 4 + R) * 64 + S * 16 + (dy * 2 + dx) * 3 + c] =
+                            w2[(((size_t)co * 4 + R) * 4 + S) * 16 + (dy * 2 + dx) * 3 + c] =
                                 d.weights[(((size_t)co * 7 + r) * 7 + s) * 3 + c];
                     }
     iconv_desc in = d;
     in.h = hp;
     in.w = wp;
-    in.c_in = 64;
-    in.in_c_total = 64;
+    in.c_in = 16;
+    in.in_c_total = 16;
     in.in_c_offset = 0;
     in.kh = 4;
-    in.kw = 1;
+    in.kw = 4;
     in.stride = 1;
     in.pad = 0;
     in.in_dtype = d.in_dtype == ICONV_U8 ? ICONV_U8 : ICONV_S8;
@@ -99,7 +97,7 @@ int stem_setup(iconv_plan_t *p)
     in.weights = w2.data();
     int rc = iconv_plan(&in, &p->inner);
     if (rc != ICONV_OK) return rc;
-    p->workspace_bytes = (size_t)d.n * hp * wp * 64;
+    p->workspace_bytes = (size_t)d.n * hp * wp * 16;
     if (p->workspace_bytes) ICONV_CUDA_TRY(cudaMalloc(&p->workspace, p->workspace_bytes));
     return ICONV_OK;
 }
@@ -107,8 +105,8 @@ int stem_setup(iconv_plan_t *p)
 int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
 {
     const iconv_desc &d = p->d;
-    const int hp = p->h_out + 3, wp = p->w_out;
-    const long long total = (long long)d.n * hp * wp * 4;
+    const int hp = p->h_out + 3, wp = p->w_out + 3;
+    const long long total = (long long)d.n * hp * wp;
     long long blocks = (total + 255) / 256;
     if (blocks > 148ll * 32) blocks = 148ll * 32;
     stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)p->workspace, d.n, d.h, d.w,
@@ -131,7 +129,7 @@ namespace iconv {
 
 namespace {
 
-constexpr size_t STEM_STATIC_W_BYTES = 64 * 1024;       // rearranged weights: 256 channels x 4 x 64
+constexpr size_t STEM_STATIC_W_BYTES = 128 * 1024;      // rearranged weights: 256 channels x 16 taps x 32 bytes
 constexpr size_t STEM_STATIC_PAR_BYTES = 64 * 1024;     // {c_a, mul, shift, h_i} x 256 int32 (+ slack)
 constexpr size_t STEM_STATIC_T_OFFSET = STEM_STATIC_W_BYTES + STEM_STATIC_PAR_BYTES;
 
@@ -156,17 +154,16 @@ int stem_static_base(unsigned char **base)
     return ICONV_OK;
 }
 
-// Writes W'[co][R][S*16 + (dy*2+dx)*3 + c] = W[co][2R+dy-1][2S+dx-1][c] (0 where an index is
+// Writes W'[co][R][S][(dy*2+dx)*3 + c] = W[co][2R+dy-1][2S+dx-1][c], 32 bytes per tap (0 where an index is
 // -1, in the padding lanes and in the padded channels) and the epilogue constants.  Every
 // byte the GEMM reads is written here, so the array's previous contents never matter.
 __global__ void __launch_bounds__(256)
 stem_static_prepare_kernel(const int8_t *__restrict__ w, const int32_t *__restrict__ bias, int8_t *__restrict__ w2,
                            int32_t *__restrict__ par, int c_out, int c_out_pad, int mul, int shift, int h_i, int *status)
 {
-    const int total = c_out_pad * 256;
+    const int total = c_out_pad * 512;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
-        const int j = e & 63, R = (e >> 6) & 3, co = e >> 8;
-        const int S = j >> 4, k = j & 15;
+        const int k = e & 31, S = (e >> 5) & 3, R = (e >> 7) & 3, co = e >> 9;
         int8_t v = 0;
         if (co < c_out && k < 12) {
             const int tap = k / 3, c = k - 3 * tap;
@@ -213,8 +210,8 @@ extern "C" int iconv_stem_forward_static(const istem_desc *sd, const void *x, co
         return ICONV_ERR_ARG;
     }
     const int h_out = (sd->h + 6 - 7) / 2 + 1, w_out = (sd->w + 6 - 7) / 2 + 1;
-    const int hp = h_out + 3, wp = w_out;
-    const unsigned long long t_bytes = (unsigned long long)sd->n * hp * wp * 64ull;
+    const int hp = h_out + 3, wp = w_out + 3;
+    const unsigned long long t_bytes = (unsigned long long)sd->n * hp * wp * 16ull;
     if (STEM_STATIC_T_OFFSET + t_bytes > (unsigned long long)ICONV_STEM_STATIC_BYTES) {
         set_error("iconv_stem_forward_static: %d images of %d x %d need %llu bytes of scratch, the static array holds %llu",
                   sd->n, sd->h, sd->w, STEM_STATIC_T_OFFSET + t_bytes, (unsigned long long)ICONV_STEM_STATIC_BYTES);
@@ -240,15 +237,15 @@ extern "C" int iconv_stem_forward_static(const istem_desc *sd, const void *x, co
     iconv_plan_s tmp;
     iconv_desc &d = tmp.d;
     memset(&d, 0, sizeof(d));
-    d.n = sd->n; d.h = hp; d.w = wp; d.c_in = 64; d.c_out = sd->c_out; d.kh = 4; d.kw = 1; d.stride = 1; d.pad = 0;
-    d.in_dtype = sd->in_dtype == ICONV_U8 ? ICONV_U8 : ICONV_S8; d.in_c_total = 64; d.in_c_offset = 0;
+    d.n = sd->n; d.h = hp; d.w = wp; d.c_in = 16; d.c_out = sd->c_out; d.kh = 4; d.kw = 4; d.stride = 1; d.pad = 0;
+    d.in_dtype = sd->in_dtype == ICONV_U8 ? ICONV_U8 : ICONV_S8; d.in_c_total = 16; d.in_c_offset = 0;
     d.out_dtype = ICONV_U8; d.out_c_total = sd->out_c_total; d.out_c_offset = sd->out_c_offset;
     d.brelu = 1; d.per_channel = 0; d.out_lo = sd->out_lo; d.out_hi = sd->out_hi; d.out_zero = sd->out_zero;
     d.skip_dtype = -1; d.kernel = ICONV_KERNEL_UMMA;
     tmp.h_out = h_out; tmp.w_out = w_out; tmp.kernel = ICONV_KERNEL_UMMA;
     rc = umma_geometry(&tmp);
     if (rc != ICONV_OK) return rc;
-    if ((size_t)tmp.c_out_pad * 256 > STEM_STATIC_W_BYTES || (size_t)tmp.c_out_pad * 16 > STEM_STATIC_PAR_BYTES) {
+    if ((size_t)tmp.c_out_pad * 16 * tmp.c_in_pad > STEM_STATIC_W_BYTES || tmp.c_in_pad != 32 || (size_t)tmp.c_out_pad * 20 > STEM_STATIC_PAR_BYTES) {
         set_error("iconv_stem_forward_static: channel count beyond the static array's weight region");
         return ICONV_ERR_SHAPE;
     }
@@ -259,10 +256,11 @@ extern "C" int iconv_stem_forward_static(const istem_desc *sd, const void *x, co
         tmp.epi = umma_epilogue_safe();      // explicit clamps: no bound on the weights is known on the host
         tmp.tail = 1;
         tmp.q_mul = sd->mul; tmp.q_shift = sd->shift; tmp.q_h = sd->h_i;
+        window_plan(&tmp);                   // one patch of T per tile where the geometry allows
 
-        stem_static_prepare_kernel<<<(tmp.c_out_pad * 256 + 255) / 256, 256, 0, stream>>>(weights, bias, w2, par, sd->c_out, tmp.c_out_pad,
+        stem_static_prepare_kernel<<<(tmp.c_out_pad * 512 + 255) / 256, 256, 0, stream>>>(weights, bias, w2, par, sd->c_out, tmp.c_out_pad,
                                                                                     sd->mul, sd->shift, sd->h_i, status);
-        const long long total = (long long)sd->n * hp * wp * 4;
+        const long long total = (long long)sd->n * hp * wp;
         long long blocks = (total + 255) / 256;
         if (blocks > 148ll * 32) blocks = 148ll * 32;
         stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)x, T, sd->n, sd->h, sd->w, hp, wp,
@@ -275,9 +273,9 @@ extern "C" int iconv_stem_forward_static(const istem_desc *sd, const void *x, co
         memset(&a, 0, sizeof(a));
         a.x = T; a.skip = nullptr; a.out = out;
         a.w = w2; a.bias = par; a.mul = par + tmp.c_out_pad; a.shift = par + 2 * tmp.c_out_pad; a.h_i = par + 3 * tmp.c_out_pad;
-        a.n = d.n; a.h = d.h; a.w_ = d.w; a.c_in = 64; a.c_out = d.c_out; a.kh = 4; a.kw = 1; a.stride = 1; a.pad = 0;
+        a.n = d.n; a.h = d.h; a.w_ = d.w; a.c_in = 16; a.c_out = d.c_out; a.kh = 4; a.kw = 4; a.stride = 1; a.pad = 0;
         a.h_out = h_out; a.w_out = w_out;
-        a.in_dtype = d.in_dtype; a.in_c_total = 64; a.in_c_offset = 0;
+        a.in_dtype = d.in_dtype; a.in_c_total = 16; a.in_c_offset = 0;
         a.out_dtype = ICONV_U8; a.out_c_total = d.out_c_total; a.out_c_offset = d.out_c_offset;
         a.brelu = 1; a.per_channel = 0; a.out_lo = d.out_lo; a.out_hi = d.out_hi; a.out_zero = d.out_zero;
         a.skip_dtype = -1; a.skip_mul = 1;

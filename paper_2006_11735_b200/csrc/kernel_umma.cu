@@ -1324,6 +1324,19 @@ int umma_init_once()
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         attr_set = true;
     }
+    static bool win_attr_set = false;
+    if (!win_attr_set) {
+#define ICONV_WIN_ATTR(E)                                                                                                          \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 5, 5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 4, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM))
+        ICONV_WIN_ATTR(EPI_FAST);
+        ICONV_WIN_ATTR(EPI_SAFE);
+#undef ICONV_WIN_ATTR
+        win_attr_set = true;
+    }
     return ICONV_OK;
 }
 
@@ -1544,18 +1557,6 @@ int umma_setup(iconv_plan_t *p)
 
     window_plan(p);
     if (p->window) {
-        static bool win_attr_set = false;
-        if (!win_attr_set) {
-#define ICONV_WIN_ATTR(E)                                                                                                          \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 5, 5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM))
-            ICONV_WIN_ATTR(EPI_FAST);
-            ICONV_WIN_ATTR(EPI_SAFE);
-#undef ICONV_WIN_ATTR
-            win_attr_set = true;
-        }
         CUtensorMap probe2;     // the tiled patch map must be encodable as well
         if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
     }
@@ -1670,6 +1671,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         if (d.kh == 3 && d.kw == 3 && kj == 2) umma_window_kernel<E, 3, 3, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);      \
         else if (d.kh == 3 && d.kw == 3 && kj == 4) umma_window_kernel<E, 3, 3, 4><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
         else if (d.kh == 5 && d.kw == 5 && kj == 2) umma_window_kernel<E, 5, 5, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
+        else if (d.kh == 4 && d.kw == 4 && kj == 1) umma_window_kernel<E, 4, 4, 1><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
         else umma_window_kernel<E, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);                        \
     } while (0)
         if (p->epi == EPI_FAST) ICONV_WIN(EPI_FAST);

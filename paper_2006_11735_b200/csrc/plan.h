@@ -48,6 +48,7 @@ int umma_setup(iconv_plan_t *p);
 int umma_init_once();                        // driver entry points, shared-memory opt-in; allocates nothing
 int umma_geometry(iconv_plan_t *p);           // host-only tile / pipeline / epilogue geometry
 int umma_encode_weight_map(iconv_plan_t *p);  // TMA map over p->w_packed
+void window_plan(iconv_plan_t *p);            // window mode if the layer allows (needs p->epi); host only
 int umma_epilogue_safe();                     // id of the explicit-clamp 32-bit epilogue variant
 int thin_supported(const iconv_plan_t *p);
 int thin_setup(iconv_plan_t *p);

@@ -66,8 +66,8 @@ def test_static_scratch_first_layer_equals_the_planned_one_twice_in_a_row():
 
 
 def test_static_scratch_entry_refuses_what_does_not_fit():
-    with pytest.raises(B.IconvError) as e:      # 64 images of 224 x 224 need 52.9 MB, the array has 32 MiB
-        B.iconv_stem_forward_static(16, 16, 16, 16, 0, n=64, h=224, w=224, c_out=64, mul=100, shift=16, h_i=100000)
+    with pytest.raises(B.IconvError) as e:      # 200 images of 224 x 224 need 42.5 MB, the array has 32 MiB
+        B.iconv_stem_forward_static(16, 16, 16, 16, 0, n=200, h=224, w=224, c_out=64, mul=100, shift=16, h_i=100000)
     assert e.value.status == B.ERR_SHAPE and "scratch" in str(e.value)
     with pytest.raises(B.IconvError) as e:
         B.iconv_stem_forward_static(16, 16, 16, 16, 0, n=1, h=32, w=32, c_out=24, mul=100, shift=16, h_i=100000)
