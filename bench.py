@@ -197,6 +197,7 @@ def main():
     kernels = g.kernels()
     described = g.describe()
     macs = g.conv_macs()
+    abytes = g.algorithmic_bytes()
 
     for _ in range(args.warmup):
         g.forward(x_dev)
@@ -227,24 +228,31 @@ def main():
     launches = (len(g.steps) + sum(1 for k in kernels.values() if k == "stem")) * args.steps
 
     # per-kernel-family time inside the timed region
-    fam_ms, fam_macs, layer_ms = {}, {}, {}
+    fam_ms, fam_macs, fam_bytes, layer_ms = {}, {}, {}, {}
     for marks in all_marks:
         for (_, prev), (name, ev) in zip(marks[:-1], marks[1:]):
             dt = prev.elapsed_time(ev)
             fam = kernels.get(name, "pool")
             fam_ms[fam] = fam_ms.get(fam, 0.0) + dt
             fam_macs[fam] = fam_macs.get(fam, 0) + macs.get(name, 0)
+            fam_bytes[fam] = fam_bytes.get(fam, 0) + abytes.get(name, 0)
             layer_ms[name] = layer_ms.get(name, 0.0) + dt / args.steps
     int8_peak, hbm_peak, peak_kind = measured_peaks()
     issue_tops, issue_cycles = B.iconv_probe_mma_rate(256, 100000)     # outside every timed region
     umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
-    roofline = {"kernel": "umma_conv_kernel", "bound": "tensor", "achieved": umma_tops, "peak": int8_peak,
+    roofline = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "tensor", "achieved": umma_tops, "peak": int8_peak,
                 "unit": "TOP/s", "frac": umma_tops / int8_peak, "traffic": None, "peak_kind": peak_kind + " 2 x bf16 sustained",
                 "launches": umma_launches, "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
                 "frac_of_nominal_4500": umma_tops / NOMINAL_INT8_TOPS,
                 "issue_rate_peak": issue_tops, "frac_of_issue_rate_peak": umma_tops / issue_tops,
                 "time_share": {k: v / sum(fam_ms.values()) for k, v in fam_ms.items()}}
+    # the same launches against the memory roofline: most layers of this workload are bound by it
+    umma_gbs = fam_bytes.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e9
+    roofline_hbm = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "hbm", "achieved": umma_gbs, "peak": hbm_peak,
+                    "unit": "GB/s", "frac": umma_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind + " copy bandwidth",
+                    "algorithmic_bytes_per_step": int(sum(abytes.values())),
+                    "whole_step_gbs": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9}
 
     # ---- end to end: pinned host input in, logits out, every step ----
     D.barrier()
@@ -285,7 +293,7 @@ def main():
                 "clocks": clocks,
                 "e2e": {"value": total_images / (ms_e2e * 1e-3), "unit": UNIT,
                         "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(logits_host.numel() * logits_host.element_size())},
-                "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+                "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "cpu_baseline": cpu}
         print(json.dumps(line))
     g.close()
     D.finish()

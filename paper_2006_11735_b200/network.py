@@ -130,6 +130,29 @@ class Network:
             out[name] = out.get(name, 0) + self.n * dst.h * dst.w * op.c_out * op.c_in * op.k * op.k
         return out
 
+    def algorithmic_bytes(self) -> dict:
+        """Bytes every executed step must move at least once when the network runs layer at a time:
+        its input slice, its output slice, its skip operand and its weights (a fused projection
+        adds its own input and weights to the layer that runs it and writes nothing)."""
+        esz = {"u8": 1, "i32": 4}
+        out = {}
+        for op in self.net.ops:
+            src, dst = self.net.tensors[op.src], self.net.tensors[op.dst]
+            if isinstance(op, (MaxPool, AvgPool)):
+                out[op.name] = self.n * (src.h * src.w * src.c + dst.h * dst.w * dst.c)
+                continue
+            b = self.n * src.h * src.w * op.c_in + op.c_out * op.c_in * op.k * op.k + 4 * op.c_out
+            if op.name in self.fused:
+                name = self.fused[op.name]
+            else:
+                name = op.name
+                b += self.n * dst.h * dst.w * op.c_out * esz[dst.dtype]
+                if op.skip and op.skip in self.tensors:
+                    sk = self.net.tensors[op.skip]
+                    b += self.n * sk.h * sk.w * op.c_out * esz[sk.dtype]
+            out[name] = out.get(name, 0) + b
+        return out
+
     def forward(self, x: torch.Tensor = None, marks: list = None) -> torch.Tensor:
         """x: uint8 device tensor [n][h][w][c] (or None to reuse the resident input).
         marks: if a list, receives (op name, event recorded after that op's launch); the
