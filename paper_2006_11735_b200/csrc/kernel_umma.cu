@@ -130,17 +130,47 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait.  Returns false when the limit ran out or another role already gave up.
-// The limit is counted on the SM's own cycle counter, read only every 1024 failed polls:
-// a wait that succeeds costs no timer read.
+// Probe that may suspend the thread in hardware until the phase completes or `hint_ns` pass:
+// a suspended thread takes no issue slots from the warps that do the arithmetic.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
+// 16-byte shared-memory accesses by 32-bit shared address (no generic-pointer arithmetic)
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Bounded wait of a single-thread role (TMA producer, MMA issuer).  Returns false when the
+// limit ran out or another role already gave up.  A few plain probes first (the common short
+// wait), then suspending probes; the limit is counted on the SM's own cycle counter, read
+// only every 64 failed suspending probes, so a wait that succeeds soon costs no timer read.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (mbar_test_wait(bar, parity)) return true;
-    long long t0 = 0;
-    for (uint32_t i = 1;; ++i) {
+#pragma unroll 1
+    for (int i = 0; i < 4; ++i)
         if (mbar_test_wait(bar, parity)) return true;
-        if (i >= 4) __nanosleep(20);      // a thread that polls flat out slows the MMA issuer's own shared-memory traffic
-        if ((i & 1023u) == 0) {
+    long long t0 = 0;
+#pragma unroll 1
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity, 2000u)) return true;
+        if ((i & 63u) == 0) {
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
@@ -149,9 +179,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// The same wait taken by one lane on behalf of its warp (32 lanes polling one barrier word
-// only add shared-memory traffic).  Backs off between polls; __syncwarp orders the other
-// lanes' later reads after lane 0's acquire.
+// The wait of an epilogue warp, taken by one lane on behalf of the warp (32 lanes polling one
+// barrier word only add shared-memory traffic).  These warps are the critical path of the
+// epilogue-bound layers, so they poll (with a back-off) rather than suspend; __syncwarp
+// orders the other lanes' later reads after lane 0's acquire.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane)
 {
     int ok = 1;
@@ -718,8 +749,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const bool row_ok = m < u.m_total;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.acc_cols + col_lo);
 
-            for (int pc = 0; pc < ncols; pc += pcols, ++pieces) {
+            for (int pc = 0, piece = 0; pc < ncols; pc += pcols, ++pieces, ++piece) {
                 uint8_t *ob = obuf + (size_t)(pieces & 1) * piece_smem;
+                const uint32_t ob_row = smem_u32(ob) + row_off;                                  // this lane's staged output row
+                const uint32_t sk_row = smem_u32(sbuf) + (uint32_t)(piece * piece_smem) + row_off;   // and its staged skip row
+                const int4 *cap = (const int4 *)(u.c_a + n0 + pc);
+                const uint32_t t_piece = t_row + (uint32_t)pc;
                 // the store issued two pieces ago must have finished reading this buffer
                 if (pieces >= 2) {
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -732,7 +767,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 // they would spill)
                 constexpr bool PIPE = EPI != EPI_PROJ && EPI != EPI_SAFE_SKIP32 && EPI != EPI_WIDE;
                 int accA[16], accB[16], accpA[16];
-                if (PIPE) tmem_ld16(t_row + (uint32_t)pc, accA);
+                if (PIPE) tmem_ld16(t_piece, accA);
                 for (int gi = 0; gi < ngroups; gi += 2) {
 #pragma unroll
                     for (int hf = 0; hf < 2; ++hf) {
@@ -740,19 +775,18 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         if (gcur >= ngroups) break;
                         const int cc = gcur << 4;
                         const int co0 = n0 + pc + cc;
+                        const uint32_t goff = ((unsigned)gcur ^ row_swz) << 4;       // swizzled 16-byte chunk of the row
                         if (!PIPE) {
-                            tmem_ld16(t_row + (uint32_t)(pc + cc), accA);
-                            if (EPI == EPI_PROJ) tmem_ld16(t_row + (uint32_t)(u.block_n + pc + cc), accpA);
+                            tmem_ld16(t_piece + (uint32_t)cc, accA);
+                            if (EPI == EPI_PROJ) tmem_ld16(t_piece + (uint32_t)(u.block_n + cc), accpA);
                         }
                         int4 ca[4];
-                        const int4 *cap = (const int4 *)(u.c_a + co0);
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + g);
+                        for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + 4 * gcur + g);
                         uint4 sk = make_uint4(0, 0, 0, 0);
-                        if (SKIP8)
-                            sk = *(const uint4 *)(sbuf + (size_t)(pc / pcols) * piece_smem + row_off + (((unsigned)gcur ^ row_swz) << 4));
+                        if (SKIP8) sk = lds128(sk_row + goff);
                         tmem_ld_wait();
-                        if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)(pc + cc + 16), hf ? accA : accB);
+                        if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_piece + (uint32_t)(cc + 16), hf ? accA : accB);
                         int V[16];
                         epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, es, a, u);
                         if (esz_rt == 4) {
@@ -770,7 +804,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                 o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
                                 o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
                             }
-                            *(uint4 *)(ob + row_off + (((unsigned)gcur ^ row_swz) << 4)) = o;
+                            sts128(ob_row + goff, o);
                         }
                     }
                 }
