@@ -41,6 +41,7 @@ constexpr int BLOCK_M = 128;
 constexpr int EPI_WARPS_MAX = 16;
 constexpr int NUM_PRODUCERS = 3;          // TMA warps: one thread issues a load per 300-400 cycles, the unit takes three times that
 constexpr int MMA_WARP = NUM_PRODUCERS;
+constexpr int MMA_WARP2 = 1;           // window mode (one TMA warp): a second MMA issuer
 constexpr int EPI_WARP0 = 4;              // first epilogue warp (a multiple of 4: warp % 4 is its TMEM lane quadrant)
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS_MAX);
 constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces (+ the skip rows of one tile)
@@ -906,7 +907,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)(4 * u.cs));
         }
         mbar_init(smem_u32(&sh->b_full), 1);
-        mbar_init(smem_u32(&sh->drain), 1);
+        mbar_init(smem_u32(&sh->drain), 2);          // one arrival per MMA issuer
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -949,11 +950,17 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
         }
         __syncwarp();
-    } else if (warp == MMA_WARP) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0 && (int)blockIdx.x < num_tiles) {
-            int t = 0, stage = 0;
-            uint32_t parity = 0;
+    } else if (warp == MMA_WARP || warp == MMA_WARP2) {
+        // ---------------------------------------------------------------- MMA issuers
+        // Two threads issue alternate tiles.  Between two tiles an issuer spends several hundred
+        // cycles on its barrier round (two commits, two waits), longer than the tensor pipe's
+        // queue covers; with two issuers one thread's round hides behind the other's MMAs.
+        // Tiles are independent (own accumulator buffer, own patch), so no order is needed
+        // between the two instruction streams, and each thread's commits cover its own MMAs.
+        const int which = warp == MMA_WARP ? 0 : 1;
+        if (lane == 0 && (int)blockIdx.x + which * (int)gridDim.x < num_tiles) {
+            int t = which, stage = which % u.stages;
+            uint32_t parity = (uint32_t)((which / u.stages) & 1);
             bool ok = mbar_wait(smem_u32(&sh->b_full), 0, &sh->abort_flag);
             if (!ok) give_up(sh, u.status, 6);
             const int kj = u.kc >> 5;
@@ -963,7 +970,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, row_step = (uint32_t)u.kc >> 4;
             const uint32_t b_step = (uint32_t)u.b_tile_bytes >> 4;
             const uint32_t line_step = (uint32_t)u.win_bw * row_step;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+            for (int tile = blockIdx.x + which * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x, t += 2) {
                 const int buf = t & (u.nbuf - 1);
                 uint32_t off0 = 0;
                 if (u.win_full_width) {
@@ -1009,7 +1016,8 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 }
                 umma_commit(smem_u32(&sh->empty[stage]));
                 umma_commit(smem_u32(&sh->tmem_full[buf]));
-                if (++stage == u.stages) { stage = 0; parity ^= 1u; }
+                stage += 2;
+                if (stage >= u.stages) { stage -= u.stages; parity ^= 1u; }
             }
         }
         __syncwarp();
@@ -1083,7 +1091,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const long long t0 = clock64();
             while (clock64() - t0 < 2000000) {}
         }
-        if (warp == MMA_WARP && lane == 0) {
+        if ((warp == MMA_WARP || warp == MMA_WARP2) && lane == 0) {
             umma_commit(smem_u32(&sh->drain));
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }
