@@ -205,7 +205,9 @@ extern "C" int iconv_plan_destroy(iconv_plan_t *p)
     return ICONV_OK;
 }
 
-extern "C" int iconv_plan(const iconv_desc *desc, iconv_plan_t **plan_out)
+extern "C" int iconv_plan(const iconv_desc *desc, iconv_plan_t **plan_out) { return iconv::plan_create(desc, 0, plan_out); }
+
+int iconv::plan_create(const iconv_desc *desc, int pair16, iconv_plan_t **plan_out)
 {
     if (!desc || !plan_out) {
         set_error("iconv_plan: null argument");
@@ -224,6 +226,7 @@ extern "C" int iconv_plan(const iconv_desc *desc, iconv_plan_t **plan_out)
     p->d = *desc;
     p->h_out = h_out;
     p->w_out = w_out;
+    p->pair16 = pair16;
     const iconv_desc &d = *desc;
     const size_t K = (size_t)d.kh * d.kw * d.c_in;
     const int np = d.per_channel ? d.c_out : 1;
@@ -266,7 +269,7 @@ extern "C" int iconv_plan_describe(const iconv_plan_t *p, char *text, size_t siz
     static const char *fam[] = {"auto", "direct", "umma", "thin", "stem", "umma"};
     if (p->kernel == ICONV_KERNEL_UMMA)
         snprintf(text, size, "umma %s block_n=%d kc=%d stages=%d kg=%d resident_b=%d epi_warps=%d cs=%d bi=%d nbuf=%d epi=%d proj_iters=%d",
-                 p->window ? (p->win_full_width ? "window(rows)" : "window(strips)") : "im2col", p->block_n, p->kc,
+                 p->window ? (p->win_blocks ? "window(blocks)" : p->win_full_width ? "window(rows)" : "window(strips)") : "im2col", p->block_n, p->kc,
                  p->window ? p->win_stages : p->stages, p->kg, p->window ? 1 : p->resident_b, p->epi_warps, p->cs, p->bi, p->nbuf, p->epi,
                  p->proj_iters);
     else if (p->kernel == ICONV_KERNEL_STEM && p->inner)

@@ -95,10 +95,14 @@ int stem_setup(iconv_plan_t *p)
     in.in_dtype = d.in_dtype == ICONV_U8 ? ICONV_U8 : ICONV_S8;
     in.kernel = ICONV_KERNEL_UMMA;
     in.weights = w2.data();
-    int rc = iconv_plan(&in, &p->inner);
+    // two horizontally adjacent taps per K step where the driver accepts the overlapping view
+    // of T (half the MMAs); T gets 16 bytes of slack for the last position's neighbour
+    int rc = plan_create(&in, 1, &p->inner);
+    if (rc != ICONV_OK) rc = iconv_plan(&in, &p->inner);
     if (rc != ICONV_OK) return rc;
-    p->workspace_bytes = (size_t)d.n * hp * wp * 16;
-    if (p->workspace_bytes) ICONV_CUDA_TRY(cudaMalloc(&p->workspace, p->workspace_bytes));
+    p->workspace_bytes = (size_t)d.n * hp * wp * 16 + 16;
+    ICONV_CUDA_TRY(cudaMalloc(&p->workspace, p->workspace_bytes));
+    ICONV_CUDA_TRY(cudaMemset((uint8_t *)p->workspace + p->workspace_bytes - 16, 0, 16));
     return ICONV_OK;
 }
 

@@ -91,6 +91,9 @@ struct UmmaArgs {
     int *status;
     // window mode (stride-1 filters: one patch load per tile, every tap a shifted view of it)
     int win_vw, win_bw, win_bh, win_full_width, win_tpi;    // virtual row width, patch width / height, mode, tiles per image
+    int win_tap_step;               // patch positions between two horizontal taps (2 with paired taps)
+    int win_blocks;                 // 1: tiles are blocks of 8 x 16 output pixels (win_vw = blocks per image row)
+    unsigned desc_hi_a;             // upper descriptor word of the A operand in block mode (8-row groups one patch line apart)
     unsigned div_tpi_mul, div_tpi_shr, div_vw_mul, div_vw_shr;
     // exact division of a tile index by n_tiles and of a pixel index by w_out and by
     // h_out * w_out without a divide instruction: q = umulhi(x, mul) >> shr  (x < 2^31)
@@ -259,6 +262,28 @@ __device__ __forceinline__ void umma_i8_split(uint32_t d_tmem, uint32_t a_lo, ui
         "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// The same with separate upper descriptor words for A and B (block-mode patches space A's 8-row
+// groups one patch line apart).
+__device__ __forceinline__ void umma_i8_split2(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+template <int KJ>
+__device__ __forceinline__ void umma_slot2(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                           uint32_t accumulate_first)
+{
+    umma_i8_split2(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
+#pragma unroll
+    for (int j = 1; j < KJ; ++j) umma_i8_split2(d_tmem, a_lo + 2u * j, a_hi, b_lo + 2u * j, b_hi, idesc, 1u);
 }
 // KJ instructions over the KJ 32-byte K slices of one slot (+2 in 16-byte units per slice).
 template <int KJ>
@@ -933,9 +958,17 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const uint32_t tx = (uint32_t)(u.kc * u.win_bw * u.win_bh);
             for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
                 const int img = (int)fast_div((unsigned)tile, u.div_tpi_mul, u.div_tpi_shr);
-                const unsigned i0 = (unsigned)(tile - img * u.win_tpi) * BLOCK_M;
-                const int y0 = (int)fast_div(i0, u.div_vw_mul, u.div_vw_shr);
-                const int c0 = (int)i0 - y0 * u.win_vw;
+                const unsigned rem = (unsigned)(tile - img * u.win_tpi);
+                int cx, cy;                                   // first output pixel of the tile
+                if (u.win_blocks) {
+                    const int by = (int)fast_div(rem, u.div_vw_mul, u.div_vw_shr);
+                    cx = ((int)rem - by * u.win_vw) * 8;
+                    cy = by * 16;
+                } else {
+                    const unsigned i0 = rem * BLOCK_M;
+                    cy = (int)fast_div(i0, u.div_vw_mul, u.div_vw_shr);
+                    cx = u.win_full_width ? 0 : (int)i0 - cy * u.win_vw;
+                }
                 if (!mbar_wait(smem_u32(&sh->empty[stage]), parity ^ 1u, &sh->abort_flag)) {
                     give_up(sh, u.status, 1);
                     break;
@@ -943,7 +976,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 const uint32_t full = smem_u32(&sh->full[stage]);
                 mbar_expect_tx(full, tx);
                 tma_load_tile_4d(smem_u32(tiles + (size_t)stage * u.stage_bytes), &tmap_x, full, 0,
-                                 (u.win_full_width ? 0 : c0) - a.pad, y0 - a.pad, img);
+                                 cx - a.pad, cy - a.pad, img);
                 last_stage = stage;
                 last_parity = parity;
                 if (++stage == u.stages) { stage = 0; parity ^= 1u; }
@@ -965,11 +998,13 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             if (!ok) give_up(sh, u.status, 6);
             const int kj = u.kc >> 5;
             const uint32_t desc_hi32 = (uint32_t)(u.desc_hi >> 32);
+            const uint32_t a_hi32 = u.win_blocks ? u.desc_hi_a : desc_hi32;
             const uint32_t a_lo0 = ((smem_u32(tiles) & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t b_lo0 = ((smem_u32(b_res) & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, row_step = (uint32_t)u.kc >> 4;
             const uint32_t b_step = (uint32_t)u.b_tile_bytes >> 4;
             const uint32_t line_step = (uint32_t)u.win_bw * row_step;
+            const uint32_t tap_step = (uint32_t)u.win_tap_step * row_step;
             for (int tile = blockIdx.x + which * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x, t += 2) {
                 const int buf = t & (u.nbuf - 1);
                 uint32_t off0 = 0;
@@ -995,7 +1030,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     for (int r = 0; r < (KH ? KH : 1); ++r) {
 #pragma unroll
                         for (int sx = 0; sx < (KW ? KW : 1); ++sx)
-                            umma_slot<KJ ? KJ : 1>(d_tmem, a_line + (uint32_t)sx * row_step, b_lo + (uint32_t)(r * KW + sx) * b_step, desc_hi32,
+                            umma_slot2<KJ ? KJ : 1>(d_tmem, a_line + (uint32_t)sx * tap_step, a_hi32, b_lo + (uint32_t)(r * KW + sx) * b_step, desc_hi32,
                                                    u.idesc, (uint32_t)((r | sx) != 0));
                         a_line += line_step;
                     }
@@ -1004,9 +1039,9 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     for (int r = 0; r < a.kh; ++r) {
                         uint32_t a_lo = a_line;
                         for (int sx = 0; sx < a.kw; ++sx) {
-                            if (kj == 4) umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                            else if (kj == 2) umma_slot<2>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
-                            else umma_slot<1>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, acc);
+                            if (kj == 4) umma_slot2<4>(d_tmem, a_lo, a_hi32, b_lo, desc_hi32, u.idesc, acc);
+                            else if (kj == 2) umma_slot2<2>(d_tmem, a_lo, a_hi32, b_lo, desc_hi32, u.idesc, acc);
+                            else umma_slot2<1>(d_tmem, a_lo, a_hi32, b_lo, desc_hi32, u.idesc, acc);
                             acc = 1;
                             a_lo += row_step;
                             b_lo += b_step;
@@ -1035,9 +1070,18 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles; t += u.bi, tile += tile_step) {
             const int buf = t & (u.nbuf - 1);
             const int img = (int)fast_div((unsigned)tile, u.div_tpi_mul, u.div_tpi_shr);
-            const unsigned i = (unsigned)(tile - img * u.win_tpi) * BLOCK_M + (unsigned)(quad * 32 + lane);   // this lane's virtual pixel
-            const int y = (int)fast_div(i, u.div_vw_mul, u.div_vw_shr);
-            const int xq = (int)i - y * u.win_vw;
+            const unsigned rem = (unsigned)(tile - img * u.win_tpi);
+            int y, xq;                                        // this lane's (virtual) output pixel
+            if (u.win_blocks) {
+                const int by = (int)fast_div(rem, u.div_vw_mul, u.div_vw_shr);
+                const int mm = quad * 32 + lane;
+                y = by * 16 + (mm >> 3);
+                xq = ((int)rem - by * u.win_vw) * 8 + (mm & 7);
+            } else {
+                const unsigned i = rem * BLOCK_M + (unsigned)(quad * 32 + lane);
+                y = (int)fast_div(i, u.div_vw_mul, u.div_vw_shr);
+                xq = (int)i - y * u.win_vw;
+            }
             const bool valid = xq < a.w_out && y < a.h_out;
             uint8_t *orow = (uint8_t *)a.out + (((long long)img * a.h_out + y) * a.w_out + xq) * a.out_c_total + a.out_c_offset;
             if (!mbar_wait_warp(smem_u32(&sh->tmem_full[buf]), (uint32_t)((t >> u.lg_nbuf) & 1), &sh->abort_flag, lane)) {
@@ -1181,7 +1225,9 @@ int encode_activation_map(const iconv_plan_t *p, const void *x, CUtensorMap *map
 int encode_patch_map(const iconv_plan_t *p, const void *x, CUtensorMap *map)
 {
     const iconv_desc &d = p->d;
-    const cuuint64_t dims[4] = {(cuuint64_t)d.c_in, (cuuint64_t)d.w, (cuuint64_t)d.h, (cuuint64_t)d.n};
+    // (paired taps: every position is read together with its right-hand neighbour, as 32
+    // channels at a 16-byte pitch; the caller keeps 16 readable bytes behind the tensor)
+    const cuuint64_t dims[4] = {(cuuint64_t)(p->pair16 ? 32 : d.c_in), (cuuint64_t)d.w, (cuuint64_t)d.h, (cuuint64_t)d.n};
     const cuuint64_t strides[3] = {(cuuint64_t)d.in_c_total, (cuuint64_t)d.in_c_total * d.w, (cuuint64_t)d.in_c_total * d.w * d.h};
     const cuuint32_t box[4] = {(cuuint32_t)p->kc, (cuuint32_t)p->win_bw, (cuuint32_t)p->win_bh, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -1373,6 +1419,7 @@ int umma_init_once()
     ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
     ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 5, 5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
     ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 4, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
+    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 4, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
     ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM))
         ICONV_WIN_ATTR(EPI_FAST);
         ICONV_WIN_ATTR(EPI_SAFE);
@@ -1381,6 +1428,10 @@ int umma_init_once()
     }
     return ICONV_OK;
 }
+
+// Reduction steps along the filter: kh * kw taps, or half of that when two horizontally
+// adjacent 16-channel taps share one 32-byte K step (paired taps).
+int plan_taps(const iconv_plan_t *p) { return p->pair16 ? p->d.kh * (p->d.kw / 2) : p->d.kh * p->d.kw; }
 
 // Tile, pipeline and epilogue geometry of a layer, from its descriptor alone (host only).
 int umma_geometry(iconv_plan_t *p)
@@ -1403,7 +1454,7 @@ int umma_geometry(iconv_plan_t *p)
     const int n_tiles = (d.c_out + n_max - 1) / n_max;
     p->block_n = ((d.c_out + n_tiles - 1) / n_tiles + 15) / 16 * 16;
     p->c_out_pad = p->block_n * n_tiles;
-    const int taps = d.kh * d.kw;
+    const int taps = plan_taps(p);
     p->proj_iters = proj ? d.proj_k * d.proj_k * (p->proj_c_in_pad / p->kc) : 0;
     const int k_iters = p->proj_iters + taps * (p->c_in_pad / p->kc);
     const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
@@ -1482,29 +1533,55 @@ void window_plan(iconv_plan_t *p)
     const iconv_desc &d = p->d;
     p->window = 0;
     if (d.kernel == ICONV_KERNEL_UMMA_IM2COL) return;
-    if (d.stride != 1 || d.kh * d.kw < 2 || d.proj_weights || d.skip_dtype >= 0 || d.out_dtype == ICONV_I32) return;
+    if (d.stride != 1 || d.proj_weights || d.skip_dtype >= 0 || d.out_dtype == ICONV_I32) return;
     if (p->c_in_pad != p->kc || p->c_out_pad != p->block_n) return;
     if (p->epi != EPI_FAST && p->epi != EPI_SAFE) return;
-    const int taps = d.kh * d.kw;
+    const int taps = plan_taps(p);
     const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
     const long long bank = (long long)b_tile * taps;
     const int wp = p->w_out + d.kw - 1;
-    int vw, bw, bh, full_width;
-    if (p->w_out >= 128) {                      // strips of 128 pixels inside one row
-        vw = (p->w_out + 127) / 128 * 128; bw = 128 + d.kw - 1; bh = d.kh; full_width = 0;
-    } else {                                    // the padded width, tiles run across rows
-        vw = wp; bw = wp; bh = (wp - 1 + 127) / wp + d.kh; full_width = 1;
-    }
-    if (bw > 256 || bh > 256) return;
-    const long long patch = ((long long)(bh * bw + d.kw) * p->kc + 1023) / 1024 * 1024;
-    if (patch > 64 * 1024) return;
     const long long room = MAX_SMEM - 1024 - (long long)sizeof(Shared) - bank;
-    if (room < 2 * patch) return;
-    const long long tpi = ((long long)p->h_out * vw + BLOCK_M - 1) / BLOCK_M;
-    if ((long long)p->h_out * p->w_out * 10 < tpi * BLOCK_M * 6) return;          // under 60 % real pixels
-    if (tpi * d.n >= (1ll << 31) / BLOCK_M) return;
+    // Three tilings of an image into 128 output pixels per tile; the cheapest by a simple
+    // model wins (per tile the patch comes in at about 20 bytes per clock, an MMA takes 64 or
+    // 128 clocks, and the two overlap only in part):
+    //   rows    the padded width, tiles run on across rows        (narrow images)
+    //   strips  128 pixels of one row                              (wide images)
+    //   blocks  8 x 16 pixels: the smallest halo, 8-row operand groups one patch line apart
+    const int n_mma = taps * (p->kc / 32);
+    const double mma_clk = (double)n_mma * (p->block_n > 128 ? 128 : 64);
+    double best = -1;
+    int vw = 0, bw = 0, bh = 0, full_width = 0, blocks = 0;
+    long long tpi = 0, patch = 0;
+    for (int mode = 0; mode < 3; ++mode) {
+        int m_vw, m_bw, m_bh;
+        long long m_tpi;
+        if (mode == 0) {
+            if (p->w_out >= 128) continue;
+            m_vw = wp; m_bw = wp; m_bh = (wp - 1 + 127) / wp + d.kh;
+            m_tpi = ((long long)p->h_out * m_vw + BLOCK_M - 1) / BLOCK_M;
+        } else if (mode == 1) {
+            if (p->w_out < 128) continue;
+            m_vw = (p->w_out + 127) / 128 * 128; m_bw = 128 + d.kw - 1; m_bh = d.kh;
+            m_tpi = ((long long)p->h_out * m_vw + BLOCK_M - 1) / BLOCK_M;
+        } else {
+            m_vw = (p->w_out + 7) / 8; m_bw = 8 + d.kw - 1; m_bh = 16 + d.kh - 1;
+            m_tpi = (long long)m_vw * ((p->h_out + 15) / 16);
+            if ((long long)m_bw * p->kc >= (1 << 18)) continue;     // the group stride field holds 14 bits of 16-byte units
+        }
+        if (m_bw > 256 || m_bh > 256) continue;
+        const long long m_patch = ((long long)(m_bh * m_bw + d.kw) * p->kc + 1023) / 1024 * 1024;
+        if (m_patch > 64 * 1024 || room < 2 * m_patch) continue;
+        if ((long long)p->h_out * p->w_out * 10 < m_tpi * BLOCK_M * 6) continue;      // under 60 % real pixels
+        if (m_tpi * d.n >= (1ll << 31) / BLOCK_M) continue;
+        const double tma_clk = (double)m_patch / 20.0;
+        const double cost = (double)m_tpi * ((mma_clk > tma_clk ? mma_clk : tma_clk) + 0.25 * (mma_clk > tma_clk ? tma_clk : mma_clk));
+        if (best < 0 || cost < best) {
+            best = cost; vw = m_vw; bw = m_bw; bh = m_bh; full_width = mode == 0; blocks = mode == 2; tpi = m_tpi; patch = m_patch;
+        }
+    }
+    if (best < 0) return;
     p->window = 1;
-    p->win_vw = vw; p->win_bw = bw; p->win_bh = bh; p->win_full_width = full_width; p->win_tpi = (int)tpi;
+    p->win_vw = vw; p->win_bw = bw; p->win_bh = bh; p->win_full_width = full_width; p->win_blocks = blocks; p->win_tpi = (int)tpi;
     p->win_patch_bytes = (int)patch;
     p->win_stages = (int)(room / patch < 6 ? room / patch : 6);
     // sixteen epilogue warps: no staging memory is needed here
@@ -1520,8 +1597,7 @@ void window_plan(iconv_plan_t *p)
 // 2-D tiled map over the packed weights p->w_packed, [c_out_pad][taps * c_in_pad].
 int umma_encode_weight_map(iconv_plan_t *p)
 {
-    const iconv_desc &d = p->d;
-    const size_t k_pad = (size_t)d.kh * d.kw * p->c_in_pad + (size_t)p->proj_iters * p->kc;
+    const size_t k_pad = (size_t)plan_taps(p) * p->c_in_pad + (size_t)p->proj_iters * p->kc;
     const cuuint64_t dims[2] = {(cuuint64_t)k_pad, (cuuint64_t)p->c_out_pad};
     const cuuint64_t strides[1] = {(cuuint64_t)k_pad};
     const cuuint32_t box[2] = {(cuuint32_t)p->kc, (cuuint32_t)p->block_n};
@@ -1546,7 +1622,7 @@ int umma_setup(iconv_plan_t *p)
 
     // repack weights [c_out][tap][c_in] -> [c_out_pad][tap][c_in_pad], zero filled; a fused
     // projection's weights come first in every row
-    const int taps = d.kh * d.kw, ptaps = d.proj_weights ? d.proj_k * d.proj_k : 0;
+    const int taps = plan_taps(p), ptaps = d.proj_weights ? d.proj_k * d.proj_k : 0;
     const size_t kp_pad = (size_t)ptaps * p->proj_c_in_pad;
     const size_t k_pad = kp_pad + (size_t)taps * p->c_in_pad;
     std::vector<int8_t> packed((size_t)p->c_out_pad * k_pad, 0);
@@ -1554,6 +1630,10 @@ int umma_setup(iconv_plan_t *p)
         for (int t = 0; t < ptaps; ++t)
             memcpy(&packed[(size_t)co * k_pad + (size_t)t * p->proj_c_in_pad], d.proj_weights + ((size_t)co * ptaps + t) * d.proj_c_in,
                    (size_t)d.proj_c_in);
+        if (p->pair16) {    // [R][S][16] read as [R][S / 2][32]: the row as it stands
+            memcpy(&packed[(size_t)co * k_pad], d.weights + (size_t)co * k_pad, k_pad);
+            continue;
+        }
         for (int t = 0; t < taps; ++t)
             memcpy(&packed[(size_t)co * k_pad + kp_pad + (size_t)t * p->c_in_pad], d.weights + ((size_t)co * taps + t) * d.c_in, (size_t)d.c_in);
     }
@@ -1602,6 +1682,10 @@ int umma_setup(iconv_plan_t *p)
         CUtensorMap probe2;     // the tiled patch map must be encodable as well
         if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
     }
+    if (p->pair16 && !p->window) {
+        set_error("tensor-core path: paired taps need window mode");
+        return ICONV_ERR_UNSUPPORTED;
+    }
     return ICONV_OK;
 }
 
@@ -1618,6 +1702,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
 
     UmmaArgs u;
     u.win_vw = p->win_vw; u.win_bw = p->win_bw; u.win_bh = p->win_bh; u.win_full_width = p->win_full_width; u.win_tpi = p->win_tpi;
+    u.win_blocks = p->win_blocks;
     find_divisor((unsigned)(p->win_tpi > 0 ? p->win_tpi : 1), u.div_tpi_mul, u.div_tpi_shr);
     find_divisor((unsigned)(p->win_vw > 0 ? p->win_vw : 1), u.div_vw_mul, u.div_vw_shr);
     u.m_total = (long long)d.n * p->h_out * p->w_out;
@@ -1626,7 +1711,8 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.block_n = p->block_n;
     u.kc = p->kc;
     u.cchunks = p->c_in_pad / p->kc;
-    u.taps = d.kh * d.kw;
+    u.taps = plan_taps(p);
+    u.win_tap_step = p->pair16 ? 2 : 1;
     u.p_iters = p->proj_iters;
     u.p_taps = p->proj_iters ? d.proj_k * d.proj_k : 0;
     u.p_cchunks = p->proj_iters ? p->proj_c_in_pad / p->kc : 0;
@@ -1661,6 +1747,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     // units), descriptor version 1, swizzle mode (128B = 2, 64B = 4, 32B = 6)
     const unsigned long long layout = p->kc == 128 ? 2ull : (p->kc == 64 ? 4ull : 6ull);
     u.desc_hi = ((unsigned long long)((8 * p->kc) >> 4) << 32) | (1ull << 46) | (layout << 61);
+    u.desc_hi_a = (unsigned)((((unsigned long long)((p->win_bw * p->kc) >> 4) << 32) | (1ull << 46) | (layout << 61)) >> 32);
     u.q_mul = p->q_mul;
     u.q_shift = p->q_shift;
     u.q_half = p->q_shift > 0 && p->q_shift <= 31 ? (int)(1u << (p->q_shift - 1)) : 0;
@@ -1713,6 +1800,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         if (d.kh == 3 && d.kw == 3 && kj == 2) umma_window_kernel<E, 3, 3, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);      \
         else if (d.kh == 3 && d.kw == 3 && kj == 4) umma_window_kernel<E, 3, 3, 4><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
         else if (d.kh == 5 && d.kw == 5 && kj == 2) umma_window_kernel<E, 5, 5, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
+        else if (d.kh == 4 && d.kw == 4 && kj == 1 && p->pair16) umma_window_kernel<E, 4, 2, 1><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
         else if (d.kh == 4 && d.kw == 4 && kj == 1) umma_window_kernel<E, 4, 4, 1><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
         else umma_window_kernel<E, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);                        \
     } while (0)

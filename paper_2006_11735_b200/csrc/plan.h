@@ -23,7 +23,7 @@ struct iconv_plan_s {
     int half_n = 0, piece_bytes = 0;   // columns per epilogue warp and staged piece width
     int proj_c_in_pad = 0, proj_iters = 0, proj32 = 0;   // fused projection: padded channels, k-iterations, 32-bit rescale proven
     // window mode of the tensor-core kernel (stride-1 filters: one patch load per tile)
-    int window = 0, win_vw = 0, win_bw = 0, win_bh = 0, win_full_width = 0, win_tpi = 0, win_patch_bytes = 0, win_stages = 0;
+    int window = 0, win_vw = 0, win_bw = 0, win_bh = 0, win_full_width = 0, win_blocks = 0, win_tpi = 0, win_patch_bytes = 0, win_stages = 0;
     int thin_narrow = 0;     // thin kernels: BReLU + Eq. 4 provably fit 32 bits
     int kg = 1;              // k-iterations grouped behind one pair of pipeline barriers
     int nbuf = 2;            // TMEM accumulator buffers
@@ -31,6 +31,7 @@ struct iconv_plan_s {
     int epi_warps = 8, cs = 1, bi = 1;   // epilogue warps; column split per tile; tiles in flight
     int tail = 1;            // 0: zero point and output range are provably no-ops
     int q_mul = 1, q_shift = 0, q_h = 0; // per-layer Eq. 4 / BReLU scalars
+    int pair16 = 0;                      // internal (stem): 16-channel positions read in pairs, two taps per K step
     // stem path: repacked image (plan-owned scratch) and the plan of the GEMM that follows
     iconv_plan_s *inner = nullptr;
     void *workspace = nullptr;
@@ -40,6 +41,9 @@ struct iconv_plan_s {
 namespace iconv {
 
 int choose_kernel(iconv_plan_t *p);      // fills p->kernel and the kernel-specific fields
+// iconv_plan with the internal options: pair16 plans a 16-channel layer with paired taps (the
+// input must be followed by 16 readable bytes; the tensor-core window path or failure)
+int plan_create(const iconv_desc *desc, int pair16, iconv_plan_t **plan_out);
 
 int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);

@@ -198,7 +198,18 @@ WINDOW_SHAPES = [
     (2, 20, 17, 32, 64, 3, 1, 0),       # no padding: the output is narrower than the input
     (1, 40, 33, 16, 256, 3, 1, 1),      # two column halves per tile
     (2, 12, 50, 64, 48, 5, 1, 4),       # padding wider than the filter needs
+    (1, 37, 150, 64, 64, 3, 1, 1),      # 8 x 16 pixel blocks, ragged on the right and at the bottom
+    (2, 35, 133, 64, 16, 5, 1, 2),      # blocks under a 5x5 filter
+    (1, 6, 260, 48, 32, 1, 1, 0),       # a 1x1 layer as strips of one row
+    (2, 24, 24, 64, 64, 1, 1, 0),       # a 1x1 layer as blocks
 ]
+
+# the tiling (of the three window mode has) that the plan's cost model picks for these shapes
+WINDOW_TILINGS = {
+    (1, 37, 150, 64, 64, 3, 1, 1): "window(blocks)",
+    (3, 28, 28, 128, 128, 3, 1, 1): "window(rows)",
+    (1, 6, 260, 48, 32, 1, 1, 0): "window(strips)",
+}
 
 
 @pytest.mark.parametrize("shape", UMMA_SHAPES + WINDOW_SHAPES, ids=lambda s: "x".join(map(str, s)))
@@ -218,6 +229,8 @@ def test_tensor_core_kernel_matches_oracle(shape, kernel):
             assert "im2col" in text[0], text[0]
         elif shape in WINDOW_SHAPES:
             assert "window" in text[0], text[0]
+            if shape in WINDOW_TILINGS:      # so that every tiling is known to be covered
+                assert WINDOW_TILINGS[shape] in text[0], text[0]
         want = oracle_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad)
         assert 0.05 < (want == 0).mean() < 0.95
     assert fam == B.KERNEL_UMMA
