@@ -11,6 +11,13 @@
 //      out(oh, ow) = sum_{R,S} T[oh+R][ow+S] . W'[R][S],  W'[R][S][(dy*2+dx)*3+c] = W[2R+dy-1][2S+dx-1][c].
 //
 // The sum is the same integers in another order, so the result is bit-identical.
+//
+// A single-channel image under a stride-1 kh x kw filter (the first layer of the regression
+// networks) takes the same two steps with another repack: T[n][Y][x][j] = in[n][Y-pad][x-pad+j],
+// j < kw (the kw input bytes an output column needs, side by side as "channels"), after which
+// the layer is a kh x 1 filter over 16 channels: out(oh, ow) = sum_r T[oh+r][ow] . W'[r],
+// W'[r][j] = W[r][j].  Sixteen bytes per position instead of one, but the arithmetic moves
+// to the tensor cores and the CUDA cores keep only the epilogue.
 #include <cstring>
 #include <vector>
 
@@ -53,21 +60,101 @@ stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int 
     }
 }
 
+// One thread writes the 16 bytes of one position (n, Y, x) of T for a single-channel image:
+// bytes 0 .. kw-1 are in[n][Y - pad][x - pad + j] (0 outside the image), the rest 0.
+__global__ void __launch_bounds__(256)
+rows_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int n, int h, int w, int hp, int wo, int pad, int kw,
+                   int raw128)
+{
+    const long long total = (long long)n * hp * wo;
+    for (long long pos = (long long)blockIdx.x * blockDim.x + threadIdx.x; pos < total;
+         pos += (long long)gridDim.x * blockDim.x) {
+        const int x = (int)(pos % wo);
+        const int Y = (int)((pos / wo) % hp);
+        const int img = (int)(pos / ((long long)wo * hp));
+        const int ih = Y - pad;
+        unsigned wds[4] = {0, 0, 0, 0};
+        if (ih >= 0 && ih < h) {
+            const uint8_t *row = in + ((long long)img * h + ih) * w;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int iw = x - pad + j;
+                if (j < kw && iw >= 0 && iw < w) {
+                    unsigned v = row[iw];
+                    if (raw128) v ^= 0x80u;                              // raw - 128 as int8
+                    wds[j >> 2] |= v << (8 * (j & 3));
+                }
+            }
+        }
+        *(uint4 *)(T + pos * 16) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    }
+}
+
+// 1: the 7x7 stride-2 stem over 3 channels; 2: a stride-1 filter over a single-channel image
+int stem_kind(const iconv_desc &d)
+{
+    if (d.c_in == 3 && d.in_c_total == 3 && d.in_c_offset == 0 && d.kh == 7 && d.kw == 7 && d.stride == 2 &&
+        d.pad == 3 && d.c_out >= 16)
+        return 1;
+    if (d.c_in == 1 && d.in_c_total == 1 && d.in_c_offset == 0 && d.stride == 1 && d.kw <= 16 && d.kh * d.kw > 1 &&
+        d.c_out >= 32 && d.skip_dtype < 0)
+        return 2;
+    return 0;
+}
+
 }  // namespace
 
 int stem_supported(const iconv_plan_t *p)
 {
-    const iconv_desc &d = p->d;
-    if (d.c_in == 3 && d.in_c_total == 3 && d.in_c_offset == 0 && d.kh == 7 && d.kw == 7 && d.stride == 2 &&
-        d.pad == 3 && d.c_out >= 16)
-        return ICONV_OK;
-    set_error("stem path: needs a 7x7 stride-2 pad-3 layer over a 3-channel tensor");
+    if (stem_kind(p->d)) return ICONV_OK;
+    set_error("stem path: needs a 7x7 stride-2 pad-3 layer over a 3-channel tensor, or a stride-1 filter at most 16 wide "
+              "over a single-channel tensor with at least 32 output channels and no skip");
     return ICONV_ERR_UNSUPPORTED;
 }
+
+namespace {
+
+int rows_setup(iconv_plan_t *p)
+{
+    const iconv_desc &d = p->d;
+    const int hp = d.h + 2 * d.pad, wo = p->w_out;
+    std::vector<int8_t> w2((size_t)d.c_out * d.kh * 16, 0);
+    for (int co = 0; co < d.c_out; ++co)
+        for (int r = 0; r < d.kh; ++r)
+            for (int s = 0; s < d.kw; ++s)
+                w2[((size_t)co * d.kh + r) * 16 + s] = d.weights[((size_t)co * d.kh + r) * d.kw + s];
+    iconv_desc in = d;
+    in.h = hp;
+    in.w = wo;
+    in.c_in = 16;
+    in.in_c_total = 16;
+    in.in_c_offset = 0;
+    in.kw = 1;
+    in.stride = 1;
+    in.pad = 0;
+    in.in_dtype = d.in_dtype == ICONV_U8 ? ICONV_U8 : ICONV_S8;
+    in.kernel = ICONV_KERNEL_UMMA;
+    in.weights = w2.data();
+    int rc = iconv_plan(&in, &p->inner);
+    if (rc != ICONV_OK) return rc;
+    if (!p->inner->window) {
+        // only worth the repack when the layer then runs from one patch per tile
+        iconv_plan_destroy(p->inner);
+        p->inner = nullptr;
+        set_error("stem path: the repacked single-channel layer does not fit the tensor-core window mode");
+        return ICONV_ERR_UNSUPPORTED;
+    }
+    p->workspace_bytes = (size_t)d.n * hp * wo * 16;
+    ICONV_CUDA_TRY(cudaMalloc(&p->workspace, p->workspace_bytes ? p->workspace_bytes : 16));
+    return ICONV_OK;
+}
+
+}  // namespace
 
 int stem_setup(iconv_plan_t *p)
 {
     const iconv_desc &d = p->d;
+    if (stem_kind(d) == 2) return rows_setup(p);
     const int hp = p->h_out + 3, wp = p->w_out + 3;
     // W'[co][R][S][(dy*2+dx)*3 + c] = W[co][2R+dy-1][2S+dx-1][c]  (0 where an index is -1)
     std::vector<int8_t> w2((size_t)d.c_out * 16 * 16, 0);
@@ -109,6 +196,17 @@ int stem_setup(iconv_plan_t *p)
 int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
 {
     const iconv_desc &d = p->d;
+    if (stem_kind(d) == 2) {
+        const int hp = d.h + 2 * d.pad, wo = p->w_out;
+        const long long total = (long long)d.n * hp * wo;
+        long long blocks = (total + 255) / 256;
+        if (blocks > 148ll * 32) blocks = 148ll * 32;
+        if (blocks > 0)
+            rows_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)p->workspace, d.n, d.h, d.w, hp, wo,
+                                                                     d.pad, d.kw, d.in_dtype == ICONV_U8_RAW128);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        return iconv_forward(p->inner, p->workspace, a.skip, a.out, (void *)stream);
+    }
     const int hp = p->h_out + 3, wp = p->w_out + 3;
     const long long total = (long long)d.n * hp * wp;
     long long blocks = (total + 255) / 256;

@@ -188,23 +188,32 @@ __global__ void __launch_bounds__(256) thin_out_kernel(const __grid_constant__ C
             const int ow = (int)rem - oh * a.w_out;
             const uint8_t *ximg = x + (size_t)img * a.h * a.w_ * a.in_c_total;
             if (K3) {
+                // nine loads with no branch between them (a tap outside the image reads the
+                // image's first pixel instead and is zeroed afterwards), so that all nine are
+                // in flight together
+                uint4 xv[9];
 #pragma unroll
                 for (int r = 0; r < 3; ++r) {
                     const int ih = oh * a.stride - a.pad + r;
-                    if (ih < 0 || ih >= a.h) continue;
 #pragma unroll
                     for (int s = 0; s < 3; ++s) {
                         const int iw = ow * a.stride - a.pad + s;
-                        if (iw < 0 || iw >= a.w_) continue;
-                        const uint4 xv = __ldg((const uint4 *)(ximg + (size_t)(ih * a.w_ + iw) * a.in_c_total));
-                        const int4 wv = wr[r * 3 + s];
-                        if (SIGNED) {
-                            U = dp4a_ss((int)xv.x, wv.x, U); U = dp4a_ss((int)xv.y, wv.y, U);
-                            U = dp4a_ss((int)xv.z, wv.z, U); U = dp4a_ss((int)xv.w, wv.w, U);
-                        } else {
-                            U = dp4a_us(xv.x, wv.x, U); U = dp4a_us(xv.y, wv.y, U);
-                            U = dp4a_us(xv.z, wv.z, U); U = dp4a_us(xv.w, wv.w, U);
-                        }
+                        const bool in = ih >= 0 && ih < a.h && iw >= 0 && iw < a.w_;
+                        const size_t off = in ? (size_t)(ih * a.w_ + iw) * a.in_c_total : 0;
+                        uint4 v = __ldg((const uint4 *)(ximg + off));
+                        if (!in) v = make_uint4(0, 0, 0, 0);
+                        xv[r * 3 + s] = v;
+                    }
+                }
+#pragma unroll
+                for (int tap = 0; tap < 9; ++tap) {
+                    const int4 wv = wr[tap];
+                    if (SIGNED) {
+                        U = dp4a_ss((int)xv[tap].x, wv.x, U); U = dp4a_ss((int)xv[tap].y, wv.y, U);
+                        U = dp4a_ss((int)xv[tap].z, wv.z, U); U = dp4a_ss((int)xv[tap].w, wv.w, U);
+                    } else {
+                        U = dp4a_us(xv[tap].x, wv.x, U); U = dp4a_us(xv[tap].y, wv.y, U);
+                        U = dp4a_us(xv[tap].z, wv.z, U); U = dp4a_us(xv[tap].w, wv.w, U);
                     }
                 }
             } else {

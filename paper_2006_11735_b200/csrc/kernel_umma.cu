@@ -61,7 +61,8 @@ enum {
     EPI_SAFE = 4,        // explicit BReLU clamp, 32-bit Eq. 4, optional zero point / range tail
     EPI_SAFE_SKIP8 = 5,  // ... with an 8-bit skip staged by TMA
     EPI_SAFE_SKIP32 = 6, // ... with an int32 skip (projection), rescaled in 64 bits
-    EPI_PROJ = 7         // ... with the projection convolution fused: a second accumulator tile beside the first
+    EPI_PROJ = 7,        // ... with the projection convolution fused: a second accumulator tile beside the first
+    EPI_NARROW = 8       // window mode only: fewer than 16 output channels (or unaligned ones), any descriptor; byte stores
 };
 
 struct UmmaArgs {
@@ -1093,7 +1094,31 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const int ngroups = ncols >> 4;
             int accA[16], accB[16];
             tmem_ld16(t_row, accA);
-            for (int gi = 0; gi < ngroups; gi += 2) {
+            if (EPI == EPI_NARROW) {
+                // a handful of channels per pixel (the regression networks' last layer): the general
+                // 64-bit epilogue channel by channel, the skip read and the output written byte-wise
+                const long long mpix = ((long long)img * a.h_out + y) * a.w_out + xq;
+                for (int g0 = 0; g0 < ngroups; ++g0) {
+                    if (g0) tmem_ld16(t_row + (uint32_t)(g0 << 4), accA);
+                    tmem_ld_wait();
+                    const int co0 = col_lo + (g0 << 4);
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const int co = co0 + k;
+                        if (valid && co < a.c_out) {
+                            const int pc = a.per_channel ? co : 0;
+                            long long Y = (long long)accA[k] + __ldg(u.c_a + co);
+                            if (a.skip_dtype >= 0)
+                                Y += round_shift64((long long)load_skip(a.skip, mpix * a.skip_c_total + a.skip_c_offset + co, a.skip_dtype) * a.skip_mul,
+                                                   a.skip_shift);
+                            const int v = requant_tail(Y, a.brelu, __ldg(u.c_h + pc), __ldg(u.c_mul + pc), __ldg(u.c_shift + pc), a.out_zero,
+                                                       a.out_lo, a.out_hi);
+                            orow[co] = (uint8_t)v;
+                        }
+                    }
+                }
+            }
+            for (int gi = 0; EPI != EPI_NARROW && gi < ngroups; gi += 2) {
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
                     const int gcur = gi + hf;
@@ -1371,17 +1396,29 @@ int encode_rows_map(const void *base, int elem_bytes, int c_slice, int c_total, 
 
 }  // namespace
 
+// A layer whose 8-bit output (or skip) is too narrow or too oddly placed for 16-byte stores:
+// window mode writes it byte by byte (EPI_NARROW) where its other conditions hold.
+bool umma_narrow(const iconv_desc &d)
+{
+    if (d.out_dtype == ICONV_I32) return false;
+    const bool odd_out = d.c_out % 16 || d.out_c_total % 16 || d.out_c_offset % 16;
+    const bool odd_skip = d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && (d.skip_c_total % 16 || d.skip_c_offset % 16);
+    return (odd_out || odd_skip) && d.stride == 1 && d.c_in <= 128 && d.c_out <= 64 && !d.proj_weights &&
+           d.kernel != ICONV_KERNEL_UMMA_IM2COL;
+}
+
 int umma_supported(const iconv_plan_t *p)
 {
     const iconv_desc &d = p->d;
     const char *why = nullptr;
+    const bool narrow = umma_narrow(d);
     if (d.in_dtype == ICONV_U8_RAW128) why = "raw-128 inputs are not GEMM operands";
     else if (d.c_in % 16 || d.in_c_total % 16 || d.in_c_offset % 16) why = "input channels must be multiples of 16";
-    else if (d.c_out < 16) why = "c_out below 16";
+    else if (d.c_out < 16 && !narrow) why = "c_out below 16";
     else if (d.out_dtype == ICONV_I32 && (d.c_out % 4 || d.out_c_total % 4 || d.out_c_offset % 4)) why = "int32 output channels must be multiples of 4";
-    else if (d.out_dtype != ICONV_I32 && (d.c_out % 16 || d.out_c_total % 16 || d.out_c_offset % 16)) why = "8-bit output channels must be multiples of 16";
+    else if (!narrow && d.out_dtype != ICONV_I32 && (d.c_out % 16 || d.out_c_total % 16 || d.out_c_offset % 16)) why = "8-bit output channels must be multiples of 16";
     else if (d.skip_dtype == ICONV_I32 && (d.skip_c_total % 4 || d.skip_c_offset % 4)) why = "int32 skip channels must be multiples of 4";
-    else if (d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && (d.skip_c_total % 16 || d.skip_c_offset % 16)) why = "8-bit skip channels must be multiples of 16";
+    else if (!narrow && d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && (d.skip_c_total % 16 || d.skip_c_offset % 16)) why = "8-bit skip channels must be multiples of 16";
     else if (d.kh > 16 || d.kw > 16 || d.pad > 16 || d.stride > 8) why = "filter, padding or stride beyond the im2col descriptor's range";
     else if ((long long)d.kh * d.kw * ((d.c_in + 127) / 128 * 128) >= (1ll << 24)) why = "reduction too long";
     else if ((long long)d.n * p->h_out * p->w_out >= (1ll << 31) - 256) why = "more than 2^31 output pixels";
@@ -1410,6 +1447,8 @@ int umma_init_once()
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         attr_set = true;
     }
     static bool win_attr_set = false;
@@ -1533,9 +1572,9 @@ void window_plan(iconv_plan_t *p)
     const iconv_desc &d = p->d;
     p->window = 0;
     if (d.kernel == ICONV_KERNEL_UMMA_IM2COL) return;
-    if (d.stride != 1 || d.proj_weights || d.skip_dtype >= 0 || d.out_dtype == ICONV_I32) return;
+    if (d.stride != 1 || d.proj_weights || (d.skip_dtype >= 0 && p->epi != EPI_NARROW) || d.out_dtype == ICONV_I32) return;
     if (p->c_in_pad != p->kc || p->c_out_pad != p->block_n) return;
-    if (p->epi != EPI_FAST && p->epi != EPI_SAFE) return;
+    if (p->epi != EPI_FAST && p->epi != EPI_SAFE && p->epi != EPI_NARROW) return;
     const int taps = plan_taps(p);
     const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
     const long long bank = (long long)b_tile * taps;
@@ -1661,6 +1700,11 @@ int umma_setup(iconv_plan_t *p)
     } else {
         p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail);
         c_b.assign((size_t)p->c_out_pad, 0);
+        if (umma_narrow(d)) {
+            p->epi = EPI_NARROW;
+            p->tail = 1;
+            for (int co = 0; co < d.c_out; ++co) c_a[co] = d.bias[co];
+        }
     }
     std::vector<int32_t> par((size_t)5 * p->c_out_pad, 0);
     for (int co = 0; co < p->c_out_pad; ++co) {
@@ -1681,6 +1725,10 @@ int umma_setup(iconv_plan_t *p)
     if (p->window) {
         CUtensorMap probe2;     // the tiled patch map must be encodable as well
         if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
+    }
+    if (p->epi == EPI_NARROW && !p->window) {
+        set_error("tensor-core path: a narrow or unaligned 8-bit output needs window mode");
+        return ICONV_ERR_UNSUPPORTED;
     }
     if (p->pair16 && !p->window) {
         set_error("tensor-core path: paired taps need window mode");
@@ -1762,9 +1810,12 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.c_b = p->params_packed + 4 * (size_t)p->c_out_pad;
     const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
     CUtensorMap tmap_out, tmap_skip;
-    rc = encode_rows_map((uint8_t *)a.out + (size_t)d.out_c_offset * esz, esz, d.c_out, d.out_c_total, u.m_total,
-                         p->piece_bytes, &tmap_out);
-    if (rc != ICONV_OK) return rc;
+    memset(&tmap_out, 0, sizeof(tmap_out));
+    if (!p->window) {       // window mode stores from registers
+        rc = encode_rows_map((uint8_t *)a.out + (size_t)d.out_c_offset * esz, esz, d.c_out, d.out_c_total, u.m_total,
+                             p->piece_bytes, &tmap_out);
+        if (rc != ICONV_OK) return rc;
+    }
     tmap_skip = tmap_out;
     if (p->epi == EPI_PROJ) {
         rc = encode_projection_map(p, a.skip, &tmap_skip);      // the slot of the skip map carries the projection's input
@@ -1805,6 +1856,10 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         else umma_window_kernel<E, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);                        \
     } while (0)
         if (p->epi == EPI_FAST) ICONV_WIN(EPI_FAST);
+        else if (p->epi == EPI_NARROW) {
+            if (d.kh == 3 && d.kw == 3 && kj == 2) umma_window_kernel<EPI_NARROW, 3, 3, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
+            else umma_window_kernel<EPI_NARROW, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
+        }
         else ICONV_WIN(EPI_SAFE);
 #undef ICONV_WIN
         ICONV_CUDA_TRY(cudaGetLastError());

@@ -39,12 +39,8 @@ int choose_kernel(iconv_plan_t *p)
         p->kernel = ICONV_KERNEL_STEM;
         return stem_setup(p);
     }
-    // AUTO: thin layers first (they are bandwidth-bound), then the tensor-core path,
-    // the direct kernel for whatever is left.
-    if (thin_supported(p) == ICONV_OK) {
-        p->kernel = ICONV_KERNEL_THIN;
-        return thin_setup(p);
-    }
+    // AUTO: the repacking paths of the first layers (tensor cores), then the thin layers on
+    // the CUDA cores, then the tensor-core path proper, the direct kernel for whatever is left.
     if (stem_supported(p) == ICONV_OK) {
         const int rc = stem_setup(p);
         if (rc == ICONV_OK) {
@@ -52,6 +48,23 @@ int choose_kernel(iconv_plan_t *p)
             return ICONV_OK;
         }
         if (rc != ICONV_ERR_UNSUPPORTED) return rc;
+    }
+    if (umma_narrow(p->d) && umma_supported(p) == ICONV_OK) {
+        // a narrow output whose reduction is wide enough for the tensor cores (window mode, byte stores)
+        const int rc = umma_setup(p);
+        if (rc == ICONV_OK) {
+            p->kernel = ICONV_KERNEL_UMMA;
+            return ICONV_OK;
+        }
+        if (rc != ICONV_ERR_UNSUPPORTED) return rc;
+        cudaFree(p->w_packed);
+        p->w_packed = nullptr;
+        cudaFree(p->params_packed);
+        p->params_packed = nullptr;
+    }
+    if (thin_supported(p) == ICONV_OK) {
+        p->kernel = ICONV_KERNEL_THIN;
+        return thin_setup(p);
     }
     if (umma_supported(p) == ICONV_OK) {
         const int rc = umma_setup(p);

@@ -48,6 +48,7 @@ int plan_create(const iconv_desc *desc, int pair16, iconv_plan_t **plan_out);
 int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int umma_supported(const iconv_plan_t *p);   // ICONV_OK or the reason it is not
+bool umma_narrow(const iconv_desc &d);      // an 8-bit output too narrow or unaligned for 16-byte stores that window mode could still take
 int umma_setup(iconv_plan_t *p);
 int umma_init_once();                        // driver entry points, shared-memory opt-in; allocates nothing
 int umma_geometry(iconv_plan_t *p);           // host-only tile / pipeline / epilogue geometry

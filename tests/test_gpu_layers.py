@@ -274,6 +274,71 @@ def test_stem_path_matches_oracle(shape, in_dtype):
     assert fam == B.KERNEL_STEM and np.array_equal(got, want)      # AUTO picks it too
 
 
+ROWS_SHAPES = [
+    # single-channel images repacked for the tensor cores: n, h, w, c_out, kh, kw, pad
+    (2, 40, 48, 64, 3, 3, 1),           # VDSR first layer
+    (2, 21, 37, 64, 5, 5, 2),           # VRCNN first layer, ragged sizes
+    (1, 37, 150, 32, 3, 5, 2),          # a filter that is not square, padding beyond what it needs vertically
+    (3, 19, 9, 48, 7, 2, 0),            # no padding, output narrower than the image
+    (1, 18, 140, 64, 1, 16, 3),         # the widest filter row the repack holds
+]
+
+
+@pytest.mark.parametrize("shape", ROWS_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("in_dtype", [B.U8_RAW128, B.U8, B.S8])
+def test_single_channel_repack_path_matches_oracle(shape, in_dtype):
+    n, h, w, c_out, kh, kw, pad = shape
+    rng = np.random.default_rng(sum(shape) + in_dtype)
+    X = rng.integers(0, 256, size=(n, h, w, 1), dtype=np.uint8)
+    if in_dtype == B.S8:
+        X = X.view(np.int8)
+    W = np.clip(np.floor(rng.normal(0, 40, size=(c_out, kh, kw, 1)) + 0.5), -127, 127).astype(np.int8)
+    b = rng.integers(-2048, 2049, size=(c_out,), dtype=np.int32)
+    h_i = np.array([int(40 * 74 * np.sqrt(kh * kw) * 2)], dtype=np.int32)
+    mul = np.array([int(np.floor(255.0 * 2.0 ** 16 / h_i[0] + 0.5))], dtype=np.int32)
+    shift = np.array([16], dtype=np.int32)
+    want = oracle_conv(X, W, b, mul, shift, h_i, pad=pad, in_dtype=in_dtype)
+    assert 0.05 < (want == 0).mean() < 0.95
+    for kernel in (B.KERNEL_STEM, B.KERNEL_AUTO):
+        got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=pad, in_dtype=in_dtype, kernel=kernel)
+        assert fam == B.KERNEL_STEM
+        bad = np.argwhere(got != want)
+        assert bad.shape[0] == 0, "%d mismatches, first at %s: got %s want %s" % (
+            bad.shape[0], bad[0], got[tuple(bad[0])], want[tuple(bad[0])])
+
+
+NARROW_SHAPES = [
+    # 8-bit outputs too narrow or too oddly placed for 16-byte stores: n, h, w, c_in, c_out, k, pad, out_c_total, out_c_offset
+    (2, 40, 48, 64, 1, 3, 1, 1, 0),         # VDSR last layer
+    (1, 37, 150, 48, 1, 3, 1, 1, 0),        # VRCNN last layer, block tiling with ragged edges
+    (2, 21, 19, 32, 3, 5, 2, 3, 0),         # three channels (a colour picture)
+    (1, 30, 26, 64, 24, 3, 1, 40, 9),       # 24 channels at an odd offset of a wider tensor
+    (2, 16, 16, 16, 7, 1, 0, 7, 0),         # a 1x1 layer
+]
+
+
+@pytest.mark.parametrize("shape", NARROW_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("skip_dtype", [-1, B.U8_RAW128, B.S8], ids=["noskip", "skipraw", "skips8"])
+def test_narrow_outputs_on_the_tensor_cores_match_oracle(shape, skip_dtype):
+    n, h, w, c_in, c_out, k, pad, out_c_total, out_c_offset = shape
+    X, W, b, mul, shift, h_i = _layer(sum(shape) + 5, n, h, w, c_in, c_out, k, per_channel=(c_out == 24))
+    ho, wo = h + 2 * pad - k + 1, w + 2 * pad - k + 1
+    kw = dict(pad=pad, out_c_total=out_c_total, out_c_offset=out_c_offset)
+    if skip_dtype >= 0:
+        S = np.random.default_rng(7).integers(0, 256, size=(n, ho, wo, c_out + 2), dtype=np.uint8)
+        if skip_dtype == B.S8:
+            S = S.view(np.int8)
+        kw.update(skip=S, skip_dtype=skip_dtype, skip_c_offset=1, skip_mul=int(h_i[0]) // 300, skip_shift=1)
+    want = oracle_conv(X, W, b, mul, shift, h_i, **kw)
+    text = []
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, kernel=B.KERNEL_UMMA, describe=text, **kw)
+    assert fam == B.KERNEL_UMMA and "window" in text[0], text
+    bad = np.argwhere(got != want)
+    assert bad.shape[0] == 0, "%d mismatches, first at %s: got %s want %s" % (
+        bad.shape[0], bad[0], got[tuple(bad[0])], want[tuple(bad[0])])
+    assert np.unique(want[..., out_c_offset:out_c_offset + c_out]).size > 8
+
+
 def test_mma_issue_rate_probe_reports_a_plausible_peak():
     tops, cycles = B.iconv_probe_mma_rate(256, 20000)
     assert 100.0 <= cycles <= 400.0          # 128 cycles per M128 N256 K32 instruction at the nominal rate
@@ -310,27 +375,38 @@ def test_thin_kernels_match_oracle(shape, in_dtype):
         assert (want == 0).mean() < 0.95 and np.unique(want).size > 8
     else:
         assert 0.05 < (want == 0).mean() < 0.95
+    # AUTO picks it too, except where a single-channel layer can be repacked for the tensor cores
+    # or a single-channel output comes out of the tensor-core window mode byte by byte
+    repack = c_in == 1 and stride == 1 and k > 1 and c_out >= 32
+    narrow = c_out == 1 and c_in <= 128 and h * w >= 256
     got, fam = gpu_conv(X, W, b, mul, shift, h_i, stride=stride, pad=pad, in_dtype=in_dtype)
-    assert fam == B.KERNEL_THIN and np.array_equal(got, want)        # AUTO picks it too
+    assert fam == (B.KERNEL_STEM if repack else B.KERNEL_UMMA if narrow else B.KERNEL_THIN) and np.array_equal(got, want)
 
 
 def test_thin_kernels_variants():
     # c_in = 1 into a channel offset of a wider tensor, per-channel parameters, wide (64-bit) Eq. 4
     X, W, b, mul, shift, h_i = _layer(91, 2, 17, 13, 1, 32, 3, B.U8_RAW128, per_channel=True)
-    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.U8_RAW128, out_c_total=64, out_c_offset=16)
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.U8_RAW128, out_c_total=64, out_c_offset=16,
+                        kernel=B.KERNEL_THIN)
     want = oracle_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.U8_RAW128, out_c_total=64, out_c_offset=16)
     assert fam == B.KERNEL_THIN and np.array_equal(got, want)
-    got, fam = gpu_conv(X, W, b, mul * 4096, shift + 12, h_i, pad=1, in_dtype=B.U8_RAW128)      # h_i * mul >= 2^32
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, in_dtype=B.U8_RAW128, out_c_total=64, out_c_offset=16)
+    assert fam == B.KERNEL_STEM and np.array_equal(got, want)      # repacked: per-channel parameters on the tensor-core path
+    # h_i * mul >= 2^32: no 32-bit epilogue, so no window mode, so AUTO leaves the layer to the thin kernel
+    got, fam = gpu_conv(X, W, b, mul * 4096, shift + 12, h_i, pad=1, in_dtype=B.U8_RAW128)
     want = oracle_conv(X, W, b, mul * 4096, shift + 12, h_i, pad=1, in_dtype=B.U8_RAW128)
     assert fam == B.KERNEL_THIN and np.array_equal(got, want)
     # c_out = 1 with the global residual: raw image skip, no BReLU, zero point 128 (the regression output)
     X, W, b, mul, shift, h_i = _layer(92, 2, 18, 22, 64, 1, 3)
     S = np.random.default_rng(5).integers(0, 256, size=(2, 18, 22, 1), dtype=np.uint8)
     kw = dict(pad=1, brelu=False, out_zero=128, skip=S, skip_dtype=B.U8_RAW128, skip_mul=3000, skip_shift=2)
-    got, fam = gpu_conv(X, W, b, [20], [14], [0], **kw)
+    got, fam = gpu_conv(X, W, b, [20], [14], [0], kernel=B.KERNEL_THIN, **kw)
     want = oracle_conv(X, W, b, [20], [14], [0], **kw)
     assert fam == B.KERNEL_THIN and np.array_equal(got, want)
     assert (want == 0).any() and (want == 255).any() and ((want > 0) & (want < 255)).mean() > 0.3
+    text = []
+    got, fam = gpu_conv(X, W, b, [20], [14], [0], describe=text, **kw)       # AUTO: the tensor cores, byte stores
+    assert fam == B.KERNEL_UMMA and "window" in text[0] and np.array_equal(got, want)
     # c_out = 1, raw int32 output
     got, fam = gpu_conv(X, W, b, [1], [0], [0], pad=1, out_dtype=B.I32, brelu=False)
     want = oracle_conv(X, W, b, [1], [0], [0], pad=1, out_dtype=B.I32, brelu=False)
