@@ -86,6 +86,7 @@ struct UmmaArgs {
     int skip_half;                  // 2^(skip_shift-1), or 0
     unsigned skip_xor;              // 0x80808080 turns int8 skip bytes into offset-binary
     int tail;                       // 1: out_zero / out_lo / out_hi are not provably no-ops
+    int group_uniform;              // per-channel parameters that are equal within every group of 16 channels
     const int32_t *c_a;             // [c_out_pad] per-channel additive constant of the variant
     const int32_t *c_b;             // [c_out_pad] projection bias (64-bit form of EPI_PROJ)
     const int32_t *c_mul, *c_shift, *c_h;   // [c_out_pad] copies for per-channel layers
@@ -367,7 +368,7 @@ struct EpiScalars {
     int skip_mul, skip_shift;
     unsigned skip_xor;
     int out_zero, out_lo, out_hi, tail;
-    int per_channel, proj32, brelu, skip_dtype, out_dtype, c_out;
+    int per_channel, group_uniform, proj32, brelu, skip_dtype, out_dtype, c_out;
 };
 
 __device__ __forceinline__ EpiScalars epi_scalars(const ConvArgs &a, const UmmaArgs &u)
@@ -376,9 +377,21 @@ __device__ __forceinline__ EpiScalars epi_scalars(const ConvArgs &a, const UmmaA
     e.q_mul = u.q_mul; e.q_shift = u.q_shift; e.q_half = u.q_half; e.q_h = u.q_h;
     e.skip_mul = a.skip_mul; e.skip_shift = a.skip_shift; e.skip_xor = u.skip_xor;
     e.out_zero = a.out_zero; e.out_lo = a.out_lo; e.out_hi = a.out_hi; e.tail = u.tail;
-    e.per_channel = a.per_channel; e.proj32 = u.proj32; e.brelu = a.brelu; e.skip_dtype = a.skip_dtype;
+    e.per_channel = a.per_channel && !u.group_uniform; e.group_uniform = u.group_uniform; e.proj32 = u.proj32; e.brelu = a.brelu; e.skip_dtype = a.skip_dtype;
     e.out_dtype = a.out_dtype; e.c_out = a.c_out;
     return e;
+}
+
+// Per-channel parameters that are uniform within each group of 16 channels (merged sibling
+// branches): the group's own scalars take the place of the layer's, three loads per group.
+__device__ __forceinline__ EpiScalars group_scalars(const EpiScalars &s, const UmmaArgs &u, int co0)
+{
+    EpiScalars g = s;
+    if (s.group_uniform) {
+        g.q_mul = __ldg(u.c_mul + co0); g.q_shift = __ldg(u.c_shift + co0); g.q_h = __ldg(u.c_h + co0);
+        g.q_half = (int)(1u << (g.q_shift - 1));
+    }
+    return g;
 }
 
 // BReLU clamp + 32-bit Eq. 4 (+ zero point / range when they are not provable no-ops)
@@ -815,7 +828,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         tmem_ld_wait();
                         if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_piece + (uint32_t)(cc + 16), hf ? accA : accB);
                         int V[16];
-                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, es, a, u);
+                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, group_scalars(es, u, co0), a, u);
                         if (esz_rt == 4) {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) {
@@ -1131,7 +1144,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     tmem_ld_wait();
                     if (gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
                     int V[16];
-                    epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), es, a, u);
+                    epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), group_scalars(es, u, co0), a, u);
                     uint4 o;
                     if (EPI == EPI_FAST || a.out_dtype == ICONV_U8) {
                         o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
@@ -1312,6 +1325,17 @@ int choose_projection_epilogue(const iconv_desc &d, int c_out_pad, std::vector<i
     return EPI_PROJ;
 }
 
+// Per-channel parameters equal within every group of 16 channels?
+bool group_uniform(const iconv_desc &d)
+{
+    if (!d.per_channel) return false;
+    for (int co = 0; co < d.c_out; ++co) {
+        const int g = co / 16 * 16;
+        if (d.mul[co] != d.mul[g] || d.shift[co] != d.shift[g] || d.h_i[co] != d.h_i[g]) return false;
+    }
+    return true;
+}
+
 // Picks the cheapest epilogue whose 32-bit arithmetic is provably exact for this layer and
 // fills the per-channel additive constant of that variant (c_a, c_out_pad entries).
 //   worst[co] = sum |w| * max|x|: no accumulator of channel co can exceed it in magnitude.
@@ -1349,13 +1373,14 @@ int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_
         skip_bound = ((255ll * d.skip_mul) >> d.skip_shift) + 1;
     }
     // the fast form: no clamp before the multiplication, the u8 saturation does both clamps
-    bool fast = !d.per_channel && d.out_dtype == ICONV_U8 && d.out_zero == 0 && d.out_lo == 0 && d.out_hi == 255 &&
+    bool fast = (!d.per_channel || group_uniform(d)) && d.out_dtype == ICONV_U8 && d.out_zero == 0 && d.out_lo == 0 && d.out_hi == 255 &&
                 d.skip_dtype != ICONV_I32;
     if (fast) {
-        const long long mul = d.mul[0], half = 1ll << (d.shift[0] - 1);
-        // BReLU's upper clamp may only be dropped when h_i already maps to the saturation bound
-        if ((long long)(((unsigned long long)d.h_i[0] * (unsigned long long)mul + (unsigned long long)half) >> d.shift[0]) < 255) fast = false;
         for (int co = 0; co < d.c_out && fast; ++co) {
+            const int q = d.per_channel ? co : 0;
+            const long long mul = d.mul[q], half = 1ll << (d.shift[q] - 1);
+            // BReLU's upper clamp may only be dropped when h_i already maps to the saturation bound
+            if ((long long)(((unsigned long long)d.h_i[q] * (unsigned long long)mul + (unsigned long long)half) >> d.shift[q]) < 255) fast = false;
             long long sw = 0;
             const int8_t *wr = d.weights + (long long)co * K;
             for (long long k = 0; k < K; ++k) sw += wr[k] < 0 ? -(long long)wr[k] : wr[k];
@@ -1364,7 +1389,10 @@ int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_
         }
         if (fast) {
             if (!skip8)
-                for (int co = 0; co < d.c_out; ++co) c_a[co] = (int32_t)((long long)d.bias[co] * mul + half);
+                for (int co = 0; co < d.c_out; ++co) {
+                    const int q = d.per_channel ? co : 0;
+                    c_a[co] = (int32_t)((long long)d.bias[co] * d.mul[q] + (1ll << (d.shift[q] - 1)));
+                }
             return skip8 ? EPI_FAST_SKIP8 : EPI_FAST;
         }
     }
@@ -1717,6 +1745,7 @@ int umma_setup(iconv_plan_t *p)
     }
     ICONV_CUDA_TRY(cudaMalloc((void **)&p->params_packed, par.size() * sizeof(int32_t)));
     ICONV_CUDA_TRY(cudaMemcpy(p->params_packed, par.data(), par.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    p->group_uniform = d.out_dtype != ICONV_I32 && group_uniform(d) ? 1 : 0;
     p->q_mul = d.out_dtype != ICONV_I32 ? d.mul[0] : 1;
     p->q_shift = d.out_dtype != ICONV_I32 ? d.shift[0] : 0;
     p->q_h = d.out_dtype != ICONV_I32 ? d.h_i[0] : 0;
@@ -1803,6 +1832,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.skip_half = (d.skip_dtype >= 0 && d.skip_shift > 0 && d.skip_shift <= 31) ? (int)(1u << (d.skip_shift - 1)) : 0;
     u.skip_xor = d.skip_dtype == ICONV_S8 ? 0x80808080u : 0u;
     u.tail = p->tail;
+    u.group_uniform = p->group_uniform;
     u.c_a = p->params_packed;
     u.c_mul = p->params_packed + p->c_out_pad;
     u.c_shift = p->params_packed + 2 * (size_t)p->c_out_pad;

@@ -42,12 +42,18 @@ def net_input(net: Net, first: int = 0, count=None) -> np.ndarray:
 class Network:
     """Plans every layer once; ``forward`` enqueues the whole network on the current stream."""
 
-    def __init__(self, net: Net, params: dict, n=None, device="cuda:0", kernel=B.KERNEL_AUTO, fuse_projection=True):
+    def __init__(self, net: Net, params: dict, n=None, device="cuda:0", kernel=B.KERNEL_AUTO, fuse_projection=True,
+                 merge_branches=True):
         """fuse_projection: run a projection skip (a "raw" convolution whose int32 output only feeds
-        the next layer's skip) inside that layer's kernel; its int32 tensor is then never written."""
+        the next layer's skip) inside that layer's kernel; its int32 tensor is then never written.
+        merge_branches: plan two convolutions that read the same tensor and write neighbouring
+        channel ranges of the same concatenation (a variable-filter-size block) as one layer: the
+        smaller filter sits zero-padded in the middle of the larger one, every channel keeps its
+        own bias, h_i, mul and shift.  The sums only gain zero terms, so the bytes are the same."""
         self.net, self.n, self.device = net, net.n if n is None else n, torch.device(device)
         self.plans, self.steps, self.tensors = {}, [], {}
         self.fused = {}          # name of a fused projection op -> name of the layer that absorbed it
+        self.merged = {}         # name of a branch convolution -> name of the sibling whose plan runs both
         self._pending = {}
         torch.cuda.set_device(self.device)
         convs = {op.name: op for op in net.convs()}
@@ -60,8 +66,20 @@ class Network:
                         fusable[op.dst] = op
         for name, t in net.tensors.items():
             self.tensors[name] = torch.zeros((self.n, t.h, t.w, t.c), dtype=_TORCH[t.dtype], device=self.device)
+        partner = {}             # first op of a merged pair -> second
+        if merge_branches and kernel in (B.KERNEL_AUTO, B.KERNEL_UMMA):
+            for a, b in zip(net.ops, net.ops[1:]):
+                if a.name not in self.merged and self._mergeable(a, b, params):
+                    partner[a.name] = b
+                    self.merged[b.name] = a.name
         for op in net.ops:
             src, dst = net.tensors[op.src], net.tensors[op.dst]
+            if op.name in self.merged:
+                continue
+            if op.name in partner:
+                self.plans[op.name] = self._plan_merged(op, partner[op.name], params, kernel)
+                self.steps.append(("conv", op, None))
+                continue
             if isinstance(op, MaxPool):
                 self.steps.append(("max", op, None))
             elif isinstance(op, AvgPool):
@@ -103,6 +121,41 @@ class Network:
                 self.plans[op.name] = B.iconv_plan(**kw)
                 self.steps.append(("conv", op, None))
 
+    def _mergeable(self, a, b, params) -> bool:
+        if not (isinstance(a, Conv) and isinstance(b, Conv)):
+            return False
+        if a.role == "raw" or b.role == "raw" or a.skip or b.skip or a.dst == self.net.output:
+            return False
+        same = (a.src == b.src and a.dst == b.dst and a.c_in == b.c_in and a.in_c_offset == b.in_c_offset and
+                a.in_dtype == b.in_dtype and a.stride == b.stride and b.out_c_offset == a.out_c_offset + a.c_out)
+        if not same or (a.k - b.k) % 2 or a.pad - b.pad != (a.k - b.k) // 2:
+            return False
+        pa, pb = params[a.name], params[b.name]
+        return all(pa[k] == pb[k] for k in ("brelu", "out_lo", "out_hi", "out_zero")) and pa["brelu"] == 1 and \
+            len(pa["mul"]) == 1 and len(pb["mul"]) == 1
+
+    def _plan_merged(self, a, b, params, kernel):
+        """One plan for the sibling branches a and b (see merge_branches)."""
+        net = self.net
+        src, dst = net.tensors[a.src], net.tensors[a.dst]
+        k = max(a.k, b.k)
+        W = np.zeros((a.c_out + b.c_out, k, k, a.c_in), dtype=np.int8)
+        row = 0
+        for op in (a, b):
+            w_f = gen.weights_f(net.seed, op.layer, op.c_out, op.k, op.k, op.c_in)
+            o = (k - op.k) // 2
+            W[row:row + op.c_out, o:o + op.k, o:o + op.k, :] = B.iq_quantize_weights(w_f, params[op.name]["delta"])
+            row += op.c_out
+        per = lambda key: np.concatenate([np.repeat(np.asarray(params[op.name][key], dtype=np.int32), op.c_out) for op in (a, b)])
+        pa = params[a.name]
+        big = a if a.k >= b.k else b
+        return B.iconv_plan(n=self.n, h=src.h, w=src.w, c_in=a.c_in, c_out=a.c_out + b.c_out, kh=k, kw=k, stride=a.stride,
+                            pad=big.pad, in_dtype=B.DTYPE_CODE[a.in_dtype], in_c_total=src.c, in_c_offset=a.in_c_offset,
+                            out_c_total=dst.c, out_c_offset=a.out_c_offset, weights=W,
+                            bias=np.concatenate([gen.bias_i32(net.seed, op.layer, op.c_out) for op in (a, b)]),
+                            kernel=kernel, out_dtype=B.U8, brelu=1, mul=per("mul"), shift=per("shift"), h_i=per("h_i"),
+                            out_lo=pa["out_lo"], out_hi=pa["out_hi"], out_zero=pa["out_zero"])
+
     def _try_fuse(self, op, fusable, params, kernel) -> bool:
         """Remember a projection op so that its consumer plans it as a fused skip."""
         src = self.net.tensors[op.src]
@@ -127,6 +180,7 @@ class Network:
         for op in self.net.convs():
             dst = self.net.tensors[op.dst]
             name = self.fused.get(op.name, op.name)          # a fused projection counts with the layer that runs it
+            name = self.merged.get(name, name)               # and so does a merged sibling branch
             out[name] = out.get(name, 0) + self.n * dst.h * dst.w * op.c_out * op.c_in * op.k * op.k
         return out
 
@@ -144,6 +198,9 @@ class Network:
             b = self.n * src.h * src.w * op.c_in + op.c_out * op.c_in * op.k * op.k + 4 * op.c_out
             if op.name in self.fused:
                 name = self.fused[op.name]
+            elif op.name in self.merged:                     # shares its sibling's input read
+                name = self.merged[op.name]
+                b += self.n * dst.h * dst.w * op.c_out * esz[dst.dtype] - self.n * src.h * src.w * op.c_in
             else:
                 name = op.name
                 b += self.n * dst.h * dst.w * op.c_out * esz[dst.dtype]

@@ -22,16 +22,18 @@ SMALL = [
 
 @pytest.mark.parametrize("net", SMALL, ids=lambda n: n.name)
 @pytest.mark.parametrize("kernel,fuse", [(B.KERNEL_DIRECT, False), (B.KERNEL_AUTO, False), (B.KERNEL_AUTO, True)],
-                         ids=["direct", "auto", "auto-fused-projection"])
+                         ids=["direct", "auto", "auto-fused"])
 def test_every_layer_of_small_networks_matches_oracle(net, kernel, fuse):
     params = ON.calibrate(net)
     x = ON.net_input(net)
     want = ON.forward(net, params, x)
-    g = Network(net, params, kernel=kernel, fuse_projection=fuse)
+    g = Network(net, params, kernel=kernel, fuse_projection=fuse, merge_branches=fuse)
     out = g.forward(torch.from_numpy(x).cuda())
     B.iconv_check(torch.cuda.current_stream().cuda_stream)
     if fuse and net.name.startswith("resnet"):
         assert len(g.fused) == 4          # one projection per stage, each absorbed by its block's closing layer
+    if net.name.startswith("vrcnn"):      # both variable-filter-size blocks run as one layer each
+        assert len(g.merged) == (2 if fuse else 0) and len(g.plans) == (4 if fuse else 6)
     for op in net.ops:
         if op.name in g.fused:            # its int32 tensor never exists; the absorbing layer's output is checked
             continue
