@@ -828,7 +828,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         tmem_ld_wait();
                         if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_piece + (uint32_t)(cc + 16), hf ? accA : accB);
                         int V[16];
-                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, group_scalars(es, u, co0), a, u);
+                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, es, a, u);
                         if (esz_rt == 4) {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) {
@@ -905,6 +905,44 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)u.tmem_cols);
+    }
+}
+
+// Window-mode epilogue of one warp and tile: groups of 16 columns from TMEM (the first one
+// already requested into accA), each through the layer's epilogue and out with one 16-byte
+// store per pixel.  NG: the number of groups when known at compile time (0: `ngroups`).
+// GU: per-channel parameters that are uniform per group (fetched group by group).
+template <int EPI, int NG, bool GU>
+__device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, uint8_t *ocol, bool valid, int col_lo, int ngroups,
+                                              int *accA, int *accB, const EpiScalars &es, const ConvArgs &a, const UmmaArgs &u)
+{
+    const int ng = NG ? NG : ngroups;
+#pragma unroll
+    for (int gi = 0; gi < (NG ? NG : 16); gi += 2) {
+        if (!NG && gi >= ng) break;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const int gcur = gi + hf;
+            if (gcur >= ng) break;
+            const int co0 = col_lo + (gcur << 4);
+            int4 ca[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + 4 * gcur + g);
+            tmem_ld_wait();
+            if (gcur + 1 < ng) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
+            int V[16];
+            if (GU) epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), group_scalars(es, u, co0), a, u);
+            else epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), es, a, u);
+            uint4 o;
+            if (EPI == EPI_FAST || a.out_dtype == ICONV_U8) {
+                o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
+                o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
+            } else {
+                o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
+                o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
+            }
+            if (valid && co0 < a.c_out) *(uint4 *)(ocol + (gcur << 4)) = o;
+        }
     }
 }
 
@@ -1131,30 +1169,16 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     }
                 }
             }
-            for (int gi = 0; EPI != EPI_NARROW && gi < ngroups; gi += 2) {
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const int gcur = gi + hf;
-                    if (gcur >= ngroups) break;
-                    const int co0 = col_lo + (gcur << 4);
-                    int4 ca[4];
-                    const int4 *cap = (const int4 *)(u.c_a + co0);
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + g);
-                    tmem_ld_wait();
-                    if (gcur + 1 < ngroups) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
-                    int V[16];
-                    epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), group_scalars(es, u, co0), a, u);
-                    uint4 o;
-                    if (EPI == EPI_FAST || a.out_dtype == ICONV_U8) {
-                        o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
-                        o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
-                    } else {
-                        o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
-                        o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
-                    }
-                    if (valid && co0 < a.c_out) *(uint4 *)(orow + co0) = o;
-                }
+            if (EPI != EPI_NARROW) {
+                const int4 *cap = (const int4 *)(u.c_a + col_lo);
+                uint8_t *ocol = orow + col_lo;
+                // the usual widths get straight-line code: every offset an immediate, no loop control
+                if (es.group_uniform) window_groups<EPI, 0, true>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 4) window_groups<EPI, 4, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 3) window_groups<EPI, 3, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 2) window_groups<EPI, 2, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 1) window_groups<EPI, 1, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else window_groups<EPI, 0, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
             }
             tc_fence_before();
             __syncwarp();
@@ -1338,8 +1362,10 @@ bool group_uniform(const iconv_desc &d)
 
 // Picks the cheapest epilogue whose 32-bit arithmetic is provably exact for this layer and
 // fills the per-channel additive constant of that variant (c_a, c_out_pad entries).
+// group_fast: the fast forms may also take per-channel parameters that are uniform per group of
+// 16 channels (window mode fetches a group's scalars; the im2col kernel does not).
 //   worst[co] = sum |w| * max|x|: no accumulator of channel co can exceed it in magnitude.
-int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_a, int &tail)
+int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_a, int &tail, bool group_fast)
 {
     const long long K = (long long)d.kh * d.kw * d.c_in;
     const long long xmax = d.in_dtype == ICONV_U8 ? 255 : 128;
@@ -1373,7 +1399,7 @@ int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_
         skip_bound = ((255ll * d.skip_mul) >> d.skip_shift) + 1;
     }
     // the fast form: no clamp before the multiplication, the u8 saturation does both clamps
-    bool fast = (!d.per_channel || group_uniform(d)) && d.out_dtype == ICONV_U8 && d.out_zero == 0 && d.out_lo == 0 && d.out_hi == 255 &&
+    bool fast = (!d.per_channel || (group_fast && group_uniform(d))) && d.out_dtype == ICONV_U8 && d.out_zero == 0 && d.out_lo == 0 && d.out_hi == 255 &&
                 d.skip_dtype != ICONV_I32;
     if (fast) {
         for (int co = 0; co < d.c_out && fast; ++co) {
@@ -1726,13 +1752,24 @@ int umma_setup(iconv_plan_t *p)
         p->epi = choose_projection_epilogue(d, p->c_out_pad, c_a, c_b, p->tail, p->proj32);
         if (p->epi < 0) { set_error("tensor-core path: Eq. 4 of a layer with a fused projection must fit 32 bits"); return ICONV_ERR_UNSUPPORTED; }
     } else {
-        p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail);
+        p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail, true);
         c_b.assign((size_t)p->c_out_pad, 0);
         if (umma_narrow(d)) {
             p->epi = EPI_NARROW;
             p->tail = 1;
             for (int co = 0; co < d.c_out; ++co) c_a[co] = d.bias[co];
         }
+    }
+    p->group_uniform = d.out_dtype != ICONV_I32 && group_uniform(d) ? 1 : 0;
+    window_plan(p);
+    if (p->window) {
+        CUtensorMap probe2;     // the tiled patch map must be encodable as well
+        if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
+    }
+    if (p->group_uniform && !p->window) {
+        // the im2col kernel reads per-channel parameters channel by channel
+        p->group_uniform = 0;
+        if (!d.proj_weights && p->epi != EPI_NARROW) p->epi = choose_epilogue(d, p->c_out_pad, c_a, p->tail, false);
     }
     std::vector<int32_t> par((size_t)5 * p->c_out_pad, 0);
     for (int co = 0; co < p->c_out_pad; ++co) {
@@ -1745,16 +1782,10 @@ int umma_setup(iconv_plan_t *p)
     }
     ICONV_CUDA_TRY(cudaMalloc((void **)&p->params_packed, par.size() * sizeof(int32_t)));
     ICONV_CUDA_TRY(cudaMemcpy(p->params_packed, par.data(), par.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
-    p->group_uniform = d.out_dtype != ICONV_I32 && group_uniform(d) ? 1 : 0;
     p->q_mul = d.out_dtype != ICONV_I32 ? d.mul[0] : 1;
     p->q_shift = d.out_dtype != ICONV_I32 ? d.shift[0] : 0;
     p->q_h = d.out_dtype != ICONV_I32 ? d.h_i[0] : 0;
 
-    window_plan(p);
-    if (p->window) {
-        CUtensorMap probe2;     // the tiled patch map must be encodable as well
-        if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
-    }
     if (p->epi == EPI_NARROW && !p->window) {
         set_error("tensor-core path: a narrow or unaligned 8-bit output needs window mode");
         return ICONV_ERR_UNSUPPORTED;
