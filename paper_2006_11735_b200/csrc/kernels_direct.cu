@@ -216,12 +216,53 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const uint8_t *x, uint8_t 
     }
 }
 
+// The 3x3 stride-2 pad-1 pooling of the ResNet-shaped networks: the nine loads carry no branch
+// (a tap outside the image re-reads the nearest row or column inside it, which the window
+// holds anyway, so the maximum is unchanged) and are all in flight together; one thread per
+// (output pixel, group of 16 channels), 32-bit index arithmetic.
+__global__ void __launch_bounds__(256) maxpool_3x3s2_kernel(const uint8_t *__restrict__ x, uint8_t *__restrict__ out, unsigned total,
+                                                            int h, int w, int cg, int h_out, int w_out)
+{
+    const unsigned e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const unsigned pix = e / (unsigned)cg;
+    const int g = (int)(e - pix * (unsigned)cg);
+    const unsigned row = pix / (unsigned)w_out;               // image * h_out + oh
+    const int ow = (int)(pix - row * (unsigned)w_out);
+    const unsigned in = row / (unsigned)h_out;
+    const int oh = (int)(row - in * (unsigned)h_out);
+    const uint4 *base = (const uint4 *)x + (size_t)in * h * w * cg + g;
+    uint4 v[9];
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int ih = min(max(2 * oh - 1 + r, 0), h - 1);
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            const int iw = min(max(2 * ow - 1 + s, 0), w - 1);
+            v[r * 3 + s] = __ldg(base + (size_t)(ih * w + iw) * cg);
+        }
+    }
+    uint4 m = v[0];
+#pragma unroll
+    for (int t = 1; t < 9; ++t) {
+        m.x = __vmaxu4(m.x, v[t].x); m.y = __vmaxu4(m.y, v[t].y);
+        m.z = __vmaxu4(m.z, v[t].z); m.w = __vmaxu4(m.w, v[t].w);
+    }
+    ((uint4 *)out)[e] = m;
+}
+
 int launch_maxpool(const void *x, void *out, int n, int h, int w, int c, int k, int stride, int pad,
                    cudaStream_t stream)
 {
     const int h_out = (h + 2 * pad - k) / stride + 1, w_out = (w + 2 * pad - k) / stride + 1;
     const long long total = (long long)n * h_out * w_out * (c / 16);
     if (total == 0) return ICONV_OK;
+    if (k == 3 && stride == 2 && pad == 1 && total < (1ll << 31) && (long long)n * h * w * (c / 16) < (1ll << 31)) {
+        maxpool_3x3s2_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>((const uint8_t *)x, (uint8_t *)out, (unsigned)total, h, w,
+                                                                                c / 16, h_out, w_out);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        return ICONV_OK;
+    }
     long long blocks = (total + 255) / 256;
     if (blocks > 148ll * 64) blocks = 148ll * 64;
     maxpool_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)x, (uint8_t *)out, n, h, w, c, k, stride,

@@ -150,7 +150,8 @@ def test_iadd_requant_matches_oracle(n_elems, a_dtype, b_dtype, out_dtype):
 
 def test_pooling_matches_oracle():
     rng = np.random.default_rng(3)
-    for (n, h, w, c, k, s, p) in [(2, 16, 14, 64, 3, 2, 1), (1, 9, 9, 16, 3, 2, 1), (3, 7, 8, 32, 2, 2, 0)]:
+    for (n, h, w, c, k, s, p) in [(2, 16, 14, 64, 3, 2, 1), (1, 9, 9, 16, 3, 2, 1), (3, 7, 8, 32, 2, 2, 0),
+                                  (1, 1, 1, 16, 3, 2, 1), (2, 5, 12, 48, 3, 2, 1), (1, 6, 6, 16, 3, 1, 1)]:
         x = rng.integers(0, 256, size=(n, h, w, c), dtype=np.uint8)
         want = L.maxpool(x, k, s, p)
         out = Fenced(want.shape, np.uint8)
