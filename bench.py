@@ -257,11 +257,25 @@ def main():
     # ---- end to end: pinned host input in, logits out, every step ----
     D.barrier()
     torch.cuda.synchronize(dev)
+    # Two device input buffers and a copy stream, as a serving loop would run it: the batch of
+    # step i+1 crosses PCIe while step i computes.  Every step's input still comes from pinned
+    # host memory inside the timed region, and every step's result goes back to the host.
+    x_bufs = [x_dev, torch.empty_like(x_dev)]
+    copy_stream = torch.cuda.Stream(dev)
+    copied = [torch.cuda.Event() for _ in range(args.steps)]
+    consumed = [torch.cuda.Event() for _ in range(args.steps)]
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record(stream)
-    for _ in range(args.steps):
-        x_dev.copy_(x_host, non_blocking=True)
-        out = g.forward(x_dev)
+    copy_stream.wait_stream(stream)
+    for i in range(args.steps):
+        with torch.cuda.stream(copy_stream):
+            if i >= 2:
+                copy_stream.wait_event(consumed[i - 2])       # the buffer's previous batch has been read
+            x_bufs[i % 2].copy_(x_host, non_blocking=True)
+            copied[i].record(copy_stream)
+        stream.wait_event(copied[i])
+        out = g.forward(x_bufs[i % 2])
+        consumed[i].record(stream)
         logits_host.copy_(out, non_blocking=True)
     e3.record(stream)
     torch.cuda.synchronize(dev)
@@ -292,7 +306,8 @@ def main():
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
                 "clocks": clocks,
                 "e2e": {"value": total_images / (ms_e2e * 1e-3), "unit": UNIT,
-                        "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(logits_host.numel() * logits_host.element_size())},
+                        "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(logits_host.numel() * logits_host.element_size()),
+                        "overlap": "the input copy of step i+1 runs under the compute of step i (two device buffers, one copy stream)"},
                 "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "cpu_baseline": cpu}
         print(json.dumps(line))
     g.close()
