@@ -36,7 +36,8 @@ WORKLOAD = "resnet50_b256_224x224x3"
 WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"),
              "resnet152": ("ResNet-152 int8 images/sec", "resnet152_b128_224x224x3"),
              "vdsr": ("VDSR int8 images/sec", "vdsr_16x256x256x1"),
-             "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1")}
+             "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1"),
+             "vrcnn_hd": ("VRCNN int8 images/sec", "vrcnn_1x1600x2560x1")}
 NOMINAL_INT8_TOPS = 4500.0      # NVIDIA's dense INT8 figure for B200 (context only)
 INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
 

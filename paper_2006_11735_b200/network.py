@@ -23,6 +23,7 @@ PARAMS_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file
 def load_params(name: str) -> dict:
     """Cached per-layer parameters of a full-size configuration (``float.hex`` strings for
     doubles so that the quantisation steps round-trip exactly)."""
+    name = {"vrcnn_hd": "vrcnn"}.get(name, name)      # the single-picture workload runs configuration 3's layers
     with open(os.path.join(PARAMS_DIR, name + ".json")) as f:
         raw = json.load(f)
     for p in raw["layers"].values():

@@ -40,3 +40,38 @@ def test_full_size_configuration_matches_oracle_on_sampled_images(name):
     g.close()
     del g
     torch.cuda.empty_cache()
+
+
+def test_single_2560x1600_picture_matches_oracle_on_crops():
+    """The VRCNN-shaped network on one 2560 x 1600 picture (the size of Table 6's timing).  The
+    oracle runs crops of the picture; away from a crop's artificial edges by the network's
+    receptive-field radius (2 + 2 + 1 + 1 = 6 pixels) every layer of the crop equals the same
+    region of the full picture, and a crop that touches the picture's border shares its padding."""
+    net = N.by_name("vrcnn_hd")
+    params = load_params("vrcnn_hd")
+    g = Network(net, params)
+    assert len(g.merged) == 2
+    x = net_input(net)
+    H, W = x.shape[1], x.shape[2]
+    assert (H, W) == (1600, 2560)
+    out = g.forward(torch.from_numpy(x).cuda())
+    B.iconv_check(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    ch, cw, r = 160, 192, 6
+    # (top, left) of the crop and the slice of the crop that is exact
+    crops = [(0, 0, slice(0, ch - r), slice(0, cw - r)),                           # top-left corner: real padding on two sides
+             (H - ch, W - cw, slice(r, ch), slice(r, cw)),                         # bottom-right corner
+             (0, 1111, slice(0, ch - r), slice(r, cw - r)),                        # top edge
+             (733, 1283, slice(r, ch - r), slice(r, cw - r))]                      # interior, odd offsets
+    small = N.vrcnn(n=1, h=ch, w=cw)
+    for top, left, ys, xs in crops:
+        want = ON.forward(small, params, np.ascontiguousarray(x[:, top:top + ch, left:left + cw, :]))
+        for op in net.ops:
+            got = g.tensors[op.dst][:, top:top + ch, left:left + cw, :].cpu().numpy()
+            a, b = got[:, ys, xs, :], want[op.dst][:, ys, xs, :]
+            assert np.array_equal(a, b), "crop (%d, %d) layer %s: %d mismatches" % (top, left, op.name, (a != b).sum())
+        assert np.unique(want[net.output]).size > 16
+    assert out.shape == (1, H, W, 1)
+    g.close()
+    del g
+    torch.cuda.empty_cache()

@@ -185,6 +185,12 @@ def resnet152(n=128, h=224, w=224, seed=5) -> Net:
     return resnet(n, (3, 8, 36, 3), h, w, seed=seed, name="resnet152")
 
 
+def vrcnn_hd(n=1, h=1600, w=2560, seed=3) -> Net:
+    """The VRCNN-shaped network on one 2560 x 1600 picture (the size the paper times its
+    in-loop filter on, Table 6): the layers, weights and parameters of configuration 3."""
+    return vrcnn(n=n, h=h, w=w, seed=seed)
+
+
 def by_name(name: str, **kw) -> Net:
-    return {"single_conv": single_conv, "vdsr": vdsr, "vrcnn": vrcnn,
+    return {"single_conv": single_conv, "vdsr": vdsr, "vrcnn": vrcnn, "vrcnn_hd": vrcnn_hd,
             "resnet50": resnet50, "resnet152": resnet152}[name](**kw)
