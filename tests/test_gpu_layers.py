@@ -449,3 +449,27 @@ def test_fused_projection_equals_projection_layer_plus_int32_skip(case, skip_mul
     bad = np.argwhere(got != want)
     assert bad.shape[0] == 0, "%d mismatches, first at %s" % (bad.shape[0], bad[0])
     assert 0.02 < (want == 0).mean() < 0.98 and (want == 255).mean() < 0.9
+
+
+@pytest.mark.parametrize("max_int", [127, 63, 31, 15], ids=lambda m: "max_int%d" % m)
+@pytest.mark.parametrize("kernel", [B.KERNEL_UMMA, B.KERNEL_UMMA_IM2COL, B.KERNEL_DIRECT], ids=["plan", "im2col", "direct"])
+def test_activation_bit_depth_sweep_matches_oracle(max_int, kernel):
+    """Activations of 7, 6, 5 and 4 bits (the bit-depth sweep of Table 5): the stored values stay in
+    [0, max_int], the BReLU bound and Eq. 4's (mul, shift) come from Section 3.3 for that max_int,
+    and the output saturates at max_int instead of 255."""
+    from oracle import planner as OP
+    rng = np.random.default_rng(1000 + max_int)
+    n, h, w, c_in, c_out = 2, 22, 26, 64, 64
+    X = rng.integers(0, max_int + 1, size=(n, h, w, c_in), dtype=np.uint8)
+    W = np.clip(np.floor(rng.normal(0, 40, size=(c_out, 3, 3, c_in)) + 0.5), -127, 127).astype(np.int8)
+    b = rng.integers(-2048, 2049, size=(c_out,), dtype=np.int32)
+    h_ri = int(40.0 * (max_int / 2.5) * np.sqrt(c_in * 9) * 2)
+    q = OP.brelu_params_from_h_ri(h_ri, 1.0, max_int)
+    mul, shift, h_i = [q["mul"]], [q["shift"]], [q["h_i"]]
+    S = rng.integers(0, max_int + 1, size=(n, h, w, c_out), dtype=np.uint8)
+    for kw in (dict(pad=1, out_hi=max_int),
+               dict(pad=1, out_hi=max_int, skip=S, skip_dtype=B.U8, skip_mul=int(h_ri / max_int * 64), skip_shift=8)):
+        want = oracle_conv(X, W, b, mul, shift, h_i, **kw)
+        got, fam = gpu_conv(X, W, b, mul, shift, h_i, kernel=kernel, **kw)
+        assert np.array_equal(got, want)
+        assert want.max() == max_int and (want == 0).mean() > 0.02 and ((want > 0) & (want < max_int)).mean() > 0.2
