@@ -236,6 +236,17 @@ ICONV_API int iconcat_plan(int32_t n_branches, const double *ratio_y, const doub
                  int32_t shift_min, int32_t *mul, int32_t *shift,
                  double *delta_scale, double *ratio_y_new, double *ratio_v_min);
 
+/* Section 3.2.2, the n-sigma rule on the GPU: the smallest value among the largest `fraction`
+ * of an int32 feature map Y (its k-th largest element, k = max(1, ceil(count * fraction)); 0.0015
+ * for 3 sigma), never below 1.  This is the h_ri that Eq. 9-13 (`iq_brelu_params`' arithmetic)
+ * turn into mul, shift and h_i; the paper averages it over batches, which is the caller's job.
+ * y: DEVICE pointer to `count` int32 values, 4-byte aligned, read only; bound: HOST.  Exact
+ * (a four-pass radix select, no sorting, no approximation).  Enqueues on `cuda_stream` and
+ * waits for the result; keeps a 2 KB scratch per device, allocated at the first call.
+ * Errors: ICONV_ERR_ARG (null pointer, fraction outside (0, 1]), ICONV_ERR_ALIGN, ICONV_ERR_CUDA.
+ * count = 0 returns 1. */
+ICONV_API int iq_sigma_bound(const int32_t *y, int64_t count, double fraction, int32_t *bound, void *cuda_stream);
+
 /* Measurement aid: how fast this GPU's tensor pipe retires tcgen05.mma kind::i8 (M = 128,
  * N = block_n, K = 32, u8 x s8 -> s32, the instruction of the convolution kernel) when only the
  * instruction stream limits it: operands stay in shared memory, one thread per SM issues `iters`

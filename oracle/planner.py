@@ -70,6 +70,16 @@ def brelu_params_from_h_ri(h_ri: int, ratio_Y: float, max_int: int, shift_min: i
     return dict(h_ri=int(h_ri), mul=mul, shift=shift, ratio_V=ratio_V, h_f=h_f, h_i=int(h_i))
 
 
+def sigma_bound(Y, fraction: float = 0.0015) -> int:
+    """Section 3.2.2, the n-sigma rule: the minimal value among the largest ``fraction`` of the
+    feature map Y (0.15 % for three sigma), never below 1 (a BReLU bound is positive)."""
+    flat = np.sort(np.asarray(Y).reshape(-1))
+    if flat.size == 0:
+        return 1
+    k = max(1, int(np.ceil(flat.size * fraction)))
+    return max(1, int(flat[flat.size - k]))
+
+
 def requant_exact(Y: int, mul: int, shift: int) -> int:
     """Eq. 4 in exact rational arithmetic (used by tests as the definition of the bracket)."""
     return round_half_up(Fraction(Y * mul, 1 << shift))

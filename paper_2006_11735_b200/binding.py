@@ -17,7 +17,7 @@ KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin"
 
 EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_plan_describe", "iconv_forward", "iconv_check",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
-           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iconcat_plan", "iconv_probe_mma_rate",
+           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iq_sigma_bound", "iconcat_plan", "iconv_probe_mma_rate",
            "iconv_stem_forward_static", "iconv_last_error")
 
 
@@ -74,6 +74,7 @@ def _load():
     lib.iq_mul_shift.argtypes = [dbl, i32, P(i32), P(i32)]
     lib.iq_brelu_params.argtypes = [dbl, dbl, i32, i32, P(i32), P(i32), P(i32), P(i32), P(dbl), P(dbl)]
     lib.iq_skip_sync.argtypes = [dbl, dbl, i32, P(i32), P(i32), P(dbl), P(dbl)]
+    lib.iq_sigma_bound.argtypes = [C.c_void_p, C.c_int64, dbl, P(i32), C.c_void_p]
     lib.iconcat_plan.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, P(dbl)]
     lib.iconv_probe_mma_rate.argtypes = [i32, i32, P(dbl), P(dbl)]
     lib.iconv_stem_forward_static.argtypes = [P(istem_desc), vp, vp, vp, vp, vp]
@@ -211,6 +212,13 @@ def iq_skip_sync(ratio_y: float, ratio_s: float, shift_min: int = 8):
     _check(lib.iq_skip_sync(float(ratio_y), float(ratio_s), shift_min, C.byref(m), C.byref(s), C.byref(ry),
                             C.byref(ds)))
     return dict(skip_mul=m.value, skip_shift=s.value, ratio_Y_new=ry.value, delta_scale=ds.value)
+
+
+def iq_sigma_bound(y_ptr, count: int, fraction: float = 0.0015, stream=0) -> int:
+    """The n-sigma bound (Section 3.2.2) of ``count`` int32 values at the device pointer ``y_ptr``."""
+    b = C.c_int32()
+    _check(lib.iq_sigma_bound(y_ptr, int(count), float(fraction), C.byref(b), stream))
+    return b.value
 
 
 def iconcat_plan(ratio_y, ratio_v, shift_min: int = 16):

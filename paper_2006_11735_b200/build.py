@@ -7,7 +7,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libiconv_b200.so")
-SOURCES = ["iconv_api.cu", "plan.cu", "kernels_direct.cu", "kernel_thin.cu", "kernel_umma.cu", "kernel_stem.cu", "probe_mma.cu", "planner.cpp"]
+SOURCES = ["iconv_api.cu", "plan.cu", "kernels_direct.cu", "kernel_thin.cu", "kernel_umma.cu", "kernel_stem.cu", "kernel_calib.cu", "probe_mma.cu", "planner.cpp"]
 
 
 def _stale() -> bool:

@@ -65,6 +65,13 @@ def test_null_arguments():
     assert B.lib.iconv_plan_destroy(None) == B.OK
     assert B.lib.iadd_requant(None, None, None, None, None) == B.ERR_ARG
     assert B.lib.ipool_max(None, None, 1, 8, 8, 15, 3, 2, 1, None) == B.ERR_ALIGN
+    import ctypes
+    b = ctypes.c_int32(-7)
+    assert B.lib.iq_sigma_bound(None, 10, 0.0015, ctypes.byref(b), None) == B.ERR_ARG          # no tensor
+    assert B.lib.iq_sigma_bound(None, 0, 0.0015, None, None) == B.ERR_ARG                      # no place for the result
+    assert B.lib.iq_sigma_bound(None, 0, 0.0, ctypes.byref(b), None) == B.ERR_ARG              # fraction outside (0, 1]
+    assert B.lib.iq_sigma_bound(None, 0, 1.5, ctypes.byref(b), None) == B.ERR_ARG
+    assert B.lib.iq_sigma_bound(None, 0, 0.0015, ctypes.byref(b), None) == B.OK and b.value == 1   # an empty map: no GPU touched
 
 
 def test_weight_quantisation_matches_oracle_planner():

@@ -70,6 +70,30 @@ def test_h_i_always_requantises_to_max_int():
             assert q["h_i"] * q["mul"] + (1 << (q["shift"] - 1)) < 2 ** 63
 
 
+def test_sigma_bound_is_the_kth_largest_value():
+    """Section 3.2.2: the bound is characterised without sorting: at least k values reach it,
+    fewer than k exceed it (k = the size of the largest 0.15 %), and it is never below 1."""
+    rng = np.random.default_rng(11)
+    for size, frac in [(1, 0.0015), (7, 0.0015), (1000, 0.0015), (4001, 0.0015), (50000, 0.00023), (300, 0.5), (64, 1.0)]:
+        for scale in (3.0, 40000.0):
+            Y = np.floor(rng.normal(0, scale, size=size) + 0.5).astype(np.int32)
+            b = P.sigma_bound(Y, frac)
+            k = max(1, int(np.ceil(size * frac)))
+            exact = sorted(Y.tolist(), reverse=True)[k - 1]
+            assert b == max(1, exact)
+            if exact >= 1:
+                assert (Y >= b).sum() >= k and (Y > b).sum() < k
+    assert P.sigma_bound(np.array([5, 5, 5, 5], dtype=np.int32), 0.5) == 5
+    assert P.sigma_bound(np.array([-9, -3], dtype=np.int32)) == 1
+    assert P.sigma_bound(np.zeros(0, dtype=np.int32)) == 1
+    # three sigma of a wide normal sample sits near 2.97 standard deviations (the 99.85th percentile)
+    Y = np.floor(np.random.default_rng(5).normal(0, 10000.0, size=2_000_000) + 0.5).astype(np.int32)
+    assert 2.9 * 10000 < P.sigma_bound(Y) < 3.05 * 10000
+    # and it is the rule the calibration of the networks uses
+    from oracle import networks as ON
+    assert ON._three_sigma_bound(Y) == P.sigma_bound(Y, 0.0015)
+
+
 def test_concat_sync_algorithm_2():
     ry, rv = [30000.0, 52000.0, 41000.0], [90.0, 61.5, 75.25]
     s = P.concat_sync(ry, rv)
