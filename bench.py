@@ -34,6 +34,7 @@ WORKLOAD = "resnet50_b256_224x224x3"
 # the other full-size configurations can be timed the same way (--workload); the default and the
 # metric of record is the ResNet-50 one
 WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"),
+             "resnet18": ("ResNet-18 int8 images/sec", "resnet18_b256_224x224x3"),
              "resnet152": ("ResNet-152 int8 images/sec", "resnet152_b128_224x224x3"),
              "vdsr": ("VDSR int8 images/sec", "vdsr_16x256x256x1"),
              "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1"),

@@ -15,7 +15,7 @@ from workloads import networks as N
 from . import networks as ON
 
 OUT_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "params")
-CONFIGS = ("single_conv", "vdsr", "vrcnn", "resnet50", "resnet152")
+CONFIGS = ("single_conv", "vdsr", "vrcnn", "resnet18", "resnet50", "resnet152")
 
 
 def write(name: str) -> str:

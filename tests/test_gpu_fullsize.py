@@ -17,7 +17,7 @@ from workloads import networks as N
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["vdsr", "vrcnn", "resnet50", "resnet152"])
+@pytest.mark.parametrize("name", ["vdsr", "vrcnn", "resnet18", "resnet50", "resnet152"])
 def test_full_size_configuration_matches_oracle_on_sampled_images(name):
     net = N.by_name(name)
     params = load_params(name)

@@ -175,6 +175,7 @@ def _ratio_of(net, params, name):
     N.vdsr(n=2, h=24, w=20, depth=6),
     N.vrcnn(n=2, h=24, w=28),
     N.resnet(2, (2, 1), h=48, w=40, widths=(16, 32), classes=10, seed=4),
+    N.resnet_basic(2, (2, 1), h=48, w=40, widths=(16, 32), classes=10, seed=6),
 ], ids=lambda n: n.name)
 def test_integer_network_tracks_its_float_shadow_and_is_not_vacuous(net):
     params = ON.calibrate(net)

@@ -175,6 +175,54 @@ def resnet(n, blocks, h=224, w=224, widths=(64, 128, 256, 512), classes=1000, se
     return net
 
 
+def resnet_basic(n, blocks, h=224, w=224, widths=(64, 128, 256, 512), classes=1000, seed=6,
+                 name="resnet_basic") -> Net:
+    """Basic-block ResNet (the paper's Figure 3): 7x7/2 stem, 3x3/2 max-pool, stages of blocks
+    of two 3x3 convolutions, the second one closing the block with the skip: the block input
+    itself (type 1) or, where the block strides or widens, its 1x1 projection (type 2)."""
+    net = Net(name, seed, n, "x0", "logits")
+    net.add_tensor("x0", h, w, 3)
+    layer = 0
+    hh, ww = _out(h, 7, 2, 3), _out(w, 7, 2, 3)
+    net.add_tensor("stem", hh, ww, widths[0])
+    net.ops.append(Conv("stem", layer, "x0", "stem", 3, widths[0], 7, 2, 3, in_dtype="u8_raw128"))
+    layer += 1
+    hh, ww = _out(hh, 3, 2, 1), _out(ww, 3, 2, 1)
+    net.add_tensor("pool", hh, ww, widths[0])
+    net.ops.append(MaxPool("maxpool", "stem", "pool"))
+    prev, c_prev = "pool", widths[0]
+    for si, (nb, width) in enumerate(zip(blocks, widths)):
+        for b in range(nb):
+            s = 2 if (b == 0 and si > 0) else 1
+            tag = "s%db%d" % (si + 1, b)
+            h2, w2 = _out(hh, 3, s, 1), _out(ww, 3, s, 1)
+            ta = net.add_tensor(tag + "_a", h2, w2, width)
+            net.ops.append(Conv(tag + "_3x3a", layer, prev, ta, c_prev, width, 3, s, 1))
+            layer += 1
+            if s != 1 or c_prev != width:
+                tp = net.add_tensor(tag + "_p", h2, w2, width, "i32")
+                net.ops.append(Conv(tag + "_proj", layer, prev, tp, c_prev, width, 1, s, 0, role="raw"))
+                layer += 1
+                skip, skip_dtype = tp, "i32"
+            else:
+                skip, skip_dtype = prev, "u8"
+            tc = net.add_tensor(tag + "_c", h2, w2, width)
+            net.ops.append(Conv(tag + "_3x3b", layer, ta, tc, width, width, 3, 1, 1,
+                                skip=skip, skip_dtype=skip_dtype))
+            layer += 1
+            prev, c_prev, hh, ww = tc, width, h2, w2
+    net.add_tensor("avg", 1, 1, c_prev)
+    net.ops.append(AvgPool("avgpool", prev, "avg"))
+    net.add_tensor("logits", 1, 1, classes, "i32")
+    net.ops.append(Conv("fc", layer, "avg", "logits", c_prev, classes, 1, role="raw"))
+    return net
+
+
+def resnet18(n=256, h=224, w=224, seed=6) -> Net:
+    """The paper's second classification network (Tables 1 and 2), basic blocks (2, 2, 2, 2)."""
+    return resnet_basic(n, (2, 2, 2, 2), h, w, seed=seed, name="resnet18")
+
+
 def resnet50(n=256, h=224, w=224, seed=4) -> Net:
     """Configuration 4."""
     return resnet(n, (3, 4, 6, 3), h, w, seed=seed, name="resnet50")
@@ -193,4 +241,4 @@ def vrcnn_hd(n=1, h=1600, w=2560, seed=3) -> Net:
 
 def by_name(name: str, **kw) -> Net:
     return {"single_conv": single_conv, "vdsr": vdsr, "vrcnn": vrcnn, "vrcnn_hd": vrcnn_hd,
-            "resnet50": resnet50, "resnet152": resnet152}[name](**kw)
+            "resnet18": resnet18, "resnet50": resnet50, "resnet152": resnet152}[name](**kw)
