@@ -913,9 +913,10 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 // store per pixel.  NG: the number of groups when known at compile time (0: `ngroups`).
 // GU: per-channel parameters that are uniform per group (fetched group by group).
 template <int EPI, int NG, bool GU>
-__device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, uint8_t *ocol, bool valid, int col_lo, int ngroups,
-                                              int *accA, int *accB, const EpiScalars &es, const ConvArgs &a, const UmmaArgs &u)
+__device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, uint8_t *ocol, const uint8_t *scol, bool valid, int col_lo,
+                                              int ngroups, int *accA, int *accB, const EpiScalars &es, const ConvArgs &a, const UmmaArgs &u)
 {
+    constexpr bool SKIP8 = (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8);    // scol: this pixel's 8-bit skip row, read directly
     const int ng = NG ? NG : ngroups;
 #pragma unroll
     for (int gi = 0; gi < (NG ? NG : 16); gi += 2) {
@@ -928,13 +929,15 @@ __device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, u
             int4 ca[4];
 #pragma unroll
             for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + 4 * gcur + g);
+            uint4 sk = make_uint4(0, 0, 0, 0);
+            if (SKIP8 && valid && co0 < a.c_out) sk = __ldg((const uint4 *)(scol + (gcur << 4)));
             tmem_ld_wait();
             if (gcur + 1 < ng) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
             int V[16];
-            if (GU) epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), group_scalars(es, u, co0), a, u);
-            else epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, make_uint4(0, 0, 0, 0), es, a, u);
+            if (GU) epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, sk, group_scalars(es, u, co0), a, u);
+            else epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, sk, es, a, u);
             uint4 o;
-            if (EPI == EPI_FAST || a.out_dtype == ICONV_U8) {
+            if (EPI == EPI_FAST || EPI == EPI_FAST_SKIP8 || a.out_dtype == ICONV_U8) {
                 o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
                 o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
             } else {
@@ -1172,13 +1175,16 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             if (EPI != EPI_NARROW) {
                 const int4 *cap = (const int4 *)(u.c_a + col_lo);
                 uint8_t *ocol = orow + col_lo;
+                const uint8_t *scol = nullptr;
+                if (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8)
+                    scol = (const uint8_t *)a.skip + (((long long)img * a.h_out + y) * a.w_out + xq) * a.skip_c_total + a.skip_c_offset + col_lo;
                 // the usual widths get straight-line code: every offset an immediate, no loop control
-                if (es.group_uniform) window_groups<EPI, 0, true>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 4) window_groups<EPI, 4, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 3) window_groups<EPI, 3, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 2) window_groups<EPI, 2, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 1) window_groups<EPI, 1, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else window_groups<EPI, 0, false>(t_row, cap, ocol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                if (es.group_uniform) window_groups<EPI, 0, true>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 4) window_groups<EPI, 4, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 3) window_groups<EPI, 3, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 2) window_groups<EPI, 2, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else if (ngroups == 1) window_groups<EPI, 1, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                else window_groups<EPI, 0, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
             }
             tc_fence_before();
             __syncwarp();
@@ -1502,6 +1508,12 @@ int umma_init_once()
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE_SKIP8, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE_SKIP8, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE_SKIP8, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         attr_set = true;
     }
@@ -1626,9 +1638,10 @@ void window_plan(iconv_plan_t *p)
     const iconv_desc &d = p->d;
     p->window = 0;
     if (d.kernel == ICONV_KERNEL_UMMA_IM2COL) return;
-    if (d.stride != 1 || d.proj_weights || (d.skip_dtype >= 0 && p->epi != EPI_NARROW) || d.out_dtype == ICONV_I32) return;
+    const bool skip8_epi = p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8;      // the epilogue reads the skip rows itself
+    if (d.stride != 1 || d.proj_weights || (d.skip_dtype >= 0 && p->epi != EPI_NARROW && !skip8_epi) || d.out_dtype == ICONV_I32) return;
     if (p->c_in_pad != p->kc || p->c_out_pad != p->block_n) return;
-    if (p->epi != EPI_FAST && p->epi != EPI_SAFE && p->epi != EPI_NARROW) return;
+    if (p->epi != EPI_FAST && p->epi != EPI_SAFE && p->epi != EPI_NARROW && !skip8_epi) return;
     const int taps = plan_taps(p);
     const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
     const long long bank = (long long)b_tile * taps;
@@ -1920,6 +1933,17 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         else if (p->epi == EPI_NARROW) {
             if (d.kh == 3 && d.kw == 3 && kj == 2) umma_window_kernel<EPI_NARROW, 3, 3, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
             else umma_window_kernel<EPI_NARROW, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);
+        }
+        else if (p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8) {
+#define ICONV_WINS(E)                                                                                                               \
+    do {                                                                                                                            \
+        if (d.kh == 3 && d.kw == 3 && kj == 2) umma_window_kernel<E, 3, 3, 2><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);      \
+        else if (d.kh == 3 && d.kw == 3 && kj == 4) umma_window_kernel<E, 3, 3, 4><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u); \
+        else umma_window_kernel<E, 0, 0, 0><<<wgrid, NUM_THREADS, wsmem, stream>>>(tmap_x, p->tmap_w, a, u);                        \
+    } while (0)
+            if (p->epi == EPI_FAST_SKIP8) ICONV_WINS(EPI_FAST_SKIP8);
+            else ICONV_WINS(EPI_SAFE_SKIP8);
+#undef ICONV_WINS
         }
         else ICONV_WIN(EPI_SAFE);
 #undef ICONV_WIN

@@ -473,3 +473,39 @@ def test_activation_bit_depth_sweep_matches_oracle(max_int, kernel):
         got, fam = gpu_conv(X, W, b, mul, shift, h_i, kernel=kernel, **kw)
         assert np.array_equal(got, want)
         assert want.max() == max_int and (want == 0).mean() > 0.02 and ((want > 0) & (want < max_int)).mean() > 0.2
+
+
+WINDOW_SKIP_SHAPES = [
+    # stride-1 layers with an 8-bit identity skip (the closing 3x3 of a basic block): n, h, w, c, k, pad
+    (2, 28, 28, 64, 3, 1),              # block tiling, 64-byte rows
+    (1, 37, 150, 64, 3, 1),             # ragged blocks
+    (3, 14, 14, 128, 3, 1),             # 128-byte rows, tiles across rows
+    (2, 20, 24, 64, 1, 0),              # a 1x1 with a skip
+    (1, 6, 260, 32, 5, 2),              # strips, another filter size (the generic issue path)
+]
+
+
+@pytest.mark.parametrize("shape", WINDOW_SKIP_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("skip_dtype", [B.U8, B.U8_RAW128, B.S8], ids=["u8", "raw128", "s8"])
+@pytest.mark.parametrize("variant", ["fast", "safe"])
+def test_window_mode_with_identity_skip_matches_oracle(shape, skip_dtype, variant):
+    n, h, w, c, k, pad = shape
+    X, W, b, mul, shift, h_i = _layer(sum(shape) + 11, n, h, w, c, c, k)
+    ho, wo = h + 2 * pad - k + 1, w + 2 * pad - k + 1
+    rng = np.random.default_rng(sum(shape))
+    S = rng.integers(0, 256, size=(n, ho, wo, c + 16), dtype=np.uint8)
+    if skip_dtype == B.S8:
+        S = S.view(np.int8)
+    kw = dict(pad=pad, skip=S, skip_dtype=skip_dtype, skip_c_offset=16, skip_mul=int(h_i[0]) // 200, skip_shift=2)
+    if variant == "safe":               # a zero point and a narrower range: the explicit-clamp epilogue
+        kw.update(out_zero=3, out_lo=3, out_hi=200)
+    h_i = h_i * 2
+    want = oracle_conv(X, W, b, mul, shift, h_i, **kw)
+    assert 0.02 < (want == want.min()).mean() < 0.98 and np.unique(want).size > 16
+    for kernel in (B.KERNEL_UMMA, B.KERNEL_UMMA_IM2COL):
+        text = []
+        got, fam = gpu_conv(X, W, b, mul, shift, h_i, kernel=kernel, describe=text, **kw)
+        assert fam == B.KERNEL_UMMA and ("window" in text[0]) == (kernel == B.KERNEL_UMMA), text
+        bad = np.argwhere(got != want)
+        assert bad.shape[0] == 0, "%s: %d mismatches, first at %s: got %s want %s" % (
+            text[0], bad.shape[0], bad[0], got[tuple(bad[0])], want[tuple(bad[0])])
