@@ -1642,6 +1642,12 @@ void window_plan(iconv_plan_t *p)
     if (d.stride != 1 || d.proj_weights || (d.skip_dtype >= 0 && p->epi != EPI_NARROW && !skip8_epi) || d.out_dtype == ICONV_I32) return;
     if (p->c_in_pad != p->kc || p->c_out_pad != p->block_n) return;
     if (p->epi != EPI_FAST && p->epi != EPI_SAFE && p->epi != EPI_NARROW && !skip8_epi) return;
+    // Window mode stores 16 bytes per pixel and group straight from registers; the im2col kernel
+    // stages whole rows and stores them by TMA, which wins once a pixel's output is wide: a 1x1
+    // layer (no halo to save) stays there beyond 64 columns, a layer with a skip beyond 128
+    // (measured: 64 -> 256 1x1 with skip 0.134 ms by im2col, 0.217 ms in window mode).
+    if (d.kh * d.kw == 1 && p->block_n > 64 && p->epi != EPI_NARROW) return;
+    if (skip8_epi && p->block_n > 128) return;
     const int taps = plan_taps(p);
     const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
     const long long bank = (long long)b_tile * taps;
