@@ -44,3 +44,9 @@ def test_every_layer_of_small_networks_matches_oracle(net, kernel, fuse):
         assert np.array_equal(got, want[op.dst]), "%s: %d mismatches" % (op.name, (got != want[op.dst]).sum())
     assert np.array_equal(out.cpu().numpy(), want[net.output])
     g.close()
+
+
+def test_smoke_entry_point_runs():
+    """The smoke entry point (one small invocation checked against the oracle) stays runnable."""
+    import __graft_entry__
+    __graft_entry__.smoke()
