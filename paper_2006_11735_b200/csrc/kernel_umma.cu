@@ -44,7 +44,8 @@ constexpr int MMA_WARP = NUM_PRODUCERS;
 constexpr int MMA_WARP2 = 1;           // window mode (one TMA warp): a second MMA issuer
 constexpr int EPI_WARP0 = 4;              // first epilogue warp (a multiple of 4: warp % 4 is its TMEM lane quadrant)
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS_MAX);
-constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces (+ the skip rows of one tile)
+constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces of up to 4 KB together, then the skip rows of one tile
+constexpr int EPI_WARP_SMEM_SMALL = 4096; // ... when the output is 8-bit (pieces of 2 KB) and no 8-bit skip is staged
 constexpr int MAX_STAGES = 12;
 constexpr int MAX_TMEM_BUFS = 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds at the boost clock
@@ -79,6 +80,7 @@ struct UmmaArgs {
     int epi_warps, cs, bi;          // epilogue warps, column split per tile, tiles in flight
     int part_n;                     // columns one epilogue warp handles per tile
     int piece_bytes;                // row width of one staged output piece (16 ... 128 bytes)
+    int epi_warp_bytes;             // staging memory per epilogue warp
     unsigned idesc, idesc_p;        // instruction descriptors of the layer and of the projection (operand signedness)
     unsigned long long desc_hi;     // upper 32 bits of the shared-memory matrix descriptors
     // per-layer epilogue scalars (per-channel layers read the arrays instead)
@@ -742,7 +744,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int turn = slot / u.cs;
         const int col_lo = part * u.part_n;
         const int ncols = min(u.block_n - col_lo, u.part_n);
-        uint8_t *obuf = epi_smem + (size_t)ew * EPI_WARP_SMEM;        // two pieces of 32 rows x piece_bytes
+        uint8_t *obuf = epi_smem + (size_t)ew * u.epi_warp_bytes;     // two pieces of 32 rows x piece_bytes
         uint8_t *sbuf = obuf + EPI_WARP_SMEM / 2;                     // skip rows of one tile (8-bit variants)
         const uint32_t skip_bar = smem_u32(&sh->skip_full[ew]);
         constexpr int esz = (EPI == EPI_RAW) ? 4 : 1;
@@ -1582,8 +1584,12 @@ int umma_geometry(iconv_plan_t *p)
     p->epi_warps = 0;
     p->kg = 1;
     const int weight = p->block_n * (proj ? 7 : (d.skip_dtype >= 0 ? 5 : 2)) / (2 * k_iters);
+    // staging per epilogue warp: 8-bit pieces are 2 KB each, and only an 8-bit skip (not a fused
+    // projection's operand) is staged behind them
+    const bool stage_skip = d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && !proj;
+    p->epi_warp_bytes = (d.out_dtype == ICONV_I32 || stage_skip) ? EPI_WARP_SMEM : EPI_WARP_SMEM_SMALL;
     for (int ew = (weight >= 100 ? 16 : 8); ew >= 8 && !p->epi_warps; ew -= 8) {
-        const int avail = MAX_SMEM - fixed - ew * EPI_WARP_SMEM;
+        const int avail = MAX_SMEM - fixed - ew * p->epi_warp_bytes;
         const int want = 2;
         int room = 0, slot = 0;
         if (bank <= RESIDENT_B_MAX && avail - (int)bank >= want * stage_a) {
@@ -1866,6 +1872,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.bi = p->bi;
     u.part_n = p->half_n;
     u.piece_bytes = p->piece_bytes;
+    u.epi_warp_bytes = p->epi_warp_bytes;
     // instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, N/8, M/16
     u.idesc = (2u << 4) | ((d.in_dtype == ICONV_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(p->block_n >> 3) << 17) |
               ((unsigned)(BLOCK_M >> 4) << 24);
@@ -1960,7 +1967,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     const size_t smem = 1024 + (size_t)u.stages * u.stage_bytes +
                         (p->resident_b ? (size_t)u.b_tile_bytes * (u.p_iters + u.taps * u.cchunks) * u.n_tiles : 0) + sizeof(Shared) + 1024 +
-                        (size_t)p->epi_warps * EPI_WARP_SMEM;
+                        (size_t)p->epi_warps * p->epi_warp_bytes;
     if (smem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
 #define ICONV_LAUNCH(E) umma_conv_kernel<E><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u)
     switch (p->epi) {

@@ -31,6 +31,7 @@ struct iconv_plan_s {
     int epi_warps = 8, cs = 1, bi = 1;   // epilogue warps; column split per tile; tiles in flight
     int tail = 1;            // 0: zero point and output range are provably no-ops
     int q_mul = 1, q_shift = 0, q_h = 0; // per-layer Eq. 4 / BReLU scalars
+    int epi_warp_bytes = 8192;           // staging memory per epilogue warp (im2col kernel)
     int group_uniform = 0;               // per-channel parameters equal within every 16-channel group
     int pair16 = 0;                      // internal (stem): 16-channel positions read in pairs, two taps per K step
     // stem path: repacked image (plan-owned scratch) and the plan of the GEMM that follows
