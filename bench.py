@@ -304,7 +304,9 @@ def main():
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
                 "config": {"workload": workload, "global_batch": net.n * size, "parallelism": "dp%d" % size,
-                           "l2": "per-step activation traffic (~7 GB) far exceeds the 126 MB L2",
+                           "l2": "per-step algorithmic traffic (%.1f GB) far exceeds the 126 MB L2" % (sum(abytes.values()) / 1e9),
+                           "timing_note": "the timed region carries one CUDA event per layer (the per-kernel durations of "
+                                          "`roofline`); the end-to-end loop carries none, which is worth 1-2 %",
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
                 "clocks": clocks,
                 "e2e": {"value": total_images / (ms_e2e * 1e-3), "unit": UNIT,
