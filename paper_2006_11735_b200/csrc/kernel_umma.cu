@@ -693,6 +693,8 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, slot_step = (uint32_t)u.slot_bytes >> 4;
             const uint32_t slot_a_step = (uint32_t)u.slot_a_bytes >> 4;
             const uint32_t b_step = (uint32_t)(u.resident_b ? u.b_tile_bytes : u.slot_bytes) >> 4;
+            const bool simple = kj == 4 && u.kg == 1 && !u.resident_b && u.p_iters == 0;
+            const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & (u.nbuf - 1);
                 if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
@@ -705,6 +707,33 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 if (u.resident_b) {
                     const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
                     sb = ((smem_u32(b_res + (size_t)((tile - m_tile * u.n_tiles) * k_iters) * u.b_tile_bytes) & 0x3FFFFu) >> 4) | (1u << 16);
+                }
+                if (simple) {
+                    // The long reductions (one 128-byte k-iteration per stage, B riding in the stage, no
+                    // projection): a round per stage of nothing but the wait, four MMAs and the commit.
+                    // Every taken branch of this lone thread costs tens of cycles that the tensor
+                    // pipe's short queue does not cover, and here there are 8 to 36 rounds per tile.
+                    uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step;
+                    uint32_t full_bar = full0 + 8u * (uint32_t)stage, empty_bar = empty0 + 8u * (uint32_t)stage;
+                    uint32_t acc = 0;
+                    for (int ki = 0; ki < k_iters; ++ki) {
+                        if (!mbar_test_wait(full_bar, parity) && !mbar_wait(full_bar, parity, &sh->abort_flag)) {
+                            give_up(sh, u.status, 3);
+                            ok = false;
+                            break;
+                        }
+                        umma_slot<4>(d_tmem, a_lo, a_lo + slot_a_step, desc_hi32, u.idesc, acc);
+                        acc = 1;
+                        umma_commit(empty_bar);
+                        const bool wrap = ++stage == u.stages;
+                        stage = wrap ? 0 : stage;
+                        parity ^= wrap ? 1u : 0u;
+                        a_lo = wrap ? a_lo0 : a_lo + stage_step;
+                        full_bar = wrap ? full0 : full_bar + 8u;
+                        empty_bar = wrap ? empty0 : empty_bar + 8u;
+                    }
+                    if (ok) umma_commit(smem_u32(&sh->tmem_full[buf]));
+                    continue;
                 }
                 for (int ki = 0; ki < k_iters;) {
                     if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
