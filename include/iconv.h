@@ -217,6 +217,18 @@ ICONV_API int iconv_stem_forward_static(const istem_desc *desc, const void *x, c
 
 /* Eq. 2: delta = max|W_f| / 127. */
 ICONV_API int iq_weight_delta(const float *w_f, int64_t count, double *delta);
+/* Section 3.4.3: a batch-normalisation layer merged into the convolution before it, with one
+ * quantisation step per output channel.  g = gamma / sqrt(var + eps); w_out[co][i] = w_f[co][i] * g[co];
+ * b_out[co] = (b_f[co] - mean[co]) * g[co] + beta[co] (b_f may be NULL: no bias);
+ * delta[co] = max_i |w_out[co][i]| / 127 (Eq. 2 per channel; 0 when the channel's weights all
+ * vanish: such a channel can be pruned).  Everything in double.  All pointers HOST; w_f is
+ * [c_out][k], the per-channel arrays have c_out entries; w_out [c_out][k], b_out and delta [c_out]
+ * are written.  The per-channel steps give per-channel ratios, which `iconcat_plan` (Algorithm 2,
+ * one branch per channel) brings to a common output ratio: its mul / shift arrays are the
+ * per-channel parameters `iconv_plan` accepts.  Errors: ICONV_ERR_ARG (null pointer, c_out < 1,
+ * k < 1, var + eps <= 0). */
+ICONV_API int iq_bn_fold(const float *w_f, const float *b_f, const float *gamma, const float *beta, const float *mean,
+               const float *var, double eps, int32_t c_out, int64_t k, double *w_out, double *b_out, double *delta);
 /* Eq. 1: w_i = clamp([w_f / delta], -127, 127), computed in double. */
 ICONV_API int iq_quantize_weights(const float *w_f, int64_t count, double delta, int8_t *w_i);
 /* The mul_shift() named by Eq. 9: the smallest shift in [shift_min, 40] whose

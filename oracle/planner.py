@@ -70,6 +70,22 @@ def brelu_params_from_h_ri(h_ri: int, ratio_Y: float, max_int: int, shift_min: i
     return dict(h_ri=int(h_ri), mul=mul, shift=shift, ratio_V=ratio_V, h_f=h_f, h_i=int(h_i))
 
 
+def bn_fold(W_f, b_f, gamma, beta, mean, var, eps: float):
+    """Section 3.4.3: a batch-normalisation layer merged into the convolution before it, one
+    quantisation step per output channel.  With g = gamma / sqrt(var + eps) (per channel):
+    W'[co] = W[co] * g[co], b'[co] = (b[co] - mean[co]) * g[co] + beta[co], delta[co] = max|W'[co]| / 127
+    (Eq. 2 channel by channel; 0 for a channel whose weights all vanish, which can be pruned).
+    Returns (W', b', delta) in float64; W_f is [c_out][...]."""
+    W = np.asarray(W_f, dtype=np.float64)
+    c_out = W.shape[0]
+    b = np.zeros(c_out) if b_f is None else np.asarray(b_f, dtype=np.float64)
+    g = np.asarray(gamma, dtype=np.float64) / np.sqrt(np.asarray(var, dtype=np.float64) + float(eps))
+    Wp = W * g.reshape((c_out,) + (1,) * (W.ndim - 1))
+    bp = (b - np.asarray(mean, dtype=np.float64)) * g + np.asarray(beta, dtype=np.float64)
+    delta = np.max(np.abs(Wp.reshape(c_out, -1)), axis=1) / 127.0
+    return Wp, bp, delta
+
+
 def sigma_bound(Y, fraction: float = 0.0015) -> int:
     """Section 3.2.2, the n-sigma rule: the minimal value among the largest ``fraction`` of the
     feature map Y (0.15 % for three sigma), never below 1 (a BReLU bound is positive)."""

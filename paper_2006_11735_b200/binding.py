@@ -17,7 +17,7 @@ KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin"
 
 EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_plan_describe", "iconv_forward", "iconv_check",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
-           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iq_sigma_bound", "iconcat_plan", "iconv_probe_mma_rate",
+           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iq_sigma_bound", "iq_bn_fold", "iconcat_plan", "iconv_probe_mma_rate",
            "iconv_stem_forward_static", "iconv_last_error")
 
 
@@ -75,6 +75,7 @@ def _load():
     lib.iq_brelu_params.argtypes = [dbl, dbl, i32, i32, P(i32), P(i32), P(i32), P(i32), P(dbl), P(dbl)]
     lib.iq_skip_sync.argtypes = [dbl, dbl, i32, P(i32), P(i32), P(dbl), P(dbl)]
     lib.iq_sigma_bound.argtypes = [C.c_void_p, C.c_int64, dbl, P(i32), C.c_void_p]
+    lib.iq_bn_fold.argtypes = [vp, vp, vp, vp, vp, vp, dbl, i32, i64, vp, vp, vp]
     lib.iconcat_plan.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, P(dbl)]
     lib.iconv_probe_mma_rate.argtypes = [i32, i32, P(dbl), P(dbl)]
     lib.iconv_stem_forward_static.argtypes = [P(istem_desc), vp, vp, vp, vp, vp]
@@ -212,6 +213,21 @@ def iq_skip_sync(ratio_y: float, ratio_s: float, shift_min: int = 8):
     _check(lib.iq_skip_sync(float(ratio_y), float(ratio_s), shift_min, C.byref(m), C.byref(s), C.byref(ry),
                             C.byref(ds)))
     return dict(skip_mul=m.value, skip_shift=s.value, ratio_Y_new=ry.value, delta_scale=ds.value)
+
+
+def iq_bn_fold(w_f, b_f, gamma, beta, mean, var, eps: float):
+    """Batch normalisation merged into the convolution before it; returns (W', b', delta per channel)."""
+    w_f = np.ascontiguousarray(w_f, dtype=np.float32)
+    c_out = w_f.shape[0]
+    k = w_f.size // c_out
+    f32 = lambda a: None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+    b_f, gamma, beta, mean, var = f32(b_f), f32(gamma), f32(beta), f32(mean), f32(var)
+    w_out = np.empty(w_f.shape, dtype=np.float64)
+    b_out, delta = np.empty(c_out, dtype=np.float64), np.empty(c_out, dtype=np.float64)
+    _check(lib.iq_bn_fold(w_f.ctypes.data, None if b_f is None else b_f.ctypes.data, gamma.ctypes.data, beta.ctypes.data,
+                          mean.ctypes.data, var.ctypes.data, float(eps), c_out, k, w_out.ctypes.data, b_out.ctypes.data,
+                          delta.ctypes.data))
+    return w_out, b_out, delta
 
 
 def iq_sigma_bound(y_ptr, count: int, fraction: float = 0.0015, stream=0) -> int:

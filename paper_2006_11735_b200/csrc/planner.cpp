@@ -41,6 +41,30 @@ extern "C" int iq_weight_delta(const float *w_f, int64_t count, double *delta)
     return ICONV_OK;
 }
 
+extern "C" int iq_bn_fold(const float *w_f, const float *b_f, const float *gamma, const float *beta, const float *mean,
+                          const float *var, double eps, int32_t c_out, int64_t k, double *w_out, double *b_out, double *delta)
+{
+    if (!w_f || !gamma || !beta || !mean || !var || !w_out || !b_out || !delta || c_out < 1 || k < 1 || !(eps >= 0.0)) {
+        set_error("iq_bn_fold: bad argument");
+        return ICONV_ERR_ARG;
+    }
+    for (int32_t co = 0; co < c_out; ++co) {
+        const double s = (double)var[co] + eps;
+        if (!(s > 0.0)) { set_error("iq_bn_fold: var + eps must be positive (channel %d)", (int)co); return ICONV_ERR_ARG; }
+        const double g = (double)gamma[co] / std::sqrt(s);
+        double m = 0.0;
+        for (int64_t i = 0; i < k; ++i) {
+            const double w = (double)w_f[(int64_t)co * k + i] * g;
+            w_out[(int64_t)co * k + i] = w;
+            const double a = std::fabs(w);
+            if (a > m) m = a;
+        }
+        b_out[co] = ((b_f ? (double)b_f[co] : 0.0) - (double)mean[co]) * g + (double)beta[co];
+        delta[co] = m / 127.0;
+    }
+    return ICONV_OK;
+}
+
 extern "C" int iq_quantize_weights(const float *w_f, int64_t count, double delta, int8_t *w_i)
 {
     if (!w_f || !w_i || count < 0 || !(delta > 0.0)) { set_error("iq_quantize_weights: bad argument"); return ICONV_ERR_ARG; }

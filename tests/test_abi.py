@@ -106,6 +106,26 @@ def test_mul_shift_and_brelu_params_match_oracle_planner():
             assert got["ratio_V"] == want["ratio_V"] and got["h_f"] == want["h_f"]
 
 
+def test_bn_fold_matches_oracle_planner():
+    rng = np.random.default_rng(4)
+    c_out = 9
+    W = rng.normal(0, 0.1, size=(c_out, 3, 3, 5)).astype(np.float32)
+    b = rng.normal(0, 0.05, size=c_out).astype(np.float32)
+    gamma, beta = rng.uniform(0.2, 2.0, size=c_out).astype(np.float32), rng.normal(0, 0.3, size=c_out).astype(np.float32)
+    mean, var = rng.normal(0, 0.2, size=c_out).astype(np.float32), rng.uniform(0.05, 3.0, size=c_out).astype(np.float32)
+    gamma[4] = 0.0
+    for bias in (b, None):
+        got = B.iq_bn_fold(W, bias, gamma, beta, mean, var, 1e-5)
+        want = P.bn_fold(W, bias, gamma, beta, mean, var, 1e-5)
+        for g, w in zip(got, want):
+            assert np.array_equal(g, w)
+    assert got[2][4] == 0.0
+    import ctypes
+    assert B.lib.iq_bn_fold(None, None, None, None, None, None, 1e-5, 1, 1, None, None, None) == B.ERR_ARG
+    with pytest.raises(B.IconvError):
+        B.iq_bn_fold(W, b, gamma, beta, mean, -var, 0.0)          # var + eps <= 0
+
+
 def test_skip_sync_and_concat_plan_match_oracle_planner():
     rng = np.random.default_rng(2)
     for _ in range(200):

@@ -61,3 +61,48 @@ def test_sigma_bound_calibrates_a_layer_like_the_oracle():
     h_ri = _bound(Yg.astype(np.int32), 0.0015)
     assert h_ri == P.sigma_bound(Yo)
     assert B.iq_brelu_params(float(h_ri), 1.0, 255) == {k: v for k, v in P.brelu_params(float(h_ri), 1.0, 255).items()}
+
+
+def test_batch_norm_folded_per_channel_layer_end_to_end():
+    """A float convolution + batch normalisation + ReLU-like clamp becomes an integer layer with
+    one quantisation step per output channel (Section 3.4.3) and per-channel mul / shift / h_i
+    from Algorithm 2 with every channel a branch; the GPU equals the oracle bit for bit and the
+    dequantised result tracks the float layer."""
+    from gpu_util import gpu_conv, oracle_conv
+    rng = np.random.default_rng(33)
+    n, h, w, c_in, c_out, k, max_int, h_rf = 2, 20, 24, 32, 48, 3, 255, 4.0
+    x_f = rng.uniform(0.0, 1.0, size=(n, h, w, c_in))
+    ratio_X = 255.0
+    X = np.floor(x_f * ratio_X + 0.5).astype(np.uint8)
+    W_f = rng.normal(0, 0.08, size=(c_out, k, k, c_in)).astype(np.float32)
+    gamma = rng.uniform(0.05, 3.0, size=c_out).astype(np.float32)          # steps differing 60-fold between channels
+    beta = rng.normal(0, 0.2, size=c_out).astype(np.float32)
+    mean = rng.normal(0, 0.3, size=c_out).astype(np.float32)
+    var = rng.uniform(0.2, 2.0, size=c_out).astype(np.float32)
+    Wp, bp, delta = B.iq_bn_fold(W_f, None, gamma, beta, mean, var, 1e-5)
+    assert delta.max() / delta.min() > 10
+    ratio_Y = [ratio_X / d for d in delta]
+    ratio_V = [P.brelu_params(h_rf, ry, max_int)["ratio_V"] for ry in ratio_Y]
+    sync = P.concat_sync(ratio_Y, ratio_V)                                   # Algorithm 2, one branch per channel
+    got_plan = B.iconcat_plan(ratio_Y, ratio_V)
+    assert list(got_plan["mul"]) == list(sync["mul"]) and list(got_plan["shift"]) == list(sync["shift"])
+    Wq = np.stack([P.quantize_weights(Wp[c], delta[c] * sync["delta_scale"][c]) for c in range(c_out)])
+    b_i = np.array([P.round_half_up(bp[c] * sync["ratio_Y_new"][c]) for c in range(c_out)], dtype=np.int32)
+    mul = np.array(sync["mul"], dtype=np.int32)
+    shift = np.array(sync["shift"], dtype=np.int32)
+    h_i = np.array([P.round_half_up(P.Fraction(max_int * (1 << int(s)), int(m))) for m, s in zip(mul, shift)], dtype=np.int32)
+    want = oracle_conv(X, Wq, b_i, mul, shift, h_i, pad=1)
+    for kernel in (B.KERNEL_AUTO, B.KERNEL_UMMA_IM2COL, B.KERNEL_DIRECT):
+        got, _ = gpu_conv(X, Wq, b_i, mul, shift, h_i, pad=1, kernel=kernel)
+        assert np.array_equal(got, want)
+    # the float layer: convolution, batch normalisation, clamp to [0, h_f]
+    xp = np.pad(x_f, ((0, 0), (1, 1), (1, 1), (0, 0)))
+    y = np.zeros((n, h, w, c_out))
+    for r in range(k):
+        for s in range(k):
+            y += xp[:, r:r + h, s:s + w, :] @ W_f[:, r, s, :].astype(np.float64).T
+    y = (y - mean) / np.sqrt(var.astype(np.float64) + 1e-5) * gamma + beta
+    h_f = max_int / sync["ratio_V_min"]
+    y = np.clip(y, 0.0, h_f)
+    err = np.abs(want.astype(np.float64) / sync["ratio_V_min"] - y)
+    assert err.mean() < 0.02 * h_f and (want > 0).mean() > 0.2 and (want == max_int).mean() < 0.5

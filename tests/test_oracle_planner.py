@@ -94,6 +94,31 @@ def test_sigma_bound_is_the_kth_largest_value():
     assert ON._three_sigma_bound(Y) == P.sigma_bound(Y, 0.0015)
 
 
+def test_bn_fold_equals_batch_norm_after_the_convolution():
+    """Section 3.4.3: the merged layer computes what convolution followed by batch normalisation
+    computes (checked on data, in float64, against the two operations written apart), and each
+    channel's step maps that channel's largest merged weight to 127."""
+    rng = np.random.default_rng(21)
+    c_out, k, c_in, eps = 6, 3, 4, 1e-5
+    W = rng.normal(0, 0.1, size=(c_out, k, k, c_in))
+    b = rng.normal(0, 0.05, size=c_out)
+    gamma, beta = rng.uniform(0.2, 2.0, size=c_out), rng.normal(0, 0.3, size=c_out)
+    mean, var = rng.normal(0, 0.2, size=c_out), rng.uniform(0.05, 3.0, size=c_out)
+    gamma[2] = 0.0                                            # a dead channel
+    x = rng.normal(0, 1.0, size=(5, k * k * c_in))            # five receptive fields
+    conv = x @ W.reshape(c_out, -1).T + b
+    want = (conv - mean) / np.sqrt(var + eps) * gamma + beta  # batch normalisation, inference form
+    Wp, bp, delta = P.bn_fold(W, b, gamma, beta, mean, var, eps)
+    assert np.allclose(x @ Wp.reshape(c_out, -1).T + bp, want, rtol=1e-12, atol=1e-12)
+    assert np.allclose(delta, np.abs(Wp.reshape(c_out, -1)).max(axis=1) / 127.0, rtol=0, atol=0)
+    assert delta[2] == 0.0 and np.all(Wp[2] == 0) and bp[2] == beta[2]
+    for co in (0, 1, 3, 4, 5):
+        assert np.abs(P.quantize_weights(Wp[co], delta[co])).max() == 127
+    # no bias: the mean still shifts
+    Wp2, bp2, _ = P.bn_fold(W, None, gamma, beta, mean, var, eps)
+    assert np.array_equal(Wp2, Wp) and np.allclose(bp2, -mean * gamma / np.sqrt(var + eps) + beta)
+
+
 def test_concat_sync_algorithm_2():
     ry, rv = [30000.0, 52000.0, 41000.0], [90.0, 61.5, 75.25]
     s = P.concat_sync(ry, rv)
