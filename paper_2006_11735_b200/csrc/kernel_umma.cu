@@ -319,6 +319,34 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Position of the MMA issuer in the stage ring, kept as ready-made operands.
+struct IssueRing {
+    int stage;
+    uint32_t parity, a_lo, full_bar, empty_bar;
+};
+// `rounds` pipeline stages of one 128-byte k-iteration each into the accumulator at d_tmem:
+// wait for the stage, four MMAs (A at a_lo, B right behind it in the stage), commit the stage.
+// Straight-line apart from the loop itself; returns false when a wait gave up.
+__device__ __forceinline__ bool issue_rounds(IssueRing &g, uint32_t d_tmem, uint32_t idesc, int rounds, int stages, uint32_t a_lo0,
+                                             uint32_t stage_step, uint32_t slot_a_step, uint32_t desc_hi32, uint32_t full0,
+                                             uint32_t empty0, volatile int *abort_flag)
+{
+    uint32_t acc = 0;
+    for (int ki = 0; ki < rounds; ++ki) {
+        if (!mbar_test_wait(g.full_bar, g.parity) && !mbar_wait(g.full_bar, g.parity, abort_flag)) return false;
+        umma_slot<4>(d_tmem, g.a_lo, g.a_lo + slot_a_step, desc_hi32, idesc, acc);
+        acc = 1;
+        umma_commit(g.empty_bar);
+        const bool wrap = ++g.stage == stages;
+        g.stage = wrap ? 0 : g.stage;
+        g.parity ^= wrap ? 1u : 0u;
+        g.a_lo = wrap ? a_lo0 : g.a_lo + stage_step;
+        g.full_bar = wrap ? full0 : g.full_bar + 8u;
+        g.empty_bar = wrap ? empty0 : g.empty_bar + 8u;
+    }
+    return true;
+}
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int *r)
 {
     asm volatile(
@@ -693,7 +721,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, slot_step = (uint32_t)u.slot_bytes >> 4;
             const uint32_t slot_a_step = (uint32_t)u.slot_a_bytes >> 4;
             const uint32_t b_step = (uint32_t)(u.resident_b ? u.b_tile_bytes : u.slot_bytes) >> 4;
-            const bool simple = kj == 4 && u.kg == 1 && !u.resident_b && u.p_iters == 0;
+            const bool simple = kj == 4 && u.kg == 1 && !u.resident_b;
             const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & (u.nbuf - 1);
@@ -709,30 +737,27 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     sb = ((smem_u32(b_res + (size_t)((tile - m_tile * u.n_tiles) * k_iters) * u.b_tile_bytes) & 0x3FFFFu) >> 4) | (1u << 16);
                 }
                 if (simple) {
-                    // The long reductions (one 128-byte k-iteration per stage, B riding in the stage, no
-                    // projection): a round per stage of nothing but the wait, four MMAs and the commit.
-                    // Every taken branch of this lone thread costs tens of cycles that the tensor
-                    // pipe's short queue does not cover, and here there are 8 to 36 rounds per tile.
-                    uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step;
-                    uint32_t full_bar = full0 + 8u * (uint32_t)stage, empty_bar = empty0 + 8u * (uint32_t)stage;
-                    uint32_t acc = 0;
-                    for (int ki = 0; ki < k_iters; ++ki) {
-                        if (!mbar_test_wait(full_bar, parity) && !mbar_wait(full_bar, parity, &sh->abort_flag)) {
-                            give_up(sh, u.status, 3);
-                            ok = false;
-                            break;
-                        }
-                        umma_slot<4>(d_tmem, a_lo, a_lo + slot_a_step, desc_hi32, u.idesc, acc);
-                        acc = 1;
-                        umma_commit(empty_bar);
-                        const bool wrap = ++stage == u.stages;
-                        stage = wrap ? 0 : stage;
-                        parity ^= wrap ? 1u : 0u;
-                        a_lo = wrap ? a_lo0 : a_lo + stage_step;
-                        full_bar = wrap ? full0 : full_bar + 8u;
-                        empty_bar = wrap ? empty0 : empty_bar + 8u;
+                    // The long reductions (one 128-byte k-iteration per stage, B riding in the stage):
+                    // a round per stage of nothing but the wait, four MMAs and the commit.  Every
+                    // taken branch of this lone thread costs tens of cycles that the tensor pipe's
+                    // short queue does not cover, and here there are 6 to 36 rounds per tile.  A fused
+                    // projection's iterations come first, into the second accumulator tile.
+                    IssueRing ring;
+                    ring.stage = stage; ring.parity = parity;
+                    ring.a_lo = a_lo0 + (uint32_t)stage * stage_step;
+                    ring.full_bar = full0 + 8u * (uint32_t)stage; ring.empty_bar = empty0 + 8u * (uint32_t)stage;
+                    if (u.p_iters) {
+                        ok = issue_rounds(ring, d_tmem + (uint32_t)u.block_n, u.idesc_p, u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
+                                          desc_hi32, full0, empty0, &sh->abort_flag);
+                        if (ok) ok = issue_rounds(ring, d_tmem, u.idesc, k_iters - u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
+                                                  desc_hi32, full0, empty0, &sh->abort_flag);
+                    } else {
+                        ok = issue_rounds(ring, d_tmem, u.idesc, k_iters, u.stages, a_lo0, stage_step, slot_a_step, desc_hi32, full0, empty0,
+                                          &sh->abort_flag);
                     }
+                    stage = ring.stage; parity = ring.parity;
                     if (ok) umma_commit(smem_u32(&sh->tmem_full[buf]));
+                    else give_up(sh, u.status, 3);
                     continue;
                 }
                 for (int ki = 0; ki < k_iters;) {
