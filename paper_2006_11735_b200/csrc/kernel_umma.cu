@@ -722,6 +722,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const uint32_t slot_a_step = (uint32_t)u.slot_a_bytes >> 4;
             const uint32_t b_step = (uint32_t)(u.resident_b ? u.b_tile_bytes : u.slot_bytes) >> 4;
             const bool simple = kj == 4 && u.kg == 1 && !u.resident_b;
+            const bool one_round = kj == 4 && u.resident_b && k_iters <= u.kg && u.p_iters == 0;
             const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & (u.nbuf - 1);
@@ -735,6 +736,28 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 if (u.resident_b) {
                     const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
                     sb = ((smem_u32(b_res + (size_t)((tile - m_tile * u.n_tiles) * k_iters) * u.b_tile_bytes) & 0x3FFFFu) >> 4) | (1u << 16);
+                }
+                if (one_round) {
+                    // The short reductions (the whole tile in one stage, the filter bank resident): one
+                    // wait, the tile's MMAs, two commits, with as few branches as the lone thread can do with.
+                    const uint32_t full_bar = full0 + 8u * (uint32_t)stage;
+                    if (!mbar_test_wait(full_bar, parity) && !mbar_wait(full_bar, parity, &sh->abort_flag)) {
+                        give_up(sh, u.status, 3);
+                        break;
+                    }
+                    uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step, b_lo = sb;
+                    umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, 0u);
+                    for (int e = 1; e < k_iters; ++e) {
+                        a_lo += slot_step;
+                        b_lo += b_step;
+                        umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, 1u);
+                    }
+                    umma_commit(empty0 + 8u * (uint32_t)stage);
+                    umma_commit(smem_u32(&sh->tmem_full[buf]));
+                    const bool wrap = ++stage == u.stages;
+                    stage = wrap ? 0 : stage;
+                    parity ^= wrap ? 1u : 0u;
+                    continue;
                 }
                 if (simple) {
                     // The long reductions (one 128-byte k-iteration per stage, B riding in the stage):
