@@ -562,7 +562,11 @@ __device__ __forceinline__ void epilogue16(const int *acc, const int *accp, int 
 
 }  // namespace
 
-template <int EPI>
+// ISSUE selects the MMA issuer's code at compile time: 0 the general loop, 1 the long
+// reductions (one k-iteration per stage, B in the stage), 2 the tiles that fit one stage with a
+// resident filter bank.  The issuer is a lone thread: code it never runs still costs it
+// instruction fetches, so each instance carries only its own path.
+template <int EPI, int ISSUE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_skip,
@@ -721,8 +725,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, slot_step = (uint32_t)u.slot_bytes >> 4;
             const uint32_t slot_a_step = (uint32_t)u.slot_a_bytes >> 4;
             const uint32_t b_step = (uint32_t)(u.resident_b ? u.b_tile_bytes : u.slot_bytes) >> 4;
-            const bool simple = kj == 4 && u.kg == 1 && !u.resident_b;
-            const bool one_round = kj == 4 && u.resident_b && k_iters <= u.kg && u.p_iters == 0;
+            constexpr bool simple = ISSUE == 1, one_round = ISSUE == 2;
             const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & (u.nbuf - 1);
@@ -783,7 +786,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     else give_up(sh, u.status, 3);
                     continue;
                 }
-                for (int ki = 0; ki < k_iters;) {
+                for (int ki = 0; ISSUE == 0 && ki < k_iters;) {
                     if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
                         give_up(sh, u.status, 3);
                         ok = false;
@@ -1578,14 +1581,30 @@ int umma_init_once()
     if (rc != ICONV_OK) return rc;
     static bool attr_set = false;
     if (!attr_set) {
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
+        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
         ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
@@ -2046,7 +2065,15 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
                         (p->resident_b ? (size_t)u.b_tile_bytes * (u.p_iters + u.taps * u.cchunks) * u.n_tiles : 0) + sizeof(Shared) + 1024 +
                         (size_t)p->epi_warps * p->epi_warp_bytes;
     if (smem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
-#define ICONV_LAUNCH(E) umma_conv_kernel<E><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u)
+    const int kj_l = p->kc >> 5;
+    const int issue = (kj_l == 4 && p->kg == 1 && !p->resident_b) ? 1
+                      : (kj_l == 4 && p->resident_b && u.p_iters + u.taps * u.cchunks <= p->kg && u.p_iters == 0) ? 2 : 0;
+#define ICONV_LAUNCH(E)                                                                                                   \
+    do {                                                                                                                  \
+        if (issue == 1) umma_conv_kernel<E, 1><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u);      \
+        else if (issue == 2) umma_conv_kernel<E, 2><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u); \
+        else umma_conv_kernel<E, 0><<<grid, NUM_THREADS, smem, stream>>>(tmap_x, p->tmap_w, tmap_out, tmap_skip, a, u);                 \
+    } while (0)
     switch (p->epi) {
     case EPI_RAW: ICONV_LAUNCH(EPI_RAW); break;
     case EPI_FAST: ICONV_LAUNCH(EPI_FAST); break;
