@@ -644,7 +644,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const int q = (int)rem - p * a.w_out;
                 int kx = 0, ki = 0;
                 // segment 0: the fused projection (its own input tensor, stride and padding)
-                {
+                if (EPI == EPI_PROJ) {
                     const int cwp = q * u.p_stride - u.p_pad, chp = p * u.p_stride - u.p_pad;
                     int r = 0, s = 0;
                     for (int tap = 0; tap < u.p_taps && ok; ++tap) {
@@ -772,7 +772,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ring.stage = stage; ring.parity = parity;
                     ring.a_lo = a_lo0 + (uint32_t)stage * stage_step;
                     ring.full_bar = full0 + 8u * (uint32_t)stage; ring.empty_bar = empty0 + 8u * (uint32_t)stage;
-                    if (u.p_iters) {
+                    if (EPI == EPI_PROJ && u.p_iters) {
                         ok = issue_rounds(ring, d_tmem + (uint32_t)u.block_n, u.idesc_p, u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
                                           desc_hi32, full0, empty0, &sh->abort_flag);
                         if (ok) ok = issue_rounds(ring, d_tmem, u.idesc, k_iters - u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
@@ -796,9 +796,9 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step;
                     uint32_t b_lo = u.resident_b ? sb : a_lo + slot_a_step;
                     const int in_stage = min(u.kg, k_iters - ki);
-                    if (kj == 4) umma_stage<4>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, u.p_iters);
-                    else if (kj == 2) umma_stage<2>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, u.p_iters);
-                    else umma_stage<1>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, u.p_iters);
+                    if (kj == 4) umma_stage<4>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
+                    else if (kj == 2) umma_stage<2>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
+                    else umma_stage<1>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
                     ki += in_stage;
                     if (u.resident_b) sb = b_lo + (uint32_t)in_stage * b_step;
                     umma_commit(smem_u32(&sh->empty[stage]));   // frees the stage when these MMAs are done
