@@ -491,7 +491,14 @@ __device__ __forceinline__ void epilogue16_pc(const int *acc, const int *accp, i
         // S = accp + b_p is the projection's int32 Y.  32-bit form (bounds proven at plan time):
         // Y = U + ((accp * skip_mul + C) >> skip_shift), C = b_p * skip_mul + 2^(skip_shift-1) + (b << skip_shift);
         // otherwise the rescale runs in 64 bits with the two biases apart.
-        if (s.proj32) {
+        if (!PC && s.proj32 == 2) {
+            // as EPI_FAST: no clamp before Eq. 4, the u8 saturation that follows stands for both (proven at plan time)
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const int y = acc[k] + ((accp[k] * s.skip_mul + ca[k]) >> s.skip_shift);
+                V[k] = (y * s.q_mul + s.q_half) >> s.q_shift;
+            }
+        } else if (s.proj32) {
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
                 chan_params<PC>(s, u, co0 + k, h, mul, half, shift);
@@ -1428,6 +1435,25 @@ int choose_projection_epilogue(const iconv_desc &d, int c_out_pad, std::vector<i
         for (long long k = 0; k < KP; ++k) sw += wr[k] < 0 ? -(long long)wr[k] : wr[k];
         const long long C = (long long)d.proj_bias[co] * d.skip_mul + half + ((long long)d.bias[co] << d.skip_shift);
         if (sw * pmax * d.skip_mul + labs64(C) >= (1ll << 31)) proj32 = 0;
+    }
+    // The fast form (no explicit BReLU clamp, as EPI_FAST): per-layer parameters, a plain u8 output
+    // whose bound h_i already maps to 255, and |Y| * mul + half < 2^31 for the worst case of both
+    // reductions with the layer's actual weights.
+    if (proj32 && !d.per_channel && tail_free && d.out_dtype == ICONV_U8 && d.out_hi == 255 && d.brelu) {
+        const long long mul = d.mul[0], qhalf = 1ll << (d.shift[0] - 1);
+        bool fast = (long long)(((unsigned long long)d.h_i[0] * (unsigned long long)mul + (unsigned long long)qhalf) >> d.shift[0]) >= 255;
+        const long long xmax = d.in_dtype == ICONV_U8 ? 255 : 128;
+        const long long K = (long long)d.kh * d.kw * d.c_in;
+        for (int co = 0; co < d.c_out && fast; ++co) {
+            long long sw = 0, swp = 0;
+            const int8_t *wr = d.weights + (long long)co * K, *wp = d.proj_weights + (long long)co * KP;
+            for (long long k = 0; k < K; ++k) sw += wr[k] < 0 ? -(long long)wr[k] : wr[k];
+            for (long long k = 0; k < KP; ++k) swp += wp[k] < 0 ? -(long long)wp[k] : wp[k];
+            const long long C = (long long)d.proj_bias[co] * d.skip_mul + half + ((long long)d.bias[co] << d.skip_shift);
+            const long long ymax = sw * xmax + ((swp * pmax * d.skip_mul + labs64(C)) >> d.skip_shift) + 1;
+            if (ymax * mul + qhalf >= (1ll << 31)) fast = false;
+        }
+        if (fast) proj32 = 2;
     }
     for (int co = 0; co < d.c_out; ++co) {
         c_b[co] = d.proj_bias[co];
