@@ -39,6 +39,11 @@ WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"
              "vdsr": ("VDSR int8 images/sec", "vdsr_16x256x256x1"),
              "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1"),
              "vrcnn_hd": ("VRCNN int8 images/sec", "vrcnn_1x1600x2560x1")}
+# DRAM bytes (read + written) per tensor-core launch of one forward, from a one-pass ncu capture
+# of the full workload (command and per-kernel figures: profiles/dram_traffic_resnet50_b256.md),
+# valid only for the kernel source it was taken on: {workload: (bytes per launch, sha256 of
+# csrc/kernel_umma.cu)}.  A changed kernel reports null until the counters are taken again.
+DRAM_TRAFFIC = {"resnet50": (93223973, "dd97c3edb066cdea6a601480599b4600effab8ca5c46244dff8b114cbb5b85ab")}
 NOMINAL_INT8_TOPS = 4500.0      # NVIDIA's dense INT8 figure for B200 (context only)
 INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
 
@@ -243,8 +248,15 @@ def main():
     issue_tops, issue_cycles = B.iconv_probe_mma_rate(256, 100000)     # outside every timed region
     umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
+    traffic = None
+    if args.workload in DRAM_TRAFFIC and net.n == full.n:
+        import hashlib
+        src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2006_11735_b200", "csrc", "kernel_umma.cu")
+        with open(src, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() == DRAM_TRAFFIC[args.workload][1]:
+                traffic = DRAM_TRAFFIC[args.workload][0]
     roofline = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "tensor", "achieved": umma_tops, "peak": int8_peak,
-                "unit": "TOP/s", "frac": umma_tops / int8_peak, "traffic": None, "peak_kind": peak_kind + " 2 x bf16 sustained",
+                "unit": "TOP/s", "frac": umma_tops / int8_peak, "traffic": traffic, "peak_kind": peak_kind + " 2 x bf16 sustained",
                 "launches": umma_launches, "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
                 "frac_of_nominal_4500": umma_tops / NOMINAL_INT8_TOPS,
                 "issue_rate_peak": issue_tops, "frac_of_issue_rate_peak": umma_tops / issue_tops,
@@ -252,7 +264,8 @@ def main():
     # the same launches against the memory roofline: most layers of this workload are bound by it
     umma_gbs = fam_bytes.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e9
     roofline_hbm = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "hbm", "achieved": umma_gbs, "peak": hbm_peak,
-                    "unit": "GB/s", "frac": umma_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind + " copy bandwidth",
+                    "unit": "GB/s", "frac": umma_gbs / hbm_peak, "traffic": traffic,
+                    "algorithmic_bytes_per_launch": fam_bytes.get("umma", 0) / max(1, umma_launches), "peak_kind": peak_kind + " copy bandwidth",
                     "algorithmic_bytes_per_step": int(sum(abytes.values())),
                     "whole_step_gbs": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9}
 
