@@ -290,11 +290,49 @@ __global__ void __launch_bounds__(256) avgpool_kernel(const uint8_t *x, uint8_t 
     }
 }
 
+// Sixteen channels per thread (16-byte loads, a warp reads 512 contiguous bytes of every pixel),
+// byte lanes widened into 16 int sums; for channel counts that are multiples of 16 and 16-byte
+// aligned tensors.  The sums stay far inside int32 (at most hw * 255).
+__global__ void __launch_bounds__(128) avgpool16_kernel(const uint8_t *__restrict__ x, uint8_t *__restrict__ out, int n, int hw, int cg,
+                                                        int mul, int shift, int max_int)
+{
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n * cg) return;
+    const int img = e / cg, g = e - img * cg;
+    const uint4 *p = (const uint4 *)x + (size_t)img * hw * cg + g;
+    int sum[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) sum[k] = 0;
+#pragma unroll 7
+    for (int i = 0; i < hw; ++i) {
+        const uint4 v = __ldg(p + (size_t)i * cg);
+        const unsigned wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 16; ++k) sum[k] += (int)((wds[k >> 2] >> (8 * (k & 3))) & 0xffu);
+    }
+    unsigned o[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        long long V = round_shift64((long long)sum[k] * mul, shift);
+        V = V < 0 ? 0 : (V > max_int ? max_int : V);
+        o[k >> 2] |= (unsigned)V << (8 * (k & 3));
+    }
+    ((uint4 *)out)[e] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 int launch_avgpool(const void *x, void *out, int n, int h, int w, int c, int mul, int shift, int max_int,
                    cudaStream_t stream)
 {
     const long long total = (long long)n * c;
     if (total == 0) return ICONV_OK;
+    if (c % 16 == 0 && (uintptr_t)x % 16 == 0 && (uintptr_t)out % 16 == 0 && total / 16 < (1ll << 31) && max_int <= 255 &&
+        (long long)h * w * 255 < (1ll << 31)) {
+        const int groups = (int)(total / 16);
+        avgpool16_kernel<<<(unsigned)((groups + 127) / 128), 128, 0, stream>>>((const uint8_t *)x, (uint8_t *)out, n, h * w, c / 16, mul,
+                                                                             shift, max_int);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        return ICONV_OK;
+    }
     long long blocks = (total + 255) / 256;
     avgpool_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)x, (uint8_t *)out, n, h * w, c, mul, shift,
                                                          max_int);
