@@ -106,10 +106,25 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def probe_mma_rate(block_n: int = 256, iters: int = 100000):
+    """(whole-GPU int8 TOP/s, cycles per instruction) of back-to-back tcgen05.mma kind::i8: the
+    benchmark's own measurement aid, a small library of its own built next to the layer's."""
+    import ctypes as C
+    from paper_2006_11735_b200 import build as lib_build
+    lib = C.CDLL(lib_build.PROBE_LIB)
+    lib.probe_mma_rate.argtypes = [C.c_int32, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.probe_mma_rate.restype = C.c_int
+    tops, cyc = C.c_double(), C.c_double()
+    rc = lib.probe_mma_rate(block_n, iters, C.byref(tops), C.byref(cyc))
+    if rc != 0:
+        raise RuntimeError("probe_mma_rate failed with status %d" % rc)
+    return tops.value, cyc.value
+
+
 def oracle_images_per_s(n_images: int, repeats: int = 1, first: int = 0):
     """Times the CPU oracle, as it stands, on n_images of the workload (forward only)."""
     from oracle import networks as ON
-    from paper_2006_11735_b200.network import load_params
+    from workloads.params import load_params
     from workloads import networks as N
     net = N.resnet50()
     params = load_params("resnet50")
@@ -135,7 +150,7 @@ def run_reference(args):
         oracle_images_per_s(1)
     t0 = time.perf_counter()
     from oracle import networks as ON
-    from paper_2006_11735_b200.network import load_params
+    from workloads.params import load_params
     from workloads import networks as N
     net = N.resnet50()
     params = load_params("resnet50")
@@ -245,7 +260,7 @@ def main():
             fam_bytes[fam] = fam_bytes.get(fam, 0) + abytes.get(name, 0)
             layer_ms[name] = layer_ms.get(name, 0.0) + dt / args.steps
     int8_peak, hbm_peak, peak_kind = measured_peaks()
-    issue_tops, issue_cycles = B.iconv_probe_mma_rate(256, 100000)     # outside every timed region
+    issue_tops, issue_cycles = probe_mma_rate(256, 100000)             # outside every timed region
     umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
     traffic = None

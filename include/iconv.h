@@ -25,6 +25,11 @@
  *   - Weights are [c_out][kh][kw][c_in] int8.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     Forward calls only enqueue work on it and return; they never synchronise.
+ *   - Devices: a plan belongs to the device that was current when iconv_plan ran (its weights and
+ *     constants live there); forwards run on the current device.  The library keeps a small
+ *     table per device (shared-memory opt-in of its kernels, SM count, address of the status
+ *     word), filled by the first call on each device, so one process may drive several GPUs;
+ *     device indices up to 63 are supported.
  */
 #ifndef ICONV_H_
 #define ICONV_H_
@@ -50,7 +55,7 @@ typedef enum {
     ICONV_ERR_OVERFLOW = -4,     /* worst-case |Y| could exceed int32 */
     ICONV_ERR_UNSUPPORTED = -5,  /* valid request that no kernel implements */
     ICONV_ERR_CUDA = -6,         /* a CUDA call failed; text in iconv_last_error() */
-    ICONV_ERR_TIMEOUT = -7       /* a bounded device-side wait ran out (reported by iconv_check) */
+    ICONV_ERR_TIMEOUT = -7       /* a bounded device-side wait ran out (reported by iconv_check; nothing else maps to it) */
 } iconv_status;
 
 typedef enum {
@@ -67,9 +72,10 @@ typedef enum {
     ICONV_KERNEL_DIRECT = 1,   /* CUDA-core direct convolution, any shape */
     ICONV_KERNEL_UMMA = 2,     /* tcgen05.mma kind::i8 implicit GEMM, TMA im2col staging */
     ICONV_KERNEL_THIN = 3,     /* bandwidth-bound layers: c_in <= 4 or c_out == 1 */
-    ICONV_KERNEL_STEM = 4,     /* 7x7/2 layer over a 3-channel image: space-to-depth repack into
-                                  plan-owned scratch, then the tensor-core kernel.  Forwards of
-                                  one such plan must not overlap on the GPU (they share the scratch). */
+    ICONV_KERNEL_STEM = 4,     /* first layers the tensor cores cannot read directly (7x7/2 over a 3-channel
+                                  image; stride-1 filters over a single-channel image): a repack of the
+                                  image into the caller's workspace (iconv_workspace_bytes), then the
+                                  tensor-core kernel on the repacked tensor */
     ICONV_KERNEL_UMMA_IM2COL = 5  /* the tensor-core kernel with im2col staging even where the plan
                                   would load one input patch per tile (stride-1 filters); reported
                                   as ICONV_KERNEL_UMMA by iconv_plan_kernel */
@@ -114,8 +120,8 @@ typedef struct iconv_plan_s iconv_plan_t;
 /*
  * iconv_plan -- validate a layer, choose its kernel, upload its parameters (Section 3.1's
  * W_i, b_i; Eq. 4's mul, shift; Section 3.3's h_i) and build its TMA descriptors.
- * Allocates device memory with cudaMalloc on the current device; call it outside any
- * stream capture.  Rejects layers whose worst-case |Y| (c_in*kh*kw * 255 * 127 + |b| +
+ * Allocates device memory with cudaMalloc on the current device for those parameters only (a plan
+ * owns no activation-sized memory); call it outside any stream capture.  Rejects layers whose worst-case |Y| (c_in*kh*kw * 255 * 127 + |b| +
  * skip bound) reaches 2^31 with ICONV_ERR_OVERFLOW.  *plan_out is owned by the caller
  * and released with iconv_plan_destroy.
  */
@@ -131,24 +137,51 @@ ICONV_API int iconv_plan_kernel(const iconv_plan_t *plan);
 ICONV_API int iconv_plan_describe(const iconv_plan_t *plan, char *text, size_t size);
 
 /*
+ * iconv_workspace_bytes -- bytes of caller-owned device scratch one forward of this plan needs
+ * (Section 3.1's layer takes X_i, W_i, b_i; the scratch only holds a rearranged copy of X_i for the
+ * first layers of kernel family ICONV_KERNEL_STEM: 16 bytes per repacked position).  0 for every
+ * other plan and for a NULL plan.  The size depends on the plan alone, so one buffer of the
+ * largest size over a network's plans serves all of them in turn.
+ */
+ICONV_API size_t iconv_workspace_bytes(const iconv_plan_t *plan);
+
+/*
  * iconv_forward -- one layer forward (Section 3.1 / Eq. 4 / Eq. 5 as listed at the top).
  * x, skip, out: DEVICE pointers owned by the caller.  x holds n*h*w*in_c_total elements
  * of in_dtype; out holds n*h_out*w_out*out_c_total elements of out_dtype, of which only
  * the slice [out_c_offset, out_c_offset + c_out) of each pixel is written; skip (NULL when
  * skip_dtype < 0) holds n*h_out*w_out*skip_c_total elements (or, with a fused projection, the
- * projection's input: n*proj_h*proj_w*proj_c_total elements).  Asynchronous on cuda_stream.
- * The plan is not modified: concurrent forwards on different streams are allowed.
+ * projection's input: n*proj_h*proj_w*proj_c_total elements).  workspace: DEVICE, 16-byte aligned,
+ * at least iconv_workspace_bytes(plan) bytes, owned by the caller, contents undefined before and
+ * after the call (NULL when that size is 0; ICONV_ERR_ARG when it is missing).  Asynchronous on
+ * cuda_stream.  The plan is not modified and holds no per-call state: concurrent forwards of one
+ * plan on different streams are allowed as long as each has its own workspace (and output).
  */
 ICONV_API int iconv_forward(const iconv_plan_t *plan, const void *x, const void *skip, void *out,
-                  void *cuda_stream);
+                  void *workspace, void *cuda_stream);
 
 /*
  * Device-side waits (mbarrier phases) are bounded.  A kernel whose wait runs out records
  * a code (1-7) in a per-device status word and returns early.  iconv_check synchronises the
- * stream and returns ICONV_ERR_TIMEOUT if any kernel recorded a code since the last call,
- * ICONV_ERR_CUDA on a CUDA error, ICONV_OK otherwise.
+ * stream, reads and clears the word of the current device and returns ICONV_ERR_TIMEOUT if a
+ * kernel recorded such a code since the last call, ICONV_ERR_ARG for code 8 (a bias that
+ * iconv_stem_forward_static found out of range on the device), ICONV_ERR_CUDA on a CUDA error,
+ * ICONV_OK otherwise.
  */
 ICONV_API int iconv_check(void *cuda_stream);
+
+/*
+ * Test hooks (the paper has no counterpart).
+ * iconv_selftest_wait_timeout enqueues one tiny kernel (one CTA) that waits, with the very wait
+ * routine of the convolution kernels, on a barrier that nothing ever arrives at, with a limit of
+ * `limit_cycles` SM cycles (1e3 .. 2e8) instead of the kernels' two seconds; which = 0 the wait of
+ * a single-thread role, 1 the wait of an epilogue warp.  The wait gives up, records code 7 and the
+ * kernel returns, so the next iconv_check reports ICONV_ERR_TIMEOUT once and the context stays
+ * usable.  iconv_device_initialised returns the SM count recorded for `device` once a
+ * tensor-core plan or launch initialised that device's table, else -1.
+ */
+ICONV_API int iconv_selftest_wait_timeout(int32_t which, int64_t limit_cycles, void *cuda_stream);
+ICONV_API int iconv_device_initialised(int32_t device);
 
 /* Feature-map addition with ratio synchronisation as a stand-alone step (Sections 3.4.2,
  * 4.1):  Y = [(A - a_zero) * mul_a / 2^sh_a] + [(B - b_zero) * mul_b / 2^sh_b], then the
@@ -186,7 +219,7 @@ ICONV_API int ipool_avg_requant(const void *x, void *out, int32_t n, int32_t h, 
  *   x        DEVICE uint8 (or int8) [n][h][w][3], 16-byte aligned
  *   weights  DEVICE int8 [c_out][7][7][3]
  *   bias     DEVICE int32 [c_out], |b| <= 2^30 (a larger one is replaced by 0 and recorded in the
- *            device status word as code 8, which the next iconv_check reports)
+ *            device status word as code 8, which the next iconv_check reports as ICONV_ERR_ARG)
  *   out      DEVICE uint8 [n][h_out][w_out][out_c_total], 16-byte aligned; only the slice
  *            [out_c_offset, out_c_offset + c_out) of each pixel is written
  *
@@ -194,7 +227,8 @@ ICONV_API int ipool_avg_requant(const void *x, void *out, int32_t n, int32_t h, 
  * bit-identical to a planned forward of the same layer.  Returns ICONV_ERR_SHAPE with the sizes in
  * iconv_last_error() when n * (h_out + 3) * (w_out + 3) * 16 + 196608 exceeds ICONV_STEM_STATIC_BYTES
  * (157 images of 224 x 224 fit), ICONV_ERR_ARG unless c_out is a multiple of 16 in [16, 256],
- * 1 <= shift <= 31 and h_i * mul + 2^(shift-1) < 2^32.  Asynchronous on cuda_stream.
+ * 1 <= shift <= 31 and h_i * mul + 2^(shift-1) < 2^32, ICONV_ERR_UNSUPPORTED (before anything is
+ * enqueued) when a TMA descriptor of the repacked layer cannot be encoded.  Asynchronous on cuda_stream.
  *
  * The first call on each device looks up the array's device address (the GPU with that array
  * must be current); make that first call outside any stream capture.  All calls on a device share
@@ -258,14 +292,6 @@ ICONV_API int iconcat_plan(int32_t n_branches, const double *ratio_y, const doub
  * Errors: ICONV_ERR_ARG (null pointer, fraction outside (0, 1]), ICONV_ERR_ALIGN, ICONV_ERR_CUDA.
  * count = 0 returns 1. */
 ICONV_API int iq_sigma_bound(const int32_t *y, int64_t count, double fraction, int32_t *bound, void *cuda_stream);
-
-/* Measurement aid: how fast this GPU's tensor pipe retires tcgen05.mma kind::i8 (M = 128,
- * N = block_n, K = 32, u8 x s8 -> s32, the instruction of the convolution kernel) when only the
- * instruction stream limits it: operands stay in shared memory, one thread per SM issues `iters`
- * dependent instructions.  Returns whole-GPU TOP/s (2 * MACs / event time of the launch) and the
- * slowest SM's cycles per instruction.  Synchronous; allocates a few KB on the current device.
- * The paper has no counterpart: its GPU had no tensor cores. */
-ICONV_API int iconv_probe_mma_rate(int32_t block_n, int32_t iters, double *tops, double *cycles_per_mma);
 
 /* Text of the calling thread's last error (never NULL; valid until its next failing call). */
 ICONV_API const char *iconv_last_error(void);

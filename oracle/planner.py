@@ -58,7 +58,9 @@ def mul_shift(r, shift_min: int = 16, mul_min: int = MUL_MIN):
 
 def brelu_params(h_rf: float, ratio_Y: float, max_int: int, shift_min: int = 16):
     """Section 3.3.  Returns dict(h_ri, mul, shift, ratio_V, h_f, h_i)."""
-    h_ri = max(1, round_half_up(float(h_rf) * float(ratio_Y)))                # Eq. 8 (double product)
+    # Eq. 8: the bracket is taken of the exact product of the two given numbers (the doubles as
+    # they are, multiplied as rationals), not of a product already rounded to a double
+    h_ri = max(1, round_half_up(Fraction(float(h_rf)) * Fraction(float(ratio_Y))))
     return brelu_params_from_h_ri(h_ri, ratio_Y, max_int, shift_min)
 
 

@@ -1,14 +1,16 @@
 // Issue-rate probe of tcgen05.mma kind::i8: what the tensor pipe of this GPU sustains when
 // nothing but the instruction stream limits it (operands resident in shared memory, one
-// issuing thread per SM, every instruction accumulating into the same TMEM tile).  The
-// convolution kernel's achieved TOP/s is reported against this figure as well as against
-// the nominal one.
+// issuing thread per SM, every instruction accumulating into the same TMEM tile).  A
+// measurement aid of the benchmark, built into a library of its own (libiconv_probe.so): the
+// convolution kernel's achieved TOP/s is reported against this figure as well as against the
+// nominal one.  Not part of the layer's C ABI.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
 #include <algorithm>
 #include <vector>
 
-#include "plan.h"
-
-namespace iconv {
+namespace iconv_probe {
 
 namespace {
 
@@ -75,23 +77,25 @@ __global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int iters, Prob
 
 }  // namespace
 
-}  // namespace iconv
+}  // namespace iconv_probe
 
-using namespace iconv;
+using namespace iconv_probe;
 
-extern "C" int iconv_probe_mma_rate(int32_t block_n, int32_t iters, double *tops, double *cycles_per_mma)
+// How fast this GPU's tensor pipe retires tcgen05.mma kind::i8 (M = 128, N = block_n, K = 32,
+// u8 x s8 -> s32) when only the instruction stream limits it: one thread per SM issues `iters`
+// dependent instructions on operands in shared memory.  Writes whole-GPU TOP/s (2 * MACs / event
+// time of the launch) and the slowest SM's cycles per instruction to the HOST pointers.
+// Synchronous; allocates a few KB on the current device.  Returns 0, -1 (bad argument),
+// -6 (a CUDA call failed) or -7 (the bounded wait for the last instruction ran out).
+extern "C" __attribute__((visibility("default"))) int probe_mma_rate(int32_t block_n, int32_t iters, double *tops, double *cycles_per_mma)
 {
-    if (!tops || !cycles_per_mma || iters < 1 || iters > (1 << 22) || block_n < 16 || block_n > 256 || block_n % 16) {
-        set_error("iconv_probe_mma_rate: need 16 <= block_n <= 256 (a multiple of 16) and 1 <= iters <= 2^22");
-        return ICONV_ERR_ARG;
-    }
+    if (!tops || !cycles_per_mma || iters < 1 || iters > (1 << 22) || block_n < 16 || block_n > 256 || block_n % 16) return -1;
     int dev = 0, sms = 0;
-    ICONV_CUDA_TRY(cudaGetDevice(&dev));
-    ICONV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -6;
     const size_t smem = 16384 + 32768 + 1024;
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(mma_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (cudaFuncSetAttribute(mma_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -6;
     ProbeResult *d_res = nullptr;
-    ICONV_CUDA_TRY(cudaMalloc((void **)&d_res, sizeof(ProbeResult) * sms));
+    if (cudaMalloc((void **)&d_res, sizeof(ProbeResult) * sms) != cudaSuccess) return -6;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     float ms = 0.f;
     cudaError_t err = cudaEventCreate(&e0);
@@ -109,13 +113,13 @@ extern "C" int iconv_probe_mma_rate(int32_t block_n, int32_t iters, double *tops
     if (e0) cudaEventDestroy(e0);
     if (e1) cudaEventDestroy(e1);
     cudaFree(d_res);
-    if (err != cudaSuccess) return cuda_fail(err, "iconv_probe_mma_rate");
+    if (err != cudaSuccess) return -6;
     long long worst = 0;
     for (const ProbeResult &r : h) {
-        if (r.timed_out) { set_error("iconv_probe_mma_rate: a bounded wait ran out"); return ICONV_ERR_TIMEOUT; }
+        if (r.timed_out) return -7;
         worst = std::max(worst, r.cycles);
     }
     *cycles_per_mma = (double)worst / iters;
     *tops = 2.0 * (double)sms * iters * 128.0 * block_n * 32.0 / (ms * 1e-3) / 1e12;
-    return ICONV_OK;
+    return 0;
 }

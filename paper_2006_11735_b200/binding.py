@@ -15,9 +15,10 @@ KERNEL_AUTO, KERNEL_DIRECT, KERNEL_UMMA, KERNEL_THIN, KERNEL_STEM, KERNEL_UMMA_I
 DTYPE_CODE = {"u8": U8, "s8": S8, "i32": I32, "u8_raw128": U8_RAW128}
 KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin", KERNEL_STEM: "stem"}
 
-EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_plan_describe", "iconv_forward", "iconv_check",
+EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_plan_describe", "iconv_workspace_bytes", "iconv_forward",
+           "iconv_check", "iconv_selftest_wait_timeout", "iconv_device_initialised",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
-           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iq_sigma_bound", "iq_bn_fold", "iconcat_plan", "iconv_probe_mma_rate",
+           "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iq_sigma_bound", "iq_bn_fold", "iconcat_plan",
            "iconv_stem_forward_static", "iconv_last_error")
 
 
@@ -64,7 +65,10 @@ def _load():
     lib.iconv_plan_destroy.argtypes = [vp]
     lib.iconv_plan_kernel.argtypes = [vp]
     lib.iconv_plan_describe.argtypes = [vp, C.c_char_p, C.c_size_t]
-    lib.iconv_forward.argtypes = [vp, vp, vp, vp, vp]
+    lib.iconv_workspace_bytes.argtypes = [vp]
+    lib.iconv_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.iconv_selftest_wait_timeout.argtypes = [i32, i64, vp]
+    lib.iconv_device_initialised.argtypes = [i32]
     lib.iconv_check.argtypes = [vp]
     lib.iadd_requant.argtypes = [P(iadd_desc), vp, vp, vp, vp]
     lib.ipool_max.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
@@ -77,12 +81,12 @@ def _load():
     lib.iq_sigma_bound.argtypes = [C.c_void_p, C.c_int64, dbl, P(i32), C.c_void_p]
     lib.iq_bn_fold.argtypes = [vp, vp, vp, vp, vp, vp, dbl, i32, i64, vp, vp, vp]
     lib.iconcat_plan.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, P(dbl)]
-    lib.iconv_probe_mma_rate.argtypes = [i32, i32, P(dbl), P(dbl)]
     lib.iconv_stem_forward_static.argtypes = [P(istem_desc), vp, vp, vp, vp, vp]
     lib.iconv_last_error.restype = C.c_char_p
     for name in EXPORTS:
-        if name != "iconv_last_error":
+        if name not in ("iconv_last_error", "iconv_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
+    lib.iconv_workspace_bytes.restype = C.c_size_t
     return lib
 
 
@@ -160,8 +164,20 @@ def iconv_plan_describe(plan) -> str:
     return buf.value.decode()
 
 
-def iconv_forward(plan, x_ptr, skip_ptr, out_ptr, stream=0):
-    _check(lib.iconv_forward(plan, x_ptr, skip_ptr, out_ptr, stream))
+def iconv_workspace_bytes(plan) -> int:
+    return int(lib.iconv_workspace_bytes(plan))
+
+
+def iconv_forward(plan, x_ptr, skip_ptr, out_ptr, workspace_ptr=None, stream=0):
+    _check(lib.iconv_forward(plan, x_ptr, skip_ptr, out_ptr, workspace_ptr, stream))
+
+
+def iconv_selftest_wait_timeout(which: int, limit_cycles: int, stream=0):
+    _check(lib.iconv_selftest_wait_timeout(which, limit_cycles, stream))
+
+
+def iconv_device_initialised(device: int) -> int:
+    return int(lib.iconv_device_initialised(device))
 
 
 def iconv_check(stream=0):
@@ -248,13 +264,6 @@ def iconcat_plan(ratio_y, ratio_v, shift_min: int = 16):
                             scale.ctypes.data, ry_new.ctypes.data, C.byref(rmin)))
     return dict(ratio_V_min=rmin.value, mul=mul.tolist(), shift=shift.tolist(), delta_scale=scale.tolist(),
                 ratio_Y_new=ry_new.tolist())
-
-
-def iconv_probe_mma_rate(block_n: int = 256, iters: int = 200000):
-    """(whole-GPU int8 TOP/s, cycles per instruction) of back-to-back tcgen05.mma kind::i8."""
-    tops, cyc = C.c_double(), C.c_double()
-    _check(lib.iconv_probe_mma_rate(block_n, iters, C.byref(tops), C.byref(cyc)))
-    return tops.value, cyc.value
 
 
 def iconv_stem_forward_static(x_ptr, weights_ptr, bias_ptr, out_ptr, stream=0, *, n, h, w, c_out, in_dtype=U8_RAW128,

@@ -1,4 +1,5 @@
 // C-ABI entry points: validation, plans, dispatch.  No arithmetic of the layer lives here.
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -30,10 +31,26 @@ int cuda_fail(cudaError_t e, const char *what)
 // status word written by kernels whose bounded waits run out
 __device__ int g_device_status = 0;
 
+// Index of the current device in the library's per-device tables, or -1.
+int current_device_slot()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+    return dev;
+}
+
+// Device address of the status word on the current device (looked up once per device: the
+// symbol has one instance per GPU that loaded the library).
 int *device_status_ptr()
 {
-    int *p = nullptr;
-    if (cudaGetSymbolAddress((void **)&p, g_device_status) != cudaSuccess) return nullptr;
+    static std::atomic<int *> cache[MAX_DEVICES];
+    const int dev = current_device_slot();
+    if (dev < 0) return nullptr;
+    int *p = cache[dev].load(std::memory_order_acquire);
+    if (!p) {
+        if (cudaGetSymbolAddress((void **)&p, g_device_status) != cudaSuccess) return nullptr;
+        cache[dev].store(p, std::memory_order_release);
+    }
     return p;
 }
 
@@ -199,7 +216,6 @@ extern "C" int iconv_plan_destroy(iconv_plan_t *p)
     cudaFree(p->h_i_dev);
     cudaFree(p->w_packed);
     cudaFree(p->params_packed);
-    cudaFree(p->workspace);
     if (p->inner) iconv_plan_destroy(p->inner);
     delete p;
     return ICONV_OK;
@@ -279,7 +295,9 @@ extern "C" int iconv_plan_describe(const iconv_plan_t *p, char *text, size_t siz
     return ICONV_OK;
 }
 
-extern "C" int iconv_forward(const iconv_plan_t *p, const void *x, const void *skip, void *out, void *cuda_stream)
+extern "C" size_t iconv_workspace_bytes(const iconv_plan_t *p) { return p ? p->workspace_bytes : 0; }
+
+extern "C" int iconv_forward(const iconv_plan_t *p, const void *x, const void *skip, void *out, void *workspace, void *cuda_stream)
 {
     if (!p) {
         set_error("iconv_forward: null plan");
@@ -290,6 +308,14 @@ extern "C" int iconv_forward(const iconv_plan_t *p, const void *x, const void *s
     if (!x || !out || (d.skip_dtype >= 0 && !skip)) {
         set_error("iconv_forward: null tensor pointer");
         return ICONV_ERR_ARG;
+    }
+    if (p->workspace_bytes && !workspace) {
+        set_error("iconv_forward: this plan needs a workspace of %zu bytes (iconv_workspace_bytes)", p->workspace_bytes);
+        return ICONV_ERR_ARG;
+    }
+    if (p->workspace_bytes && ((uintptr_t)workspace % 16)) {
+        set_error("iconv_forward: the workspace must be 16-byte aligned");
+        return ICONV_ERR_ALIGN;
     }
     ConvArgs a;
     a.x = x; a.skip = d.skip_dtype >= 0 ? skip : nullptr; a.out = out;
@@ -305,7 +331,7 @@ extern "C" int iconv_forward(const iconv_plan_t *p, const void *x, const void *s
     switch (p->kernel) {
     case ICONV_KERNEL_UMMA: return launch_umma(p, a, st);
     case ICONV_KERNEL_THIN: return launch_thin(p, a, st);
-    case ICONV_KERNEL_STEM: return launch_stem(p, a, st);
+    case ICONV_KERNEL_STEM: return launch_stem(p, a, workspace, st);
     default: return launch_direct(a, st);
     }
 }
@@ -318,11 +344,27 @@ extern "C" int iconv_check(void *cuda_stream)
     if (st != 0) {
         const int z = 0;
         ICONV_CUDA_TRY(cudaMemcpyToSymbol(g_device_status, &z, sizeof(int)));
-        set_error("a kernel recorded device status code %d (1-7: a bounded wait ran out; 8: bias out of range)", st);
+        if (st == 8) {
+            set_error("a kernel recorded device status code 8: a bias beyond 2^30 in magnitude was given to "
+                      "iconv_stem_forward_static and replaced by 0");
+            return ICONV_ERR_ARG;
+        }
+        set_error("a kernel recorded device status code %d: a bounded device-side wait ran out", st);
         return ICONV_ERR_TIMEOUT;
     }
     return ICONV_OK;
 }
+
+extern "C" int iconv_selftest_wait_timeout(int32_t which, int64_t limit_cycles, void *cuda_stream)
+{
+    if (which < 0 || which > 1 || limit_cycles < 1000 || limit_cycles > 200000000ll) {
+        set_error("iconv_selftest_wait_timeout: which must be 0 or 1 and 1e3 <= limit_cycles <= 2e8");
+        return ICONV_ERR_ARG;
+    }
+    return launch_wait_selftest(which, limit_cycles, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int iconv_device_initialised(int32_t device) { return umma_device_ready(device); }
 
 extern "C" int iadd_requant(const iadd_desc *d, const void *a, const void *b, void *out, void *cuda_stream)
 {

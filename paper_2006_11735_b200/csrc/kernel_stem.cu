@@ -18,6 +18,7 @@
 // the layer is a kh x 1 filter over 16 channels: out(oh, ow) = sum_r T[oh+r][ow] . W'[r],
 // W'[r][j] = W[r][j].  Sixteen bytes per position instead of one, but the arithmetic moves
 // to the tensor cores and the CUDA cores keep only the epilogue.
+#include <atomic>
 #include <cstring>
 #include <vector>
 
@@ -30,7 +31,7 @@ namespace {
 // One thread writes the 16 bytes of one position (n, Y, X) of T.
 __global__ void __launch_bounds__(256)
 stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int n, int h, int w, int hp, int wp,
-                   int raw128)
+                   int raw128, int slack)
 {
     const long long total = (long long)n * hp * wp;
     for (long long pos = (long long)blockIdx.x * blockDim.x + threadIdx.x; pos < total;
@@ -57,6 +58,7 @@ stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int 
             }
         }
         *(uint4 *)(T + pos * 16) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+        if (slack && pos == total - 1) *(uint4 *)(T + total * 16) = make_uint4(0, 0, 0, 0);   // the 16 bytes of slack behind T
     }
 }
 
@@ -145,7 +147,6 @@ int rows_setup(iconv_plan_t *p)
         return ICONV_ERR_UNSUPPORTED;
     }
     p->workspace_bytes = (size_t)d.n * hp * wo * 16;
-    ICONV_CUDA_TRY(cudaMalloc(&p->workspace, p->workspace_bytes ? p->workspace_bytes : 16));
     return ICONV_OK;
 }
 
@@ -187,13 +188,13 @@ int stem_setup(iconv_plan_t *p)
     int rc = plan_create(&in, 1, &p->inner);
     if (rc != ICONV_OK) rc = iconv_plan(&in, &p->inner);
     if (rc != ICONV_OK) return rc;
+    // (the slack is only ever the right-hand neighbour of the last position, which no real output
+    // pixel reads; the repack kernel zeroes it so that the workspace holds no stale bytes)
     p->workspace_bytes = (size_t)d.n * hp * wp * 16 + 16;
-    ICONV_CUDA_TRY(cudaMalloc(&p->workspace, p->workspace_bytes));
-    ICONV_CUDA_TRY(cudaMemset((uint8_t *)p->workspace + p->workspace_bytes - 16, 0, 16));
     return ICONV_OK;
 }
 
-int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
+int launch_stem(const iconv_plan_t *p, const ConvArgs &a, void *workspace, cudaStream_t stream)
 {
     const iconv_desc &d = p->d;
     if (stem_kind(d) == 2) {
@@ -202,19 +203,19 @@ int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         long long blocks = (total + 255) / 256;
         if (blocks > 148ll * 32) blocks = 148ll * 32;
         if (blocks > 0)
-            rows_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)p->workspace, d.n, d.h, d.w, hp, wo,
+            rows_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)workspace, d.n, d.h, d.w, hp, wo,
                                                                      d.pad, d.kw, d.in_dtype == ICONV_U8_RAW128);
         ICONV_CUDA_TRY(cudaGetLastError());
-        return iconv_forward(p->inner, p->workspace, a.skip, a.out, (void *)stream);
+        return iconv_forward(p->inner, workspace, a.skip, a.out, nullptr, (void *)stream);
     }
     const int hp = p->h_out + 3, wp = p->w_out + 3;
     const long long total = (long long)d.n * hp * wp;
     long long blocks = (total + 255) / 256;
     if (blocks > 148ll * 32) blocks = 148ll * 32;
-    stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)p->workspace, d.n, d.h, d.w,
-                                                             hp, wp, d.in_dtype == ICONV_U8_RAW128);
+    stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)workspace, d.n, d.h, d.w,
+                                                             hp, wp, d.in_dtype == ICONV_U8_RAW128, 1);
     ICONV_CUDA_TRY(cudaGetLastError());
-    return iconv_forward(p->inner, p->workspace, a.skip, a.out, (void *)stream);
+    return iconv_forward(p->inner, workspace, a.skip, a.out, nullptr, (void *)stream);
 }
 
 }  // namespace iconv
@@ -237,22 +238,20 @@ constexpr size_t STEM_STATIC_T_OFFSET = STEM_STATIC_W_BYTES + STEM_STATIC_PAR_BY
 
 static __device__ __align__(256) unsigned char g_stem_static[ICONV_STEM_STATIC_BYTES];
 
-constexpr int MAX_DEVICES = 64;
-unsigned char *g_stem_static_ptr[MAX_DEVICES] = {nullptr};
+std::atomic<unsigned char *> g_stem_static_ptr[MAX_DEVICES];
 
 // Device address of the array on the current device (looked up on the first call per device).
 int stem_static_base(unsigned char **base)
 {
-    int dev = 0;
-    ICONV_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= MAX_DEVICES) { set_error("iconv_stem_forward_static: device index %d not supported", dev); return ICONV_ERR_UNSUPPORTED; }
-    if (!g_stem_static_ptr[dev]) {
-        unsigned char *ptr = nullptr;
+    const int dev = current_device_slot();
+    if (dev < 0) { set_error("iconv_stem_forward_static: no current device, or its index is beyond %d", MAX_DEVICES - 1); return ICONV_ERR_UNSUPPORTED; }
+    unsigned char *ptr = g_stem_static_ptr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         ICONV_CUDA_TRY(cudaGetSymbolAddress((void **)&ptr, g_stem_static));
         if (!ptr) { set_error("iconv_stem_forward_static: the scratch array has no device address"); return ICONV_ERR_CUDA; }
-        g_stem_static_ptr[dev] = ptr;
+        g_stem_static_ptr[dev].store(ptr, std::memory_order_release);
     }
-    *base = g_stem_static_ptr[dev];
+    *base = ptr;
     return ICONV_OK;
 }
 
@@ -359,14 +358,16 @@ extern "C" int iconv_stem_forward_static(const istem_desc *sd, const void *x, co
         tmp.tail = 1;
         tmp.q_mul = sd->mul; tmp.q_shift = sd->shift; tmp.q_h = sd->h_i;
         window_plan(&tmp);                   // one patch of T per tile where the geometry allows
-
+        rc = umma_check_maps(&tmp, T, out);  // every descriptor the launch will need, before anything is enqueued
+    }
+    if (rc == ICONV_OK) {
         stem_static_prepare_kernel<<<(tmp.c_out_pad * 512 + 255) / 256, 256, 0, stream>>>(weights, bias, w2, par, sd->c_out, tmp.c_out_pad,
                                                                                     sd->mul, sd->shift, sd->h_i, status);
         const long long total = (long long)sd->n * hp * wp;
         long long blocks = (total + 255) / 256;
         if (blocks > 148ll * 32) blocks = 148ll * 32;
         stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)x, T, sd->n, sd->h, sd->w, hp, wp,
-                                                                 sd->in_dtype == ICONV_U8_RAW128);
+                                                                 sd->in_dtype == ICONV_U8_RAW128, 0);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) rc = cuda_fail(e, "iconv_stem_forward_static launches");
     }

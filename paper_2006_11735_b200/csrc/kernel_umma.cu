@@ -29,6 +29,8 @@
 // the per-stage loops (no divisions: counters and multiply-shift reciprocals).
 #include <cuda.h>
 
+#include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "plan.h"
@@ -169,7 +171,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v)
 // limit ran out or another role already gave up.  A few plain probes first (the common short
 // wait), then suspending probes; the limit is counted on the SM's own cycle counter, read
 // only every 64 failed suspending probes, so a wait that succeeds soon costs no timer read.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit = WAIT_LIMIT_CYCLES)
 {
 #pragma unroll 1
     for (int i = 0; i < 4; ++i)
@@ -182,7 +184,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_CYCLES) return false;
+            else if (now - t0 > limit) return false;
         }
     }
 }
@@ -191,7 +193,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // barrier word only add shared-memory traffic).  These warps are the critical path of the
 // epilogue-bound layers, so they poll (with a back-off) rather than suspend; __syncwarp
 // orders the other lanes' later reads after lane 0's acquire.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane,
+                                               long long limit = WAIT_LIMIT_CYCLES)
 {
     int ok = 1;
     if (lane == 0) {
@@ -204,7 +207,7 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
                 if (*abort_flag) break;
                 const long long now = clock64();
                 if (t0 == 0) t0 = now;
-                else if (now - t0 > WAIT_LIMIT_CYCLES) break;
+                else if (now - t0 > limit) break;
             }
         }
     }
@@ -1304,6 +1307,27 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     }
 }
 
+// Self-test of the bounded waits: one CTA initialises an mbarrier that nothing ever arrives at
+// and waits on it with the kernels' own wait routines and a short limit.  The wait must give up,
+// record its code in the device status word and let the kernel return normally.
+__global__ void __launch_bounds__(64, 1) wait_timeout_selftest_kernel(int which, long long limit, int *status)
+{
+    __shared__ unsigned long long bar;
+    __shared__ volatile int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (which == 0 && threadIdx.x == 0) {              // the wait of a single-thread role (TMA producer, MMA issuer)
+        if (!mbar_wait(smem_u32(&bar), 0, &abort_flag, limit)) atomicCAS(status, 0, 7);
+    } else if (which == 1 && warp == 1) {             // the wait of an epilogue warp
+        if (!mbar_wait_warp(smem_u32(&bar), 0, &abort_flag, lane, limit) && lane == 0) atomicCAS(status, 0, 7);
+    }
+}
+
 // ---------------------------------------------------------------- host side
 namespace {
 
@@ -1600,61 +1624,87 @@ int umma_supported(const iconv_plan_t *p)
     return ICONV_OK;
 }
 
-// Once per process: driver entry points and the kernels' shared-memory opt-in.  Allocates nothing.
+// Once per device: driver entry points (once per process) and the kernels' shared-memory opt-in,
+// which is an attribute of the function ON THE CURRENT DEVICE, so every GPU a process uses gets
+// its own pass.  Allocates nothing.
+namespace {
+
+template <typename K>
+cudaError_t opt_in(K kernel) { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM); }
+
+template <int EPI>
+cudaError_t opt_in_conv()
+{
+    cudaError_t e = opt_in(umma_conv_kernel<EPI, 0>);
+    if (e == cudaSuccess) e = opt_in(umma_conv_kernel<EPI, 1>);
+    if (e == cudaSuccess) e = opt_in(umma_conv_kernel<EPI, 2>);
+    return e;
+}
+
+template <int EPI>
+cudaError_t opt_in_window_all()
+{
+    cudaError_t e = opt_in(umma_window_kernel<EPI, 3, 3, 2>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 3, 3, 4>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 5, 5, 2>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 4, 4, 1>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 4, 2, 1>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 0, 0, 0>);
+    return e;
+}
+
+template <int EPI>
+cudaError_t opt_in_window_skip()
+{
+    cudaError_t e = opt_in(umma_window_kernel<EPI, 3, 3, 2>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 3, 3, 4>);
+    if (e == cudaSuccess) e = opt_in(umma_window_kernel<EPI, 0, 0, 0>);
+    return e;
+}
+
+struct DeviceInit {
+    std::atomic<int> ready{0};      // 1 once the opt-ins ran on this device
+    int sms = 0;
+};
+DeviceInit g_device_init[MAX_DEVICES];
+std::mutex g_device_init_mutex;
+
+}  // namespace
+
+// The slot of the per-device table the first call on a device fills; tests read it to see that
+// initialisation is keyed by device (-1: not initialised yet).
+int umma_device_ready(int device)
+{
+    if (device < 0 || device >= MAX_DEVICES) return -1;
+    return g_device_init[device].ready.load(std::memory_order_acquire) ? g_device_init[device].sms : -1;
+}
+
 int umma_init_once()
 {
     const int rc = load_driver_entry_points();
     if (rc != ICONV_OK) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_WIDE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_RAW, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_FAST_SKIP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_SAFE_SKIP32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_conv_kernel<EPI_PROJ, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_FAST_SKIP8, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE_SKIP8, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE_SKIP8, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_SAFE_SKIP8, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<EPI_NARROW, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM));
-        attr_set = true;
-    }
-    static bool win_attr_set = false;
-    if (!win_attr_set) {
-#define ICONV_WIN_ATTR(E)                                                                                                          \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 3, 3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 5, 5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 4, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 4, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)); \
-    ICONV_CUDA_TRY(cudaFuncSetAttribute(umma_window_kernel<E, 0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM))
-        ICONV_WIN_ATTR(EPI_FAST);
-        ICONV_WIN_ATTR(EPI_SAFE);
-#undef ICONV_WIN_ATTR
-        win_attr_set = true;
-    }
+    const int dev = current_device_slot();
+    if (dev < 0) { set_error("tensor-core path: no current device, or its index is beyond %d", MAX_DEVICES - 1); return ICONV_ERR_UNSUPPORTED; }
+    DeviceInit &di = g_device_init[dev];
+    if (di.ready.load(std::memory_order_acquire)) return ICONV_OK;
+    std::lock_guard<std::mutex> lock(g_device_init_mutex);
+    if (di.ready.load(std::memory_order_acquire)) return ICONV_OK;
+    ICONV_CUDA_TRY(opt_in_conv<EPI_WIDE>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_RAW>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_FAST>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_FAST_SKIP8>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_SAFE>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_SAFE_SKIP8>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_SAFE_SKIP32>());
+    ICONV_CUDA_TRY(opt_in_conv<EPI_PROJ>());
+    ICONV_CUDA_TRY(opt_in_window_all<EPI_FAST>());
+    ICONV_CUDA_TRY(opt_in_window_all<EPI_SAFE>());
+    ICONV_CUDA_TRY(opt_in_window_skip<EPI_FAST_SKIP8>());
+    ICONV_CUDA_TRY(opt_in_window_skip<EPI_SAFE_SKIP8>());
+    ICONV_CUDA_TRY(opt_in(umma_window_kernel<EPI_NARROW, 3, 3, 2>));
+    ICONV_CUDA_TRY(opt_in(umma_window_kernel<EPI_NARROW, 0, 0, 0>));
+    ICONV_CUDA_TRY(cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev));
+    di.ready.store(1, std::memory_order_release);
     return ICONV_OK;
 }
 
@@ -1944,6 +1994,44 @@ int umma_setup(iconv_plan_t *p)
     return ICONV_OK;
 }
 
+// Every TMA descriptor one launch of the layer needs, for these tensor addresses: the input
+// (patch map in window mode, im2col map otherwise), the output rows and the skip rows (or the
+// fused projection's input).
+int encode_launch_maps(const iconv_plan_t *p, const void *x, const void *skip, void *out, CUtensorMap *tmap_x, CUtensorMap *tmap_out,
+                       CUtensorMap *tmap_skip)
+{
+    const iconv_desc &d = p->d;
+    int rc = p->window ? encode_patch_map(p, x, tmap_x) : encode_activation_map(p, x, tmap_x);
+    if (rc != ICONV_OK) return rc;
+    const long long m_total = (long long)d.n * p->h_out * p->w_out;
+    const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
+    memset(tmap_out, 0, sizeof(*tmap_out));
+    if (!p->window) {       // window mode stores from registers
+        rc = encode_rows_map((uint8_t *)out + (size_t)d.out_c_offset * esz, esz, d.c_out, d.out_c_total, m_total, p->piece_bytes, tmap_out);
+        if (rc != ICONV_OK) return rc;
+    }
+    *tmap_skip = *tmap_out;
+    if (p->epi == EPI_PROJ) {
+        rc = encode_projection_map(p, skip, tmap_skip);      // the slot of the skip map carries the projection's input
+        if (rc != ICONV_OK) return rc;
+    }
+    if (!p->window && (p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8)) {
+        rc = encode_rows_map((const uint8_t *)skip + d.skip_c_offset, 1, d.c_out, d.skip_c_total, m_total, p->piece_bytes, tmap_skip);
+        if (rc != ICONV_OK) return rc;
+    }
+    return ICONV_OK;
+}
+
+// ICONV_OK when every descriptor of a launch on these addresses can be encoded (nothing is enqueued).
+int umma_check_maps(const iconv_plan_t *p, const void *x, void *out)
+{
+    if (((uintptr_t)x % 16) || ((uintptr_t)out % 16)) { set_error("tensor pointers must be 16-byte aligned"); return ICONV_ERR_ALIGN; }
+    const int rc = umma_init_once();
+    if (rc != ICONV_OK) return rc;
+    CUtensorMap mx, mo, ms;
+    return encode_launch_maps(p, x, out, out, &mx, &mo, &ms);
+}
+
 int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
 {
     const iconv_desc &d = p->d;
@@ -1951,8 +2039,8 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         set_error("iconv_forward: tensor pointers must be 16-byte aligned");
         return ICONV_ERR_ALIGN;
     }
-    CUtensorMap tmap_x;
-    int rc = p->window ? encode_patch_map(p, a.x, &tmap_x) : encode_activation_map(p, a.x, &tmap_x);
+    CUtensorMap tmap_x, tmap_out, tmap_skip;
+    int rc = encode_launch_maps(p, a.x, a.skip, a.out, &tmap_x, &tmap_out, &tmap_skip);
     if (rc != ICONV_OK) return rc;
 
     UmmaArgs u;
@@ -2017,36 +2105,17 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.c_shift = p->params_packed + 2 * (size_t)p->c_out_pad;
     u.c_h = p->params_packed + 3 * (size_t)p->c_out_pad;
     u.c_b = p->params_packed + 4 * (size_t)p->c_out_pad;
-    const int esz = d.out_dtype == ICONV_I32 ? 4 : 1;
-    CUtensorMap tmap_out, tmap_skip;
-    memset(&tmap_out, 0, sizeof(tmap_out));
-    if (!p->window) {       // window mode stores from registers
-        rc = encode_rows_map((uint8_t *)a.out + (size_t)d.out_c_offset * esz, esz, d.c_out, d.out_c_total, u.m_total,
-                             p->piece_bytes, &tmap_out);
-        if (rc != ICONV_OK) return rc;
-    }
-    tmap_skip = tmap_out;
-    if (p->epi == EPI_PROJ) {
-        rc = encode_projection_map(p, a.skip, &tmap_skip);      // the slot of the skip map carries the projection's input
-        if (rc != ICONV_OK) return rc;
-    }
-    if (p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8) {
-        rc = encode_rows_map((const uint8_t *)a.skip + d.skip_c_offset, 1, d.c_out, d.skip_c_total, u.m_total,
-                             p->piece_bytes, &tmap_skip);
-        if (rc != ICONV_OK) return rc;
-    }
     find_divisor((unsigned)u.n_tiles, u.div_nt_mul, u.div_nt_shr);
     find_divisor((unsigned)p->w_out, u.div_w_mul, u.div_w_shr);
     find_divisor((unsigned)(p->h_out * p->w_out), u.div_hw_mul, u.div_hw_shr);
     u.status = device_status_ptr();
     if (!u.status) { set_error("device status word not available"); return ICONV_ERR_CUDA; }
 
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        ICONV_CUDA_TRY(cudaGetDevice(&dev));
-        ICONV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    }
+    // shared-memory opt-in and SM count of the device this launch goes to (a plan made on one
+    // device may run on another)
+    rc = umma_init_once();
+    if (rc != ICONV_OK) return rc;
+    const int sms = g_device_init[current_device_slot()].sms;
     if (p->window) {
         u.m_tiles = p->win_tpi * d.n;
         u.stages = p->win_stages;
@@ -2111,6 +2180,15 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     default: ICONV_LAUNCH(EPI_WIDE); break;
     }
 #undef ICONV_LAUNCH
+    ICONV_CUDA_TRY(cudaGetLastError());
+    return ICONV_OK;
+}
+
+int launch_wait_selftest(int which, long long limit_cycles, cudaStream_t stream)
+{
+    int *status = device_status_ptr();
+    if (!status) { set_error("device status word not available"); return ICONV_ERR_CUDA; }
+    wait_timeout_selftest_kernel<<<1, 64, 0, stream>>>(which, limit_cycles, status);
     ICONV_CUDA_TRY(cudaGetLastError());
     return ICONV_OK;
 }

@@ -34,9 +34,9 @@ struct iconv_plan_s {
     int epi_warp_bytes = 8192;           // staging memory per epilogue warp (im2col kernel)
     int group_uniform = 0;               // per-channel parameters equal within every 16-channel group
     int pair16 = 0;                      // internal (stem): 16-channel positions read in pairs, two taps per K step
-    // stem path: repacked image (plan-owned scratch) and the plan of the GEMM that follows
+    // stem path: the plan of the GEMM that follows the repack, and the size of the repacked image,
+    // which lives in the caller's workspace (iconv_workspace_bytes)
     iconv_plan_s *inner = nullptr;
-    void *workspace = nullptr;
     size_t workspace_bytes = 0;
 };
 
@@ -52,7 +52,9 @@ int launch_thin(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
 int umma_supported(const iconv_plan_t *p);   // ICONV_OK or the reason it is not
 bool umma_narrow(const iconv_desc &d);      // an 8-bit output too narrow or unaligned for 16-byte stores that window mode could still take
 int umma_setup(iconv_plan_t *p);
-int umma_init_once();                        // driver entry points, shared-memory opt-in; allocates nothing
+int umma_init_once();                        // driver entry points, shared-memory opt-in of the current device; allocates nothing
+int umma_device_ready(int device);           // the device's SM count once umma_init_once ran on it, else -1
+int umma_check_maps(const iconv_plan_t *p, const void *x, void *out);   // can every TMA descriptor of a launch be encoded?
 int umma_geometry(iconv_plan_t *p);           // host-only tile / pipeline / epilogue geometry
 int umma_encode_weight_map(iconv_plan_t *p);  // TMA map over p->w_packed
 void window_plan(iconv_plan_t *p);            // window mode if the layer allows (needs p->epi); host only
@@ -61,13 +63,16 @@ int thin_supported(const iconv_plan_t *p);
 int thin_setup(iconv_plan_t *p);
 int stem_supported(const iconv_plan_t *p);
 int stem_setup(iconv_plan_t *p);
-int launch_stem(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream);
+int launch_stem(const iconv_plan_t *p, const ConvArgs &a, void *workspace, cudaStream_t stream);
 
 int launch_add_requant(const iadd_desc &d, const void *a, const void *b, void *out, cudaStream_t stream);
 int launch_maxpool(const void *x, void *out, int n, int h, int w, int c, int k, int stride, int pad,
                    cudaStream_t stream);
 int launch_avgpool(const void *x, void *out, int n, int h, int w, int c, int mul, int shift, int max_int,
                    cudaStream_t stream);
-int *device_status_ptr();
+constexpr int MAX_DEVICES = 64;               // per-device tables (shared-memory opt-in, SM count, status word) have this many slots
+int current_device_slot();                    // index of the current device in those tables, or -1
+int *device_status_ptr();                     // the status word of the current device
+int launch_wait_selftest(int which, long long limit_cycles, cudaStream_t stream);
 
 }  // namespace iconv

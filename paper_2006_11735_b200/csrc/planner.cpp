@@ -121,7 +121,15 @@ extern "C" int iq_brelu_params(double h_rf, double ratio_y, int32_t max_int, int
         set_error("iq_brelu_params: bad argument");
         return ICONV_ERR_ARG;
     }
-    double hr = round_half_up(h_rf * ratio_y);                       // Eq. 8
+    // Eq. 8: [h_rf * ratio_Y] of the EXACT product.  p is the product rounded to a double and
+    // e = h_rf * ratio_Y - p exactly (one fused multiply-add), so the product is p + e with
+    // |e| <= ulp(p) / 2: only when p sits exactly on a tie (fraction 0.5) can e move the bracket,
+    // and then its sign decides (ties go up, so e >= 0 rounds up and e < 0 rounds down).
+    const double prod = h_rf * ratio_y;
+    if (!(prod < 2147483648.0)) { set_error("iq_brelu_params: h_ri does not fit int32"); return ICONV_ERR_OVERFLOW; }
+    const double err = std::fma(h_rf, ratio_y, -prod);
+    const double fl = std::floor(prod), frac = prod - fl;
+    double hr = (frac > 0.5 || (frac == 0.5 && err >= 0.0)) ? fl + 1.0 : fl;
     if (hr < 1.0) hr = 1.0;
     if (hr >= 2147483648.0) { set_error("iq_brelu_params: h_ri does not fit int32"); return ICONV_ERR_OVERFLOW; }
     const int64_t hri = (int64_t)hr;

@@ -5,32 +5,16 @@ Per-layer integer parameters (quantisation step, mul, shift, h_i, skip rescale) 
 a dict, e.g. read from ``workloads/params/*.json``; weights are re-created from the
 network's seed with the library's own Eq. 1 (``iq_quantize_weights``).
 """
-import json
-import os
-
 import numpy as np
 import torch
 
 from workloads import generators as gen
 from workloads.networks import AvgPool, Conv, MaxPool, Net
+from workloads.params import load_params  # noqa: F401  (re-exported: callers read cached parameters through here too)
 
 from . import binding as B
 
 _TORCH = {"u8": torch.uint8, "i32": torch.int32}
-PARAMS_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "params")
-
-
-def load_params(name: str) -> dict:
-    """Cached per-layer parameters of a full-size configuration (``float.hex`` strings for
-    doubles so that the quantisation steps round-trip exactly)."""
-    name = {"vrcnn_hd": "vrcnn"}.get(name, name)      # the single-picture workload runs configuration 3's layers
-    with open(os.path.join(PARAMS_DIR, name + ".json")) as f:
-        raw = json.load(f)
-    for p in raw["layers"].values():
-        if "delta" in p:
-            p["delta"] = float.fromhex(p["delta"])
-    return raw["layers"]
-
 
 def net_input(net: Net, first: int = 0, count=None) -> np.ndarray:
     t = net.tensors[net.input]
@@ -121,6 +105,14 @@ class Network:
                     continue
                 self.plans[op.name] = B.iconv_plan(**kw)
                 self.steps.append(("conv", op, None))
+        self._alloc_workspace()
+
+    def _alloc_workspace(self):
+        """One buffer of the largest workspace any plan asks for: the layers run one after another
+        on one stream, so they can share it."""
+        size = max([B.iconv_workspace_bytes(p) for p in self.plans.values()] + [0])
+        self.workspace = torch.empty((size,), dtype=torch.uint8, device=self.device) if size else None
+        self._ws_ptr = self.workspace.data_ptr() if size else None
 
     def _mergeable(self, a, b, params) -> bool:
         if not (isinstance(a, Conv) and isinstance(b, Conv)):
@@ -229,7 +221,7 @@ class Network:
             if kind == "conv":
                 skip_name = p if p is not None else op.skip       # a fused projection reads its own input
                 B.iconv_forward(self.plans[op.name], T[op.src].data_ptr(),
-                                T[skip_name].data_ptr() if skip_name else None, T[op.dst].data_ptr(), stream)
+                                T[skip_name].data_ptr() if skip_name else None, T[op.dst].data_ptr(), self._ws_ptr, stream)
             elif kind == "max":
                 B.ipool_max(T[op.src].data_ptr(), T[op.dst].data_ptr(), self.n, src.h, src.w, src.c,
                             op.k, op.stride, op.pad, stream)

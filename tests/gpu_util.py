@@ -32,6 +32,12 @@ class Fenced:
         return h[FENCE:FENCE + self.nbytes].view(self.np_dtype).reshape(self.shape).copy()
 
 
+def workspace_for(plan):
+    """A canary-fenced device buffer of exactly ``iconv_workspace_bytes(plan)`` bytes, or None."""
+    size = B.iconv_workspace_bytes(plan)
+    return Fenced((size,), np.uint8, 0xC3) if size else None
+
+
 def gpu_conv(X, W, b, mul, shift, h_i, *, stride=1, pad=0, in_dtype=B.U8, in_c_offset=0, c_in=None,
              out_dtype=B.U8, out_c_total=None, out_c_offset=0, brelu=True, out_lo=0, out_hi=255, out_zero=0,
              skip=None, skip_dtype=-1, skip_c_offset=0, skip_mul=1, skip_shift=0, kernel=B.KERNEL_AUTO,
@@ -54,8 +60,11 @@ def gpu_conv(X, W, b, mul, shift, h_i, *, stride=1, pad=0, in_dtype=B.U8, in_c_o
         xd = dev(X)
         sd = dev(skip) if skip is not None else None
         out = Fenced((n, ho, wo, out_c_total), _NP[out_dtype], fill)
+        ws = workspace_for(plan)
         B.iconv_forward(plan, xd.data_ptr(), sd.data_ptr() if sd is not None else None, out.ptr,
-                        torch.cuda.current_stream().cuda_stream)
+                        ws.ptr if ws is not None else None, torch.cuda.current_stream().cuda_stream)
+        if ws is not None:
+            ws.get()            # the canaries around the workspace must be intact
         B.iconv_check(torch.cuda.current_stream().cuda_stream)
         return out.get(), B.iconv_plan_kernel(plan)
     finally:

@@ -61,7 +61,7 @@ def test_plan_rejects_bad_descriptors_before_touching_the_gpu(over, status):
 
 def test_null_arguments():
     assert B.lib.iconv_plan(None, None) == B.ERR_ARG
-    assert B.lib.iconv_forward(None, None, None, None, None) == B.ERR_ARG
+    assert B.lib.iconv_forward(None, None, None, None, None, None) == B.ERR_ARG
     assert B.lib.iconv_plan_destroy(None) == B.OK
     assert B.lib.iadd_requant(None, None, None, None, None) == B.ERR_ARG
     assert B.lib.ipool_max(None, None, 1, 8, 8, 15, 3, 2, 1, None) == B.ERR_ALIGN
@@ -104,6 +104,28 @@ def test_mul_shift_and_brelu_params_match_oracle_planner():
             for k in ("h_ri", "mul", "shift", "h_i"):
                 assert got[k] == want[k], (k, h_rf, ry)
             assert got["ratio_V"] == want["ratio_V"] and got["h_f"] == want["h_f"]
+
+
+def test_brelu_params_bracket_follows_the_exact_product_like_the_oracle():
+    """Eq. 8 where the double product of the two arguments lands exactly on a tie while their exact
+    product does not: the library decides by the exact product (fused multiply-add residual), as
+    the oracle's rationals do."""
+    from fractions import Fraction
+    seen = set()
+    for k in range(1000, 1400):
+        for a in (3.0, 7.0, 1.1):
+            b = (k + 0.5) / a
+            if a * b != k + 0.5 or Fraction(a) * Fraction(b) == Fraction(2 * k + 1, 2):
+                continue
+            want = P.brelu_params(a, b, 255)
+            got = B.iq_brelu_params(a, b, 255)
+            assert got["h_ri"] == want["h_ri"] and got["mul"] == want["mul"] and got["h_i"] == want["h_i"], (a, b)
+            seen.add(want["h_ri"] - k)
+    assert seen == {0, 1}
+
+
+def test_no_tensor_core_device_table_entry_without_a_gpu_call():
+    assert B.iconv_device_initialised(63) == -1 and B.iconv_device_initialised(-5) == -1 and B.iconv_device_initialised(1000) == -1
 
 
 def test_bn_fold_matches_oracle_planner():

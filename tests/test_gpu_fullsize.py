@@ -2,8 +2,12 @@
 ``bench.py`` times (same plans, same batch, kernel family chosen by the plan).
 
 Images are independent units through every layer, so the oracle's forward of ONE image is the
-exact expectation for that image's slice of every tensor of the full-batch GPU run: the first
-and the last image of each batch are checked, every layer, bit for bit.  Parameters are the
+exact expectation for that image's slice of every tensor of the full-batch GPU run.  Persistent
+CTAs walk the 128-pixel tiles round-robin, so the images are picked from the tile schedule: the
+first and the last of the batch, the middle one, and two that sit where the last, partial wave
+of tiles begins in the deep stages (e.g. ResNet-50 at batch 256, stage 4: 196 tiles on 148 SMs,
+the partial wave starts inside image 193; ResNet-152 at batch 128, stage 3: inside image 120).
+Every layer of each is checked bit for bit.  Parameters are the
 cached ones of ``workloads/params`` (written by the oracle's calibration)."""
 import numpy as np
 import pytest
@@ -26,7 +30,7 @@ def test_full_size_configuration_matches_oracle_on_sampled_images(name):
     out = g.forward(torch.from_numpy(x).cuda())
     B.iconv_check(torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
-    for img in (0, net.n - 1):
+    for img in sorted({0, net.n // 2, (3 * net.n) // 4 + 1, (15 * net.n) // 16, net.n - 1}):
         want = ON.forward(net, params, x[img:img + 1])
         for op in net.ops:
             if op.name in g.fused:        # a fused projection's int32 tensor is never written

@@ -272,3 +272,130 @@ def test_avgpool_is_rounded_exact_mean():
             tot = int(x[n, :, :, c].astype(np.int64).sum())
             assert int(got[n, 0, 0, c]) == min(255, P.round_half_up(Fraction(tot * m, 1 << s)))
             assert abs(int(got[n, 0, 0, c]) - tot / 49.0) <= 1.0
+
+
+# ---------------------------------------------------------------- stand-alone add: both operands, zero points
+# Hand-computed rows (Sections 3.4.2, 4.1: both operands rescaled, then the convolution's tail).
+#   a' = [(A - a_zero) * mul_a / 2^sh_a],  b' = [(B - b_zero) * mul_b / 2^sh_b],  Y = a' + b',
+#   Y = clamp(Y, 0, h_i) if brelu,  V = [Y * mul / 2^shift],  out = clamp(V + out_zero, lo, hi)
+# (A, a_zero, mul_a, sh_a, B, b_zero, mul_b, sh_b, brelu, h_i, mul, shift, out_zero, lo, hi) -> out
+ADD_ROWS = [
+    # the second operand does all the work: 7*3/2 = 10.5 -> 11
+    ((0, 0, 1, 0, 7, 0, 3, 1, 0, 0, 1, 0, 0, -128, 127), 11),
+    # negative tie of the second operand: -7*3/2 = -10.5 -> -10 (ties go up)
+    ((0, 0, 1, 0, -7, 0, 3, 1, 0, 0, 1, 0, 0, -128, 127), -10),
+    # b_zero: (5 - 12) * 3 / 2 = -10.5 -> -10; a: (9 - 1) * 5 / 4 = 10 -> Y = 0
+    ((9, 1, 5, 2, 5, 12, 3, 1, 0, 0, 1, 0, 0, -128, 127), 0),
+    # a distinct shift for each operand: a' = [10*7/8] = [8.75] = 9, b' = [100*500/2^10] = [48.83] = 49; Y = 58
+    ((10, 0, 7, 3, 100, 0, 500, 10, 0, 0, 1, 0, 0, -128, 127), 58),
+    # ... then Eq. 4 with a tie: 58 * 3 / 4 = 43.5 -> 44, and a zero point of -40 -> 4
+    ((10, 0, 7, 3, 100, 0, 500, 10, 0, 0, 3, 2, -40, -128, 127), 4),
+    # negative Y with a tie in Eq. 4 and a positive zero point: a' = -9 (=[-8.75]), b' = [-48.83] = -49,
+    # Y = -58, V = [-43.5] = -43, out = -43 + 128 = 85
+    ((-10, 0, 7, 3, -100, 0, 500, 10, 0, 0, 3, 2, 128, 0, 255), 85),
+    # the same through BReLU: Y = -58 clamps to 0, V = 0, out = 128
+    ((-10, 0, 7, 3, -100, 0, 500, 10, 1, 1000, 3, 2, 128, 0, 255), 128),
+    # BReLU's upper bound acts on Y before Eq. 4: Y = 58 -> h_i = 50 -> [50*3/4] = [37.5] = 38, +out_zero 10 = 48
+    ((10, 0, 7, 3, 100, 0, 500, 10, 1, 50, 3, 2, 10, 0, 255), 48),
+    # saturation after the zero point: V = 44, out_zero = 250 -> 294 -> 255
+    ((10, 0, 7, 3, 100, 0, 500, 10, 0, 0, 3, 2, 250, 0, 255), 255),
+    # and at the lower end: V = -43, out_zero = 20 -> -23 -> lo = -5
+    ((-10, 0, 7, 3, -100, 0, 500, 10, 0, 0, 3, 2, 20, -5, 127), -5),
+    # operands swapped in role (a carries mul 500 / shift 10, b carries 7 / 3) give the same sum
+    ((100, 0, 500, 10, 10, 0, 7, 3, 0, 0, 1, 0, 0, -128, 127), 58),
+]
+
+
+def _add_one(row):
+    (A, az, ma, sa, Bv, bz, mb, sb, brelu, h_i, mul, shift, oz, lo, hi) = row
+    out_dtype = L.S8 if lo < 0 else L.U8
+    out, ovf = L.add_requant(np.array([A], np.int32), np.array([Bv], np.int32), a_dtype=L.I32, b_dtype=L.I32,
+                             out_dtype=out_dtype, a_zero=az, b_zero=bz, mul_a=ma, sh_a=sa, mul_b=mb, sh_b=sb,
+                             brelu=brelu, h_i=h_i, mul=mul, shift=shift, out_zero=oz, out_lo=lo, out_hi=hi)
+    assert not ovf
+    return int(out[0])
+
+
+@pytest.mark.parametrize("row,want", ADD_ROWS)
+def test_add_requant_hand_computed_rows(row, want):
+    assert _add_one(row) == want
+
+
+def test_add_requant_both_operands_against_exact_rationals():
+    """Every field of the descriptor varies (second operand's multiplier, shift and zero included);
+    the expected value is the definition in exact rationals, element by element."""
+    rng = np.random.default_rng(21)
+    for trial in range(40):
+        a_dtype = [L.U8, L.S8, L.I32][trial % 3]
+        b_dtype = [L.I32, L.U8, L.S8][(trial // 3) % 3]
+        n = 64
+        draw = {L.U8: lambda: rng.integers(0, 256, n).astype(np.uint8), L.S8: lambda: rng.integers(-128, 128, n).astype(np.int8),
+                L.I32: lambda: rng.integers(-300000, 300000, n).astype(np.int32)}
+        A, Bv = draw[a_dtype](), draw[b_dtype]()
+        az, bz = int(rng.integers(-3, 130)), int(rng.integers(-3, 130))
+        ma, mb = int(rng.integers(1, 2000)), int(rng.integers(1, 2000))
+        sa, sb = int(rng.integers(0, 12)), int(rng.integers(0, 12))
+        brelu = trial % 2
+        h_i = int(rng.integers(1, 400000))
+        mul, shift = int(rng.integers(1, 300)), int(rng.integers(0, 20))
+        oz = int(rng.integers(-100, 200))
+        signed = trial % 4 == 3
+        lo, hi = (-128 + int(rng.integers(0, 10)), 127 - int(rng.integers(0, 10))) if signed else (int(rng.integers(0, 10)), 255 - int(rng.integers(0, 10)))
+        out, ovf = L.add_requant(A, Bv, a_dtype=a_dtype, b_dtype=b_dtype, out_dtype=L.S8 if signed else L.U8, a_zero=az, b_zero=bz,
+                                 mul_a=ma, sh_a=sa, mul_b=mb, sh_b=sb, brelu=brelu, h_i=h_i, mul=mul, shift=shift,
+                                 out_zero=oz, out_lo=lo, out_hi=hi)
+        assert not ovf
+        for i in range(n):
+            y = P.round_half_up(Fraction((int(A[i]) - az) * ma, 1 << sa)) + P.round_half_up(Fraction((int(Bv[i]) - bz) * mb, 1 << sb))
+            if brelu:
+                y = min(max(y, 0), h_i)
+            v = P.round_half_up(Fraction(y * mul, 1 << shift)) + oz
+            assert int(out[i]) == min(max(v, lo), hi), (trial, i)
+
+
+def test_add_requant_operands_are_not_interchangeable_by_accident():
+    """A slip that uses one operand's shift, multiplier or zero for the other changes these sums."""
+    base = dict(a_dtype=L.I32, b_dtype=L.I32, out_dtype=L.S8, brelu=False, mul=1, shift=0, out_lo=-128, out_hi=127)
+    A, Bv = np.array([40], np.int32), np.array([24], np.int32)
+    # a' = [40 * 3 / 2^3] = 15, b' = [24 * 5 / 2^1] = 60
+    assert int(L.add_requant(A, Bv, mul_a=3, sh_a=3, mul_b=5, sh_b=1, **base)[0][0]) == 75
+    # with the shifts exchanged it would be 60 + 15 = 75 as well, so break the symmetry: zeros
+    # a' = [(40-8) * 3 / 8] = 12, b' = [(24-4) * 5 / 2] = 50
+    assert int(L.add_requant(A, Bv, a_zero=8, b_zero=4, mul_a=3, sh_a=3, mul_b=5, sh_b=1, **base)[0][0]) == 62
+    # b_zero dropped would give 12 + 60 = 72; a_zero used for b would give 12 + 40 = 52; sh_a for b: 12 + [20*5/8] = 12 + 13 = 25
+
+
+def test_conv_out_zero_exact():
+    """Zero point and saturation of a convolution output (the regression networks' last layer)
+    against hand-computed values: one pixel, one channel, K = 2."""
+    X = np.array([[[[10, 200]]]], dtype=np.uint8)
+    W = np.array([[[[3, -1]]]], dtype=np.int8)
+    # U = 30 - 200 = -170, Y = U + 50 = -120, no BReLU, V = [-120 * 3 / 8] = [-45] = -45
+    for oz, lo, hi, want in ((128, 0, 255, 83), (0, 0, 255, 0), (300, 0, 255, 255), (45, 0, 255, 0), (46, 0, 255, 1), (40, 7, 255, 7)):
+        out, ovf = L.conv(X, W, [50], [3], [3], [0], brelu=False, out_zero=oz, out_lo=lo, out_hi=hi)
+        assert not ovf and int(out[0, 0, 0, 0]) == want, (oz, lo, hi)
+    # a tie below zero: Y = -121 -> -363/8 = -45.375 -> -45; Y = -124 -> -46.5 -> -46 (ties go up)
+    out, _ = L.conv(X, W, [46], [3], [3], [0], brelu=False, out_zero=128, out_lo=0, out_hi=255)
+    assert int(out[0, 0, 0, 0]) == 128 - 46
+    # RAW128 input: x = raw - 128 = (-118, 72): U = -354 - 72 = -426, Y = -426 + 426 = 0 -> out_zero
+    out, _ = L.conv(X, W, [426], [3], [3], [0], brelu=False, in_dtype=L.U8_RAW128, out_zero=128, out_lo=0, out_hi=255)
+    assert int(out[0, 0, 0, 0]) == 128
+
+
+# ---------------------------------------------------------------- Eq. 8: the bracket of the exact product
+def test_eq8_bracket_is_taken_of_the_exact_product():
+    """Pairs (h_rf, ratio_Y) whose product, rounded to a double, lands exactly on k + 0.5 while the
+    exact product lies just beside it: the bracket follows the exact product."""
+    below = above = 0
+    for k in range(1000, 1400):
+        b = (k + 0.5) / 3.0
+        if 3.0 * b != k + 0.5:
+            continue
+        exact = Fraction(3) * Fraction(b)
+        if exact == Fraction(2 * k + 1, 2):
+            continue
+        want = k + 1 if exact > Fraction(2 * k + 1, 2) else k
+        assert P.brelu_params(3.0, b, 255)["h_ri"] == want
+        below += want == k
+        above += want == k + 1
+    assert below > 5 and above > 5
