@@ -13,7 +13,8 @@ OBJ_DIR = os.path.join(_HERE, "_build")
 PROBE_SRC = os.path.join(_HERE, "bench_probe", "probe_mma.cu")
 PROBE_LIB = os.path.join(_HERE, "libiconv_probe.so")
 SOURCES = ["iconv_api.cu", "plan.cu", "kernels_direct.cu", "kernel_thin.cu", "kernel_umma.cu", "kernel_stem.cu",
-           "kernel_calib.cu", "planner.cpp"]
+           "kernel_calib.cu", "planner.cpp"] + ["umma_inst_conv%d.cu" % e for e in range(8)] + \
+          ["umma_inst_window%d.cu" % e for e in (2, 3, 4, 5, 8)]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-diag-suppress", "128", "-Xcompiler", "-fPIC",
          "-Xcompiler", "-fvisibility=hidden", "-I", INCLUDE, "-I", CSRC]
 
@@ -31,8 +32,7 @@ def _stale(target: str, deps) -> bool:
 
 def _compile(src: str, obj: str, verbose: bool):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    # -split-compile: the optimiser works on a translation unit's kernels in parallel
-    cmd = [nvcc] + FLAGS + ["-split-compile", "0", "-c", src, "-o", obj]
+    cmd = [nvcc] + FLAGS + ["-c", src, "-o", obj]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     subprocess.run(cmd, check=True)
@@ -49,6 +49,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         src, obj = os.path.join(CSRC, s), os.path.join(OBJ_DIR, s + ".o")
         if force or _stale(obj, [src] + headers):
             jobs.append((src, obj))
+    jobs.sort(key=lambda j: -os.path.getsize(j[0]) if "umma_inst" not in j[0] else -10 ** 9)   # the kernel instances first: they take longest
     with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as ex:
         for f in [ex.submit(_compile, src, obj, verbose) for src, obj in jobs]:
             f.result()

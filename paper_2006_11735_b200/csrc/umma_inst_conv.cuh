@@ -1,0 +1,27 @@
+// Body of one im2col-kernel translation unit: define ICONV_INST_EPI (0..7) before including.
+#include "umma_inst.h"
+
+namespace iconv {
+
+#define ICONV_CAT2(a, b) a##b
+#define ICONV_CAT(a, b) ICONV_CAT2(a, b)
+
+cudaError_t ICONV_CAT(umma_conv_launch_, ICONV_INST_EPI)(int issue, const UmmaLaunch &l)
+{
+    constexpr int E = ICONV_INST_EPI;
+    if (issue == 1) umma_conv_kernel<E, 1><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
+    else if (issue == 2) umma_conv_kernel<E, 2><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
+    else umma_conv_kernel<E, 0><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
+    return cudaGetLastError();
+}
+
+cudaError_t ICONV_CAT(umma_conv_opt_in_, ICONV_INST_EPI)()
+{
+    constexpr int E = ICONV_INST_EPI;
+    cudaError_t e = cudaFuncSetAttribute(umma_conv_kernel<E, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_conv_kernel<E, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_conv_kernel<E, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM);
+    return e;
+}
+
+}  // namespace iconv
