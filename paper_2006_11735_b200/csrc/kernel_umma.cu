@@ -168,7 +168,7 @@ int choose_projection_epilogue(const iconv_desc &d, int c_out_pad, std::vector<i
     // The fast form (no explicit BReLU clamp, as EPI_FAST): per-layer parameters, a plain u8 output
     // whose bound h_i already maps to 255, and |Y| * mul + half < 2^31 for the worst case of both
     // reductions with the layer's actual weights.
-    if (proj32 && !d.per_channel && tail_free && d.out_dtype == ICONV_U8 && d.out_hi == 255 && d.brelu) {
+    if (proj32 && !d.per_channel && tail_free && d.out_dtype == ICONV_U8 && d.out_hi == 255 && d.brelu && d.skip_shift == FAST_SKIP_SHIFT) {
         const long long mul = d.mul[0], qhalf = 1ll << (d.shift[0] - 1);
         bool fast = (long long)(((unsigned long long)d.h_i[0] * (unsigned long long)mul + (unsigned long long)qhalf) >> d.shift[0]) >= 255;
         const long long xmax = d.in_dtype == ICONV_U8 ? 255 : 128;
@@ -262,7 +262,8 @@ int choose_epilogue(const iconv_desc &d, int c_out_pad, std::vector<int32_t> &c_
                     const int q = d.per_channel ? co : 0;
                     c_a[co] = (int32_t)((long long)d.bias[co] * d.mul[q] + (1ll << (d.shift[q] - 1)));
                 }
-            return skip8 ? EPI_FAST_SKIP8 : EPI_FAST;
+            if (!skip8) return EPI_FAST;
+            if (d.skip_shift == FAST_SKIP_SHIFT) return EPI_FAST_SKIP8;     // the clamp-free skip form is compiled for this shift only
         }
     }
     if (d.skip_dtype < 0) return EPI_SAFE;
@@ -469,7 +470,7 @@ int umma_geometry(iconv_plan_t *p)
     // staging per epilogue warp: 8-bit pieces are 2 KB each, and only an 8-bit skip (not a fused
     // projection's operand) is staged behind them
     const bool stage_skip = d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && !proj;
-    p->epi_warp_bytes = (d.out_dtype == ICONV_I32 || stage_skip) ? EPI_WARP_SMEM : EPI_WARP_SMEM_SMALL;
+    p->epi_warp_bytes = stage_skip ? EPI_WARP_SMEM_SKIP : (d.out_dtype == ICONV_I32 ? EPI_WARP_SMEM : EPI_WARP_SMEM_SMALL);
     for (int ew = (weight >= 100 ? 16 : 8); ew >= 8 && !p->epi_warps; ew -= 8) {
         const int avail = MAX_SMEM - fixed - ew * p->epi_warp_bytes;
         const int want = 2;

@@ -45,8 +45,11 @@ constexpr int MMA_WARP = NUM_PRODUCERS;
 constexpr int MMA_WARP2 = 1;           // window mode (one TMA warp): a second MMA issuer
 constexpr int EPI_WARP0 = 4;              // first epilogue warp (a multiple of 4: warp % 4 is its TMEM lane quadrant)
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS_MAX);
-constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces of up to 4 KB together, then the skip rows of one tile
+constexpr int FAST_SKIP_SHIFT = 8;         // the skip shift the clamp-free epilogue forms are compiled for (what iq_skip_sync yields unless the skip is scaled down a lot)
+constexpr int SKIP_RING = 3;              // staged skip pieces per epilogue warp: the load of a piece is issued SKIP_RING - 1 pieces ahead of its use
+constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces of up to 4 KB together (int32 outputs)
 constexpr int EPI_WARP_SMEM_SMALL = 4096; // ... when the output is 8-bit (pieces of 2 KB) and no 8-bit skip is staged
+constexpr int EPI_WARP_SMEM_SKIP = 4096 + SKIP_RING * 2048;   // 8-bit output pieces and the ring of 8-bit skip pieces behind them
 constexpr int MAX_STAGES = 12;
 constexpr int MAX_TMEM_BUFS = 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds at the boost clock
@@ -188,31 +191,29 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// The wait of an epilogue warp, taken by one lane on behalf of the warp (32 lanes polling one
-// barrier word only add shared-memory traffic).  These warps are the critical path of the
-// epilogue-bound layers, so they poll (with a back-off) rather than suspend; __syncwarp
-// orders the other lanes' later reads after lane 0's acquire.
+// The wait of an epilogue warp.  Every lane probes the barrier itself (so each has its own acquire
+// and no vote or shuffle is needed on the common path): one plain probe, then probes that suspend
+// the warp in hardware until the phase completes or the hint runs out -- a suspended warp takes no
+// issue slots from the warps that are doing arithmetic on the same scheduler, which a polling
+// loop does.  The limit is counted on the SM's cycle counter, read every 16 failed probes.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane,
                                                long long limit = WAIT_LIMIT_CYCLES)
 {
-    int ok = 1;
-    if (lane == 0) {
-        ok = 0;
-        long long t0 = 0;
-        for (uint32_t i = 0;; ++i) {
-            if (mbar_test_wait(bar, parity)) { ok = 1; break; }
-            if (i >= 8) __nanosleep(32);
-            if ((i & 1023u) == 1023u) {
-                if (*abort_flag) break;
-                const long long now = clock64();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > limit) break;
-            }
+    (void)lane;
+    if (mbar_test_wait(bar, parity)) return true;
+    bool ok = true;
+    long long t0 = 0;
+#pragma unroll 1
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity, 1000u)) break;
+        if ((i & 15u) == 0) {
+            if (*abort_flag) { ok = false; break; }
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit) { ok = false; break; }
         }
     }
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    __syncwarp();
-    return ok != 0;
+    return __all_sync(0xffffffffu, ok) != 0;
 }
 
 __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w,
@@ -358,6 +359,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int *r)
         : "r"(taddr)
         : "memory");
 }
+// The load and the wait for it in one statement: the sixteen values are ready when it returns.
+// The epilogue keeps no second load in flight (measured: with sixteen epilogue warps the other
+// warps of the scheduler cover the TMEM latency, and the second register block a prefetch needs
+// cost more -- spills and moves -- than the overlap returned: 64 -> 256 1x1 with skip, batch 256,
+// 108 us with the next group's load in flight, 95 us without).
+__device__ __forceinline__ void tmem_ld16_sync(uint32_t taddr, int *r, uint4 dep = make_uint4(0, 0, 0, 0))
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr), "r"(dep.x), "r"(dep.y), "r"(dep.z), "r"(dep.w)    // dep: values that must exist before the registers are reloaded
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // d = { sat8(v3), sat8(v2), sat8(v1), sat8(v0) } (v0 in the low byte), unsigned or signed saturation
@@ -376,7 +392,7 @@ __device__ __forceinline__ unsigned pack4_sat(int v0, int v1, int v2, int v3)
 }
 
 struct Shared {
-    unsigned long long skip_full[EPI_WARPS_MAX];
+    unsigned long long skip_full[EPI_WARPS_MAX][SKIP_RING];
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
     unsigned long long tmem_full[MAX_TMEM_BUFS];
@@ -406,7 +422,11 @@ struct EpiScalars {
 __device__ __forceinline__ EpiScalars epi_scalars(const ConvArgs &a, const UmmaArgs &u)
 {
     EpiScalars e;
-    e.q_mul = u.q_mul; e.q_shift = u.q_shift; e.q_half = u.q_half; e.q_h = u.q_h;
+    e.q_mul = u.q_mul; e.q_shift = u.q_shift; e.q_h = u.q_h;
+    // y * q_mul + q_half has two warp-uniform operands and the multiply-add takes only one from a
+    // uniform register: left to itself the compiler re-creates the other in a vector register for
+    // every element (one move per output).  An opaque move pins q_half in a vector register.
+    asm volatile("mov.b32 %0, %1;" : "=r"(e.q_half) : "r"(u.q_half));
     e.skip_mul = a.skip_mul; e.skip_shift = a.skip_shift; e.skip_xor = u.skip_xor;
     e.out_zero = a.out_zero; e.out_lo = a.out_lo; e.out_hi = a.out_hi; e.tail = u.tail;
     e.per_channel = a.per_channel && !u.group_uniform; e.group_uniform = u.group_uniform; e.proj32 = u.proj32; e.brelu = a.brelu; e.skip_dtype = a.skip_dtype;
@@ -479,7 +499,9 @@ __device__ __forceinline__ void epilogue16_pc(const int *acc, const int *accp, i
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const int sv = (int)__byte_perm(w4[k >> 2], 0, 0x4440 + (k & 3));
-            const int y = acc[k] + ((sv * s.skip_mul + ca[k]) >> s.skip_shift);
+            // (the fast form is planned only for the usual skip shift of 8: as an immediate, shift and add
+            // become one instruction)
+            const int y = acc[k] + ((sv * s.skip_mul + ca[k]) >> (EPI == EPI_FAST_SKIP8 ? FAST_SKIP_SHIFT : s.skip_shift));
             if (EPI == EPI_FAST_SKIP8) {
                 V[k] = (y * s.q_mul + s.q_half) >> s.q_shift;
             } else {
@@ -494,10 +516,11 @@ __device__ __forceinline__ void epilogue16_pc(const int *acc, const int *accp, i
         // Y = U + ((accp * skip_mul + C) >> skip_shift), C = b_p * skip_mul + 2^(skip_shift-1) + (b << skip_shift);
         // otherwise the rescale runs in 64 bits with the two biases apart.
         if (!PC && s.proj32 == 2) {
-            // as EPI_FAST: no clamp before Eq. 4, the u8 saturation that follows stands for both (proven at plan time)
+            // as EPI_FAST: no clamp before Eq. 4, the u8 saturation that follows stands for both (proven at
+            // plan time, and planned only for the usual skip shift of 8)
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
-                const int y = acc[k] + ((accp[k] * s.skip_mul + ca[k]) >> s.skip_shift);
+                const int y = acc[k] + ((accp[k] * s.skip_mul + ca[k]) >> FAST_SKIP_SHIFT);
                 V[k] = (y * s.q_mul + s.q_half) >> s.q_shift;
             }
         } else if (s.proj32) {
@@ -602,7 +625,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             mbar_init(smem_u32(&sh->tmem_full[b]), 1);
             mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)(4 * u.cs));
         }
-        for (int w = 0; w < EPI_WARPS_MAX; ++w) mbar_init(smem_u32(&sh->skip_full[w]), 1);
+        for (int w = 0; w < EPI_WARPS_MAX * SKIP_RING; ++w) mbar_init(smem_u32(&sh->skip_full[0][0]) + 8u * (uint32_t)w, 1);
         mbar_init(smem_u32(&sh->b_full), 1);
         mbar_init(smem_u32(&sh->drain), 1);
         sh->abort_flag = 0;
@@ -617,7 +640,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     int last_stage = -1;   // producer: stage and phase of the last load this warp issued
     uint32_t last_parity = 0;
     int b_issued = 0;      // producer: resident filter bank requested
-    int skip_issued = 0;   // epilogue lane 0: skip prefetches issued
+    int skip_issued = 0, skip_taken = 0;   // epilogue lane 0: skip pieces requested / waited for
 
     if (warp < NUM_PRODUCERS) {
         // ---------------------------------------------------------------- TMA producers
@@ -832,34 +855,44 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int turn = slot / u.cs;
         const int col_lo = part * u.part_n;
         const int ncols = min(u.block_n - col_lo, u.part_n);
-        uint8_t *obuf = epi_smem + (size_t)ew * u.epi_warp_bytes;     // two pieces of 32 rows x piece_bytes
-        uint8_t *sbuf = obuf + EPI_WARP_SMEM / 2;                     // skip rows of one tile (8-bit variants)
-        const uint32_t skip_bar = smem_u32(&sh->skip_full[ew]);
         constexpr int esz = (EPI == EPI_RAW) ? 4 : 1;
         const int esz_rt = (EPI == EPI_WIDE && a.out_dtype == ICONV_I32) ? 4 : esz;
         const int pb = u.piece_bytes;
         const int pcols = pb / esz_rt;                                // columns per staged piece
         const int piece_smem = 32 * pb;
+        const uint32_t obuf = smem_u32(epi_smem + (size_t)ew * u.epi_warp_bytes);   // two output pieces of 32 rows x piece_bytes
+        const uint32_t sbuf = obuf + 2u * (uint32_t)piece_smem;                      // ring of SKIP_RING skip pieces (8-bit skip variants)
+        const uint32_t skip_bar0 = smem_u32(&sh->skip_full[ew][0]);
         const int swz_shift = pb == 128 ? 0 : (pb == 64 ? 1 : 2);
         const unsigned row_off = (unsigned)lane * (unsigned)pb;
-        const unsigned row_swz = pb >= 32 ? (((unsigned)lane >> swz_shift) & (unsigned)(pb / 16 - 1)) : 0u;
+        const unsigned row_swz16 = pb >= 32 ? ((((unsigned)lane >> swz_shift) & (unsigned)(pb / 16 - 1)) << 4) : 0u;   // XOR mask of the row's 16-byte chunks
         const int tile_step = u.bi * (int)gridDim.x;
         const EpiScalars es = epi_scalars(a, u);
-        int mine = 0, pieces = 0;
+        int pieces = 0;
         bool ok = true;
 
-        // first skip prefetch
-        if (SKIP8 && lane == 0 && (int)blockIdx.x + turn * (int)gridDim.x < num_tiles) {
-            const int tile0 = blockIdx.x + turn * gridDim.x;
-            const int mt0 = (int)fast_div((unsigned)tile0, u.div_nt_mul, u.div_nt_shr);
-            mbar_expect_tx(skip_bar, (uint32_t)(32 * ncols));
-            for (int c = 0; c < ncols; c += pcols)
-                tma_load_2d(smem_u32(sbuf + (size_t)(c / pcols) * piece_smem), &tmap_skip, skip_bar,
-                            (tile0 - mt0 * u.n_tiles) * u.block_n + col_lo + c, mt0 * BLOCK_M + quad * 32);
-            skip_issued = 1;
-        }
+        // The 8-bit skip operand arrives by TMA, piece by piece (32 pixels x piece_bytes), into a ring of
+        // SKIP_RING buffers: the load of a piece is issued when the piece SKIP_RING places before it has
+        // been consumed, i.e. two pieces of epilogue work ahead of its use, which covers the DRAM latency.
+        // (pf_tile, pf_pc): the next piece to request; lane 0 only.
+        int pf_tile = (int)blockIdx.x + turn * (int)gridDim.x, pf_pc = 0;
+        auto request_skip_piece = [&](int ring_slot) {
+            if (pf_tile >= num_tiles) return;
+            const int mt = (int)fast_div((unsigned)pf_tile, u.div_nt_mul, u.div_nt_shr);
+            const uint32_t bar = skip_bar0 + 8u * (uint32_t)ring_slot;
+            mbar_expect_tx(bar, (uint32_t)piece_smem);
+            tma_load_2d(sbuf + (uint32_t)(ring_slot * piece_smem), &tmap_skip, bar, (pf_tile - mt * u.n_tiles) * u.block_n + col_lo + pf_pc,
+                        mt * BLOCK_M + quad * 32);
+            ++skip_issued;
+            pf_pc += pcols;
+            if (pf_pc >= ncols) { pf_pc = 0; pf_tile += tile_step; }
+        };
+        if (SKIP8 && lane == 0)
+            for (int r = 0; r < SKIP_RING; ++r) request_skip_piece(r);
+        int ring = 0;
+        uint32_t ring_parity = 0;
 
-        for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles && ok; t += u.bi, tile += tile_step, ++mine) {
+        for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles && ok; t += u.bi, tile += tile_step) {
             const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
             const int n_tile = tile - m_tile * u.n_tiles;
             const int buf = t & (u.nbuf - 1);
@@ -869,20 +902,16 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 break;
             }
             tc_fence_after();
-            if (SKIP8) {
-                if (!mbar_wait_warp(skip_bar, (uint32_t)(mine & 1), &sh->abort_flag, lane)) {
-                    give_up(sh, u.status, 5);
-                    break;
-                }
-            }
             const long long m = (long long)m_tile * BLOCK_M + quad * 32 + lane;
             const bool row_ok = m < u.m_total;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.acc_cols + col_lo);
+            int acc[16], accp[16];
+            uint4 o_prev = make_uint4(0, 0, 0, 0);       // the packed outputs of the group before: the reload of acc is ordered after them
 
-            for (int pc = 0, piece = 0; pc < ncols; pc += pcols, ++pieces, ++piece) {
-                uint8_t *ob = obuf + (size_t)(pieces & 1) * piece_smem;
-                const uint32_t ob_row = smem_u32(ob) + row_off;                                  // this lane's staged output row
-                const uint32_t sk_row = smem_u32(sbuf) + (uint32_t)(piece * piece_smem) + row_off;   // and its staged skip row
+            for (int pc = 0; pc < ncols && ok; pc += pcols, ++pieces) {
+                const uint32_t ob = obuf + (uint32_t)((pieces & 1) * piece_smem);
+                const uint32_t ob_row = ob + row_off;                                              // this lane's staged output row
+                const uint32_t sk_row = sbuf + (uint32_t)(ring * piece_smem) + row_off;            // and its staged skip row
                 const int4 *cap = (const int4 *)(u.c_a + n0 + pc);
                 const uint32_t t_piece = t_row + (uint32_t)pc;
                 // the store issued two pieces ago must have finished reading this buffer
@@ -890,79 +919,72 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                 }
-                // 16 columns at a time, the TMEM load of the next group in flight while this one is
-                // worked on; each group's constants and skip bytes are fetched before the wait
-                const int ngroups = pcols >> 4;
-                // (the variants that hold a second accumulator or 64-bit temporaries do not prefetch:
-                // they would spill)
-                constexpr bool PIPE = EPI != EPI_PROJ && EPI != EPI_SAFE_SKIP32 && EPI != EPI_WIDE;
-                int accA[16], accB[16], accpA[16];
-                if (PIPE) tmem_ld16(t_piece, accA);
-                for (int gi = 0; gi < ngroups; gi += 2) {
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        const int gcur = gi + hf;
-                        if (gcur >= ngroups) break;
-                        const int cc = gcur << 4;
-                        const int co0 = n0 + pc + cc;
-                        const uint32_t goff = ((unsigned)gcur ^ row_swz) << 4;       // swizzled 16-byte chunk of the row
-                        if (!PIPE) {
-                            tmem_ld16(t_piece + (uint32_t)cc, accA);
-                            if (EPI == EPI_PROJ) tmem_ld16(t_piece + (uint32_t)(u.block_n + cc), accpA);
-                        }
-                        int4 ca[4];
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + 4 * gcur + g);
-                        uint4 sk = make_uint4(0, 0, 0, 0);
-                        if (SKIP8) sk = lds128(sk_row + goff);
-                        tmem_ld_wait();
-                        if (PIPE && gcur + 1 < ngroups) tmem_ld16(t_piece + (uint32_t)(cc + 16), hf ? accA : accB);
-                        int V[16];
-                        epilogue16<EPI>((PIPE && hf) ? accB : accA, accpA, V, ca, co0, m, row_ok, sk, es, a, u);
-                        if (esz_rt == 4) {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g) {
-                                const unsigned chunk = (unsigned)((cc >> 2) + g);     // 4 columns = 16 bytes
-                                *(int4 *)(ob + row_off + ((chunk ^ row_swz) << 4)) = make_int4(V[4 * g], V[4 * g + 1], V[4 * g + 2], V[4 * g + 3]);
-                            }
-                        } else {
-                            uint4 o;
-                            if (EPI == EPI_FAST || EPI == EPI_FAST_SKIP8 || a.out_dtype == ICONV_U8) {
-                                o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
-                                o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
-                            } else {
-                                o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
-                                o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
-                            }
-                            sts128(ob_row + goff, o);
-                        }
+                if (SKIP8) {
+                    if (!mbar_wait_warp(skip_bar0 + 8u * (uint32_t)ring, ring_parity, &sh->abort_flag, lane)) {
+                        give_up(sh, u.status, 5);
+                        ok = false;
+                        break;
                     }
+                    if (lane == 0) ++skip_taken;
+                }
+                // 16 columns at a time: the group's constants and skip bytes are requested, then the
+                // accumulators are read (load and wait together), worked on and staged.  The usual piece
+                // (four groups) is straight-line code.
+                auto group = [&](int gcur) {
+                    const int cc = gcur << 4;
+                    const int co0 = n0 + pc + cc;
+                    const uint32_t goff = (uint32_t)cc ^ row_swz16;                 // swizzled 16-byte chunk of the row (8-bit rows)
+                    int4 ca[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + 4 * gcur + g);
+                    uint4 sk = make_uint4(0, 0, 0, 0);
+                    if (SKIP8) sk = lds128(sk_row + goff);
+                    if (EPI == EPI_PROJ) tmem_ld16(t_piece + (uint32_t)(u.block_n + cc), accp);
+                    tmem_ld16_sync(t_piece + (uint32_t)cc, acc, o_prev);
+                    int V[16];
+                    epilogue16<EPI>(acc, accp, V, ca, co0, m, row_ok, sk, es, a, u);
+                    if (esz_rt == 4) {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)      // 4 columns = 16 bytes; 128-byte rows
+                            sts128(ob_row + ((uint32_t)((cc << 2) + (g << 4)) ^ row_swz16), make_uint4((unsigned)V[4 * g], (unsigned)V[4 * g + 1], (unsigned)V[4 * g + 2], (unsigned)V[4 * g + 3]));
+                    } else {
+                        uint4 o;
+                        if (EPI == EPI_FAST || EPI == EPI_FAST_SKIP8 || es.out_dtype == ICONV_U8) {
+                            o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
+                            o.z = pack4_sat<false>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<false>(V[12], V[13], V[14], V[15]);
+                        } else {
+                            o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
+                            o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
+                        }
+                        sts128(ob_row + goff, o);
+                        o_prev = o;
+                    }
+                };
+                const int ngroups = pcols >> 4;
+                if (ngroups == 4) {
+                    group(0); group(1); group(2); group(3);
+                } else if (ngroups == 2) {
+                    group(0); group(1);
+                } else {
+                    for (int gi = 0; gi < ngroups; ++gi) group(gi);
                 }
                 // hand the staged piece to the TMA unit (the store clips rows beyond the last
-                // pixel and columns beyond c_out)
+                // pixel and columns beyond c_out); the skip piece just consumed makes room for the
+                // one SKIP_RING places on
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) {
                     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                 ::"l"(&tmap_out), "r"(smem_u32(ob)), "r"(n0 + pc), "r"(m_tile * BLOCK_M + quad * 32)
+                                 ::"l"(&tmap_out), "r"(ob), "r"(n0 + pc), "r"(m_tile * BLOCK_M + quad * 32)
                                  : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    if (SKIP8) request_skip_piece(ring);
                 }
+                if (SKIP8 && ++ring == SKIP_RING) { ring = 0; ring_parity ^= 1u; }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
-                const int next = tile + tile_step;
-                if (SKIP8 && next < num_tiles) {     // prefetch the next tile's skip rows
-                    const int mtn = (int)fast_div((unsigned)next, u.div_nt_mul, u.div_nt_shr);
-                    mbar_expect_tx(skip_bar, (uint32_t)(32 * ncols));
-                    for (int c = 0; c < ncols; c += pcols)
-                        tma_load_2d(smem_u32(sbuf + (size_t)(c / pcols) * piece_smem), &tmap_skip, skip_bar,
-                                    (next - mtn * u.n_tiles) * u.block_n + col_lo + c, mtn * BLOCK_M + quad * 32);
-                    ++skip_issued;
-                }
-            }
+            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         __syncwarp();
@@ -988,8 +1010,9 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             umma_commit(smem_u32(&sh->drain));
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }
-        if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps && lane == 0 && skip_issued > 0)
-            mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0]), (uint32_t)((skip_issued - 1) & 1), &never);
+        if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps && lane == 0)
+            for (int j = skip_taken; j < skip_issued; ++j)      // skip pieces requested and not yet waited for (at most SKIP_RING)
+                mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0][j % SKIP_RING]), (uint32_t)((j / SKIP_RING) & 1), &never);
         __syncthreads();
     }
     if (warp == MMA_WARP) {
