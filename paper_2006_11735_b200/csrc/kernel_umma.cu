@@ -470,21 +470,32 @@ int umma_geometry(iconv_plan_t *p)
     // staging per epilogue warp: 8-bit pieces are 2 KB each, and only an 8-bit skip (not a fused
     // projection's operand) is staged behind them
     const bool stage_skip = d.skip_dtype >= 0 && d.skip_dtype != ICONV_I32 && !proj;
-    p->epi_warp_bytes = stage_skip ? EPI_WARP_SMEM_SKIP : (d.out_dtype == ICONV_I32 ? EPI_WARP_SMEM : EPI_WARP_SMEM_SMALL);
-    for (int ew = (weight >= 100 ? 16 : 8); ew >= 8 && !p->epi_warps; ew -= 8) {
-        const int avail = MAX_SMEM - fixed - ew * p->epi_warp_bytes;
+    // Candidates in order of preference: sixteen warps with the full skip ring, sixteen with a ring of
+    // two pieces (the load of a piece then leads its use by one piece instead of two), eight warps.
+    const int first_ew = weight >= 100 ? 16 : 8;
+    int cand[3][2], n_cand = 0;
+    cand[n_cand][0] = first_ew; cand[n_cand++][1] = SKIP_RING;
+    if (stage_skip) { cand[n_cand][0] = first_ew; cand[n_cand++][1] = 2; }
+    if (first_ew != 8) { cand[n_cand][0] = 8; cand[n_cand++][1] = SKIP_RING; }
+    for (int ci = 0; ci < n_cand && !p->epi_warps; ++ci) {
+        const int ew = cand[ci][0], ring = cand[ci][1];
+        const int warp_bytes = stage_skip ? 4096 + ring * 2048 : (d.out_dtype == ICONV_I32 ? EPI_WARP_SMEM : EPI_WARP_SMEM_SMALL);
+        const int avail = MAX_SMEM - fixed - ew * warp_bytes;
         const int want = 2;
+        const bool last = ci == n_cand - 1;
         int room = 0, slot = 0;
         if (bank <= RESIDENT_B_MAX && avail - (int)bank >= want * stage_a) {
             p->resident_b = 1;
             room = avail - (int)bank;
             slot = stage_a;
-        } else if (avail >= want * (stage_a + b_tile) || ew == 8) {
+        } else if (avail >= want * (stage_a + b_tile) || last) {
             room = avail;
             slot = stage_a + b_tile;
         }
         if (slot) {
             p->epi_warps = ew;
+            p->skip_ring = ring;
+            p->epi_warp_bytes = warp_bytes;
             for (int kg = k_iters < 8 ? k_iters : 8; kg >= 1; --kg)
                 if (kg * slot <= 48 * 1024 && room / (kg * slot) >= 3) { p->kg = kg; break; }
             p->stages = room / (p->kg * slot);
@@ -495,11 +506,17 @@ int umma_geometry(iconv_plan_t *p)
 
     // epilogue geometry: slots per TMEM lane quadrant, split between a tile's columns (cs)
     // and tiles in flight (bi)
+    // Twice as many accumulator buffers as tiles in flight: a group of warps that finishes a tile
+    // finds the next one computed already, and the MMAs of the tile after that (into the buffer just
+    // released) run under its epilogue.  With as many tiles in flight as buffers every group waited
+    // for its own buffer's next MMA round after every tile (a quarter to half of its time on the
+    // block-closing layers).
     const int slots = p->epi_warps / 4;
-    p->bi = slots < p->nbuf ? slots : p->nbuf;
+    p->bi = p->nbuf / 2 < slots ? p->nbuf / 2 : slots;
+    if (p->bi < 1) p->bi = 1;
     p->cs = slots / p->bi;
     while (p->cs > 1 && p->block_n < 32 * p->cs) p->cs /= 2;     // at least 32 columns per warp
-    if (p->block_n > 128 && p->cs < 2) { p->cs = 2; p->bi = slots / 2 ? slots / 2 : 1; if (p->bi > p->nbuf) p->bi = p->nbuf; }
+    if (p->block_n > 128 && p->cs < 2) p->cs = 2;
     p->epi_warps = 4 * p->cs * p->bi;
     p->half_n = p->cs > 1 ? (p->block_n / p->cs + 15) / 16 * 16 : p->block_n;
     {
@@ -794,6 +811,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.part_n = p->half_n;
     u.piece_bytes = p->piece_bytes;
     u.epi_warp_bytes = p->epi_warp_bytes;
+    u.skip_ring = p->skip_ring;
     // instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, N/8, M/16
     u.idesc = (2u << 4) | ((d.in_dtype == ICONV_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(p->block_n >> 3) << 17) |
               ((unsigned)(BLOCK_M >> 4) << 24);

@@ -32,6 +32,7 @@ struct iconv_plan_s {
     int tail = 1;            // 0: zero point and output range are provably no-ops
     int q_mul = 1, q_shift = 0, q_h = 0; // per-layer Eq. 4 / BReLU scalars
     int epi_warp_bytes = 8192;           // staging memory per epilogue warp (im2col kernel)
+    int skip_ring = 3;                   // staged 8-bit skip pieces per epilogue warp (2 or 3)
     int group_uniform = 0;               // per-channel parameters equal within every 16-channel group
     int pair16 = 0;                      // internal (stem): 16-channel positions read in pairs, two taps per K step
     // stem path: the plan of the GEMM that follows the repack, and the size of the repacked image,

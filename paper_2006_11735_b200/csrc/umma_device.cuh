@@ -46,10 +46,9 @@ constexpr int MMA_WARP2 = 1;           // window mode (one TMA warp): a second M
 constexpr int EPI_WARP0 = 4;              // first epilogue warp (a multiple of 4: warp % 4 is its TMEM lane quadrant)
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS_MAX);
 constexpr int FAST_SKIP_SHIFT = 8;         // the skip shift the clamp-free epilogue forms are compiled for (what iq_skip_sync yields unless the skip is scaled down a lot)
-constexpr int SKIP_RING = 3;              // staged skip pieces per epilogue warp: the load of a piece is issued SKIP_RING - 1 pieces ahead of its use
+constexpr int SKIP_RING = 3;              // staged skip pieces per epilogue warp at most: the load of a piece is issued ring - 1 pieces ahead of its use
 constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces of up to 4 KB together (int32 outputs)
 constexpr int EPI_WARP_SMEM_SMALL = 4096; // ... when the output is 8-bit (pieces of 2 KB) and no 8-bit skip is staged
-constexpr int EPI_WARP_SMEM_SKIP = 4096 + SKIP_RING * 2048;   // 8-bit output pieces and the ring of 8-bit skip pieces behind them
 constexpr int MAX_STAGES = 12;
 constexpr int MAX_TMEM_BUFS = 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds at the boost clock
@@ -85,6 +84,7 @@ struct UmmaArgs {
     int part_n;                     // columns one epilogue warp handles per tile
     int piece_bytes;                // row width of one staged output piece (16 ... 128 bytes)
     int epi_warp_bytes;             // staging memory per epilogue warp
+    int skip_ring;                  // staged skip pieces per epilogue warp: 2 or SKIP_RING
     unsigned idesc, idesc_p;        // instruction descriptors of the layer and of the projection (operand signedness)
     unsigned long long desc_hi;     // upper 32 bits of the shared-memory matrix descriptors
     // per-layer epilogue scalars (per-channel layers read the arrays instead)
@@ -887,8 +887,9 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             pf_pc += pcols;
             if (pf_pc >= ncols) { pf_pc = 0; pf_tile += tile_step; }
         };
+        const int skip_ring = u.skip_ring;
         if (SKIP8 && lane == 0)
-            for (int r = 0; r < SKIP_RING; ++r) request_skip_piece(r);
+            for (int r = 0; r < skip_ring; ++r) request_skip_piece(r);
         int ring = 0;
         uint32_t ring_parity = 0;
 
@@ -980,7 +981,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     if (SKIP8) request_skip_piece(ring);
                 }
-                if (SKIP8 && ++ring == SKIP_RING) { ring = 0; ring_parity ^= 1u; }
+                if (SKIP8 && ++ring == skip_ring) { ring = 0; ring_parity ^= 1u; }
             }
             tc_fence_before();
             __syncwarp();
@@ -1011,8 +1012,8 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }
         if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps && lane == 0)
-            for (int j = skip_taken; j < skip_issued; ++j)      // skip pieces requested and not yet waited for (at most SKIP_RING)
-                mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0][j % SKIP_RING]), (uint32_t)((j / SKIP_RING) & 1), &never);
+            for (int j = skip_taken; j < skip_issued; ++j)      // skip pieces requested and not yet waited for (at most the ring)
+                mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0][j % u.skip_ring]), (uint32_t)((j / u.skip_ring) & 1), &never);
         __syncthreads();
     }
     if (warp == MMA_WARP) {
