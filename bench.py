@@ -38,7 +38,8 @@ WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"
              "resnet152": ("ResNet-152 int8 images/sec", "resnet152_b128_224x224x3"),
              "vdsr": ("VDSR int8 images/sec", "vdsr_16x256x256x1"),
              "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1"),
-             "vrcnn_hd": ("VRCNN int8 images/sec", "vrcnn_1x1600x2560x1")}
+             "vrcnn_hd": ("VRCNN int8 images/sec", "vrcnn_1x1600x2560x1"),
+             "vdsr_hd": ("VDSR int8 images/sec", "vdsr_1x1080x1920x1")}
 # DRAM bytes (read + written) per tensor-core launch of one forward, from a one-pass ncu capture
 # of the full workload (command and per-kernel figures: profiles/dram_traffic_resnet50_b256.md),
 # valid only for the kernel source it was taken on: {workload: (bytes per launch, sha256 of

@@ -79,3 +79,69 @@ def test_single_2560x1600_picture_matches_oracle_on_crops():
     g.close()
     del g
     torch.cuda.empty_cache()
+
+
+def test_single_1920x1080_picture_through_the_vdsr_stack_matches_oracle_on_crops():
+    """The VDSR-shaped network on one picture-sized input (Table 4 times VDSR on whole pictures).
+    Receptive-field radius: twenty 3x3 layers = 20 pixels."""
+    net = N.by_name("vdsr_hd")
+    params = load_params("vdsr_hd")
+    g = Network(net, params)
+    x = net_input(net)
+    H, W = x.shape[1], x.shape[2]
+    assert (H, W) == (1080, 1920)
+    out = g.forward(torch.from_numpy(x).cuda())
+    B.iconv_check(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    ch, cw, r = 112, 128, 20
+    crops = [(0, 0, slice(0, ch - r), slice(0, cw - r)),
+             (H - ch, W - cw, slice(r, ch), slice(r, cw)),
+             (517, 0, slice(r, ch - r), slice(0, cw - r)),                         # left edge
+             (301, 1001, slice(r, ch - r), slice(r, cw - r))]
+    small = N.vdsr(n=1, h=ch, w=cw)
+    for top, left, ys, xs in crops:
+        want = ON.forward(small, params, np.ascontiguousarray(x[:, top:top + ch, left:left + cw, :]))
+        for op in (net.ops[0], net.ops[9], net.ops[-1]):
+            got = g.tensors[op.dst][:, top:top + ch, left:left + cw, :].cpu().numpy()
+            a, b = got[:, ys, xs, :], want[op.dst][:, ys, xs, :]
+            assert np.array_equal(a, b), "crop (%d, %d) layer %s: %d mismatches" % (top, left, op.name, (a != b).sum())
+        assert np.unique(want[net.output]).size > 16
+    assert out.shape == (1, H, W, 1)
+    g.close()
+    del g
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name,parts", [("vrcnn_hd", 2), ("vrcnn_hd", 3), ("vdsr_hd", 2), ("vdsr_hd", 3)])
+def test_row_sharded_picture_equals_the_unsplit_one(name, parts):
+    """The strips of a 2- and a 3-way row split, each run through the CUDA library as the rank that
+    owns it would (here one after another on one GPU), stitched: bit-identical to the unsplit GPU
+    forward, which the tests above tie to the oracle."""
+    from paper_2006_11735_b200 import rowshard as RS
+    net = N.by_name(name)
+    params = load_params(name)
+    x = net_input(net)
+    g = Network(net, params)
+    whole = g.forward(torch.from_numpy(x).cuda()).cpu().numpy()
+    B.iconv_check(torch.cuda.current_stream().cuda_stream)
+    g.close()
+    del g
+    torch.cuda.empty_cache()
+    halo = RS.halo_rows(net)
+    assert halo == (6 if name == "vrcnn_hd" else 20)
+
+    def forward(strip):
+        sn = N.by_name(name, h=strip.shape[1], w=strip.shape[2])
+        gs = Network(sn, params)
+        out = gs.forward(torch.from_numpy(strip).cuda()).cpu().numpy()
+        B.iconv_check(torch.cuda.current_stream().cuda_stream)
+        gs.close()
+        return out
+
+    strips = RS.partition(x.shape[1], parts, halo)
+    got = RS.stitch([RS.run_strip(x, s, forward) for s in strips])
+    assert got.shape == whole.shape
+    bad = np.argwhere(got != whole)
+    assert bad.shape[0] == 0, "%d mismatches, first at %s" % (bad.shape[0], bad[:1])
+    assert sum(s.rows for s in strips) == x.shape[1] + 2 * halo * (parts - 1)      # the redundant halo rows
+    torch.cuda.empty_cache()

@@ -239,6 +239,13 @@ def vrcnn_hd(n=1, h=1600, w=2560, seed=3) -> Net:
     return vrcnn(n=n, h=h, w=w, seed=seed)
 
 
+def vdsr_hd(n=1, h=1080, w=1920, seed=2) -> Net:
+    """The VDSR-shaped network on one picture-sized input (the paper times VDSR on whole Set-5
+    pictures, Table 4; 1920 x 1080 stands in for them): the layers, weights and parameters of
+    configuration 2."""
+    return vdsr(n=n, h=h, w=w, seed=seed)
+
+
 def by_name(name: str, **kw) -> Net:
-    return {"single_conv": single_conv, "vdsr": vdsr, "vrcnn": vrcnn, "vrcnn_hd": vrcnn_hd,
+    return {"single_conv": single_conv, "vdsr": vdsr, "vrcnn": vrcnn, "vrcnn_hd": vrcnn_hd, "vdsr_hd": vdsr_hd,
             "resnet18": resnet18, "resnet50": resnet50, "resnet152": resnet152}[name](**kw)
