@@ -9,9 +9,14 @@ average pool and the fully connected layer.  Prints ONE JSON line:
              max over ranks);
   e2e        the same metric through the network's host-buffer entry: every step copies
              the batch from pinned host memory and reads the logits back;
-  roofline   the tensor-core convolution kernel's achieved int8 TOP/s (true MACs of its
+  roofline   the tensor-core convolution kernels' achieved int8 TOP/s (true MACs of their
              launches / their summed CUDA-event duration in the timed region) against
-             2 x the measured dense bf16 peak;
+             2 x the measured dense bf16 peak (burst and sustained, both printed);
+  roofline_hbm  the same launches' algorithmic bytes per second against the measured copy rate;
+  per_layer  every layer: time, TOP/s, GB/s, percent of each peak, the bound that binds it;
+  elementwise  the bandwidth-bound kernels (pools, stand-alone add, thin layers, calibration)
+             timed alone through the C ABI, GB/s against the measured copy rate;
+  vdsr       the second target workload (VDSR-shaped, 16 x 256 x 256) timed the same way;
   cpu_baseline  the CPU oracle timed on a bounded sample of the same workload.
 
 ``--impl reference`` times the CPU oracle instead (the paper ships no code to install).
@@ -40,24 +45,40 @@ WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"
              "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1"),
              "vrcnn_hd": ("VRCNN int8 images/sec", "vrcnn_1x1600x2560x1"),
              "vdsr_hd": ("VDSR int8 images/sec", "vdsr_1x1080x1920x1")}
-# DRAM bytes (read + written) per tensor-core launch of one forward, from a one-pass ncu capture
-# of the full workload (command and per-kernel figures: profiles/dram_traffic_resnet50_b256.md),
-# valid only for the kernel source it was taken on: {workload: (bytes per launch, sha256 of
-# csrc/kernel_umma.cu)}.  A changed kernel reports null until the counters are taken again.
-DRAM_TRAFFIC = {"resnet50": (93223973, "dd97c3edb066cdea6a601480599b4600effab8ca5c46244dff8b114cbb5b85ab")}
+# DRAM bytes (read + written) per launch of the dominant kernel instance, from an ncu capture of a
+# few launches of that instance (two one-pass counters): {workload: (bytes per launch, kernel
+# instance, sha256 of csrc/umma_device.cuh the counters were taken on)}.  A changed kernel
+# reports null until the counters are taken again.
+DRAM_TRAFFIC = {}
 NOMINAL_INT8_TOPS = 4500.0      # NVIDIA's dense INT8 figure for B200 (context only)
 INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
 
 
 def measured_peaks():
-    """(int8 TOP/s peak, HBM GB/s peak, label).  Dense int8 = 2 x the measured bf16 rate; the
-    sustained figure is used because the kernel is timed inside a long step."""
+    """(int8 burst TOP/s, int8 sustained TOP/s, HBM GB/s, label).  Dense int8 = 2 x the measured
+    bf16 rate (nominal ratio 4.5 : 2.25); burst = a kernel timed at full clocks, sustained = inside
+    a long power-capped loop."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             m = json.load(f)
-        return INT8_OVER_BF16 * float(m["bf16_tflops_sustained"]), float(m["hbm_gbs"]), "measured"
-    return INT8_OVER_BF16 * 1400.0, 6650.0, "fallback"
+        return (INT8_OVER_BF16 * float(m["bf16_tflops"]), INT8_OVER_BF16 * float(m["bf16_tflops_sustained"]),
+                float(m["hbm_gbs"]), "measured")
+    return INT8_OVER_BF16 * 1590.0, INT8_OVER_BF16 * 1400.0, 6650.0, "fallback"
+
+
+def tensor_roofline(tops: float, clocks: dict, issue_tops: float) -> dict:
+    """Fractions of every int8 peak in use, and which measured one applies to this run: the burst
+    figure when the SM clock held (within 5 % of its maximum, no power cap), else the sustained one."""
+    burst, sustained, _, kind = measured_peaks()
+    held = bool(clocks.get("sm_mhz")) and bool(clocks.get("sm_max_mhz")) and clocks["sm_mhz"] >= 0.95 * clocks["sm_max_mhz"] \
+        and "sw_power_cap" not in clocks.get("reasons", [])
+    peak = burst if held else sustained
+    return {"bound": "tensor", "achieved": tops, "peak": peak, "unit": "TOP/s", "frac": tops / peak,
+            "peak_kind": "%s 2 x bf16 %s (of %s)" % (kind, "burst: the SM clock held its maximum" if held else "sustained: clocks or power capped", kind),
+            "frac_of_burst": tops / burst, "frac_of_sustained": tops / sustained, "peak_burst": burst, "peak_sustained": sustained,
+            "frac_of_nominal_4500": tops / NOMINAL_INT8_TOPS, "issue_rate_peak": issue_tops,
+            "frac_of_issue_rate_peak": tops / issue_tops if issue_tops else None}
 
 
 class ClockSampler:
@@ -173,6 +194,244 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def time_network(g, x_dev, steps, stream, sampler_index):
+    """K forwards between two events, one event per layer inside.  Returns (ms, marks, clocks)."""
+    import torch
+    sampler = ClockSampler(sampler_index)
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    all_marks = []
+    t0 = time.time()
+    e0.record(stream)
+    for _ in range(steps):
+        marks = []
+        g.forward(x_dev, marks=marks)
+        all_marks.append(marks)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    return e0.elapsed_time(e1), all_marks, sampler.stop(t0, t1)
+
+
+def layer_table(g, net, all_marks, steps, kernels, macs, abytes, int8_peak, hbm_peak):
+    """Per layer: time, TOP/s, GB/s, percent of each peak and the bound that binds it (the larger of
+    the time at the int8 peak and the time at the copy bandwidth)."""
+    layer_ms = {}
+    for marks in all_marks:
+        for (_, prev), (name, ev) in zip(marks[:-1], marks[1:]):
+            layer_ms[name] = layer_ms.get(name, 0.0) + prev.elapsed_time(ev) / steps
+    rows = []
+    for op in net.ops:
+        if op.name not in layer_ms:
+            continue
+        t = layer_ms[op.name]
+        ops = 2.0 * macs.get(op.name, 0)
+        b = abytes.get(op.name, 0)
+        t_tensor, t_hbm = ops / (int8_peak * 1e12) * 1e3, b / (hbm_peak * 1e9) * 1e3
+        rows.append({"layer": op.name, "kernel": kernels.get(op.name, "pool"), "ms": round(t, 5),
+                     "tops": round(ops / (t * 1e-3) / 1e12, 2) if t > 0 else None,
+                     "gbs": round(b / (t * 1e-3) / 1e9, 1) if t > 0 else None,
+                     "pct_int8_peak": round(100.0 * t_tensor / t, 1) if t > 0 else None,
+                     "pct_hbm_peak": round(100.0 * t_hbm / t, 1) if t > 0 else None,
+                     "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                     "roofline_frac": round(max(t_tensor, t_hbm) / t, 3) if t > 0 else None})
+    return rows, layer_ms
+
+
+def family_sums(all_marks, kernels, macs, abytes):
+    fam_ms, fam_macs, fam_bytes = {}, {}, {}
+    for marks in all_marks:
+        for (_, prev), (name, ev) in zip(marks[:-1], marks[1:]):
+            fam = kernels.get(name, "pool")
+            fam_ms[fam] = fam_ms.get(fam, 0.0) + prev.elapsed_time(ev)
+            fam_macs[fam] = fam_macs.get(fam, 0) + macs.get(name, 0)
+            fam_bytes[fam] = fam_bytes.get(fam, 0) + abytes.get(name, 0)
+    return fam_ms, fam_macs, fam_bytes
+
+
+def elementwise_kernels(dev, hbm_peak, peak_kind):
+    """The bandwidth-bound kernels, each timed alone through the C ABI on tensors of the paper's
+    shapes: CUDA events around every call, a 256 MB write between calls so that nothing is served
+    from L2.  Algorithmic bytes = every input and output once."""
+    import numpy as np
+    import torch
+    from paper_2006_11735_b200 import binding as B
+    st = torch.cuda.current_stream(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    rng = np.random.default_rng(7)
+    out = {}
+
+    def timed(name, nbytes, fn, iters=10):
+        for _ in range(3):
+            fn()
+        ms = 0.0
+        for _ in range(iters):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            fn()
+            e1.record(st)
+            torch.cuda.synchronize(dev)
+            ms += e0.elapsed_time(e1)
+        ms /= iters
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[name] = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak, "ms": ms,
+                     "algorithmic_bytes": int(nbytes), "peak_kind": peak_kind + " copy bandwidth", "traffic": None}
+
+    def u8(*shape):
+        return torch.randint(0, 256, shape, dtype=torch.uint8, device=dev)
+
+    # stand-alone add with ratio synchronisation: two 205 MB activations (stage 1 of the ResNet-50 batch)
+    n = 256 * 56 * 56 * 256
+    a, b, o = u8(n), u8(n), torch.empty(n, dtype=torch.uint8, device=dev)
+    timed("add_requant_kernel", 3 * n, lambda: B.iadd_requant(a.data_ptr(), b.data_ptr(), o.data_ptr(), st.cuda_stream, n_elems=n, a_dtype=B.U8,
+                                                              b_dtype=B.U8, out_dtype=B.U8, a_zero=0, b_zero=0, mul_a=3, sh_a=1, mul_b=5, sh_b=2,
+                                                              brelu=1, h_i=400, mul=160, shift=8, out_zero=0, out_lo=0, out_hi=255))
+    del a, b, o
+    # 3x3 / 2 max-pool of the stem output, global average of the last stage
+    x = u8(256, 112, 112, 64)
+    o = torch.empty((256, 56, 56, 64), dtype=torch.uint8, device=dev)
+    timed("maxpool_3x3s2_kernel", x.numel() + o.numel(), lambda: B.ipool_max(x.data_ptr(), o.data_ptr(), 256, 112, 112, 64, 3, 2, 1, st.cuda_stream))
+    x = u8(256, 7, 7, 2048)
+    o = torch.empty((256, 1, 1, 2048), dtype=torch.uint8, device=dev)
+    timed("avgpool16_kernel", x.numel() + o.numel(), lambda: B.ipool_avg_requant(x.data_ptr(), o.data_ptr(), 256, 7, 7, 2048, 1337, 16, 255, st.cuda_stream))
+    # the thin layers of the VDSR shape on the CUDA-core kernels (forced; the plan prefers the tensor cores)
+    W = rng.integers(-127, 128, size=(64, 3, 3, 1), dtype=np.int8)
+    plan = B.iconv_plan(n=16, h=256, w=256, c_in=1, c_out=64, kh=3, kw=3, pad=1, in_dtype=B.U8_RAW128, weights=W,
+                        bias=np.zeros(64, np.int32), mul=[200], shift=[16], h_i=[80000], kernel=B.KERNEL_THIN)
+    x = u8(16, 256, 256, 1)
+    o = torch.empty((16, 256, 256, 64), dtype=torch.uint8, device=dev)
+    timed("thin_in_kernel", x.numel() + o.numel(), lambda: B.iconv_forward(plan, x.data_ptr(), None, o.data_ptr(), None, st.cuda_stream))
+    B.iconv_plan_destroy(plan)
+    W = rng.integers(-127, 128, size=(1, 3, 3, 64), dtype=np.int8)
+    plan = B.iconv_plan(n=16, h=256, w=256, c_in=64, c_out=1, kh=3, kw=3, pad=1, weights=W, bias=np.zeros(1, np.int32), mul=[200], shift=[16],
+                        h_i=[0], brelu=0, out_zero=128, skip_dtype=B.U8_RAW128, skip_c_total=1, skip_mul=3, skip_shift=1, kernel=B.KERNEL_THIN)
+    x = u8(16, 256, 256, 64)
+    sk = u8(16, 256, 256, 1)
+    o = torch.empty((16, 256, 256, 1), dtype=torch.uint8, device=dev)
+    timed("thin_out_kernel", x.numel() + sk.numel() + o.numel(), lambda: B.iconv_forward(plan, x.data_ptr(), sk.data_ptr(), o.data_ptr(), None, st.cuda_stream))
+    B.iconv_plan_destroy(plan)
+    # the n-sigma bound of a 256 MB int32 feature map: four passes over the data
+    y = torch.randint(-200000, 200000, (64 << 20,), dtype=torch.int32, device=dev)
+    timed("select_hist_kernel (iq_sigma_bound, 4 passes)", 4 * y.numel() * 4, lambda: B.iq_sigma_bound(y.data_ptr(), y.numel(), 0.0015, st.cuda_stream), iters=5)
+    del y, flush
+    torch.cuda.empty_cache()
+    return out
+
+
+def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
+    """Times one workload; returns the dict of its figures (the caller prints the line)."""
+    import torch
+    from paper_2006_11735_b200 import binding as B
+    from paper_2006_11735_b200 import dist as D
+    from paper_2006_11735_b200.network import Network, net_input
+    from workloads import networks as N
+    from workloads.params import load_params
+
+    metric, full_name = WORKLOADS[name]
+    full = N.by_name(name)
+    net = N.by_name(name, n=args.batch) if args.batch > 0 else full       # the full batch per GPU (weak scaling)
+    workload = full_name if net.n == full.n else "%s with batch %d (reduced batch: profiling only)" % (full_name, net.n)
+    strips = None
+    if args.row_shard:
+        # one picture over the ranks: every rank convolves the strip it owns (plus the halo)
+        from paper_2006_11735_b200 import rowshard as RS
+        t_in = full.tensors[full.input]
+        strips = RS.partition(t_in.h, size, RS.halo_rows(full))
+        net = N.by_name(name, h=max(1, strips[rank].rows), w=t_in.w)
+        workload = "%s, rows sharded over %d ranks with a halo of %d rows" % (full_name, size, RS.halo_rows(full))
+    params = load_params(name)
+    g = Network(net, params, device=dev)
+    if strips is not None:
+        x_np = net_input(full)[:, strips[rank].in0:strips[rank].in1]
+    else:
+        x_np = net_input(net)
+    x_host = torch.from_numpy(x_np.copy()).pin_memory()
+    x_dev = x_host.to(dev, non_blocking=True)
+    t_out = net.tensors[net.output]
+    out_host = torch.empty((net.n, t_out.h, t_out.w, t_out.c), dtype=torch.int32 if t_out.dtype == "i32" else torch.uint8).pin_memory()
+    stream = torch.cuda.current_stream(dev)
+    kernels, macs, abytes = g.kernels(), g.conv_macs(), g.algorithmic_bytes()
+
+    for _ in range(args.warmup):
+        g.forward(x_dev)
+    B.iconv_check(stream.cuda_stream)
+
+    D.barrier()
+    torch.cuda.synchronize(dev)
+    ms_local, all_marks, clocks = time_network(g, x_dev, args.steps, stream, local_rank)
+    D.barrier()
+    ms = D.max_over_ranks(ms_local, dev)
+    B.iconv_check(stream.cuda_stream)
+    # the repacked first layers are two launches (repack + GEMM), every other step one
+    launches = (len(g.steps) + sum(1 for k in kernels.values() if k == "stem")) * args.steps
+
+    burst, sustained, hbm_peak, peak_kind = measured_peaks()
+    fam_ms, fam_macs, fam_bytes = family_sums(all_marks, kernels, macs, abytes)
+    issue_tops, _ = probe_mma_rate(256, 100000)             # outside every timed region
+    umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
+    umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
+    traffic = None
+    if name in DRAM_TRAFFIC and net.n == full.n:
+        import hashlib
+        with open(os.path.join(ROOT, "paper_2006_11735_b200", "csrc", "umma_device.cuh"), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() == DRAM_TRAFFIC[name][2]:
+                traffic = DRAM_TRAFFIC[name][0]
+    roofline = tensor_roofline(umma_tops, clocks, issue_tops)
+    roofline.update({"kernel": "umma_conv_kernel + umma_window_kernel", "traffic": traffic, "launches": umma_launches,
+                     "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
+                     "time_share": {k: v / sum(fam_ms.values()) for k, v in fam_ms.items()}})
+    umma_gbs = fam_bytes.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e9
+    roofline_hbm = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "hbm", "achieved": umma_gbs, "peak": hbm_peak,
+                    "unit": "GB/s", "frac": umma_gbs / hbm_peak, "traffic": traffic,
+                    "algorithmic_bytes_per_launch": fam_bytes.get("umma", 0) / max(1, umma_launches), "peak_kind": peak_kind + " copy bandwidth",
+                    "algorithmic_bytes_per_step": int(sum(abytes.values())),
+                    "whole_step_gbs": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9,
+                    "whole_step_frac": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9 / hbm_peak}
+    table, layer_ms = layer_table(g, net, all_marks, args.steps, kernels, macs, abytes, roofline["peak"], hbm_peak)
+
+    res = {"metric": metric, "workload": workload, "net": net, "ms": ms, "clocks": clocks, "launches": launches, "roofline": roofline,
+           "roofline_hbm": roofline_hbm, "per_layer": table, "macs": macs, "abytes": abytes, "kernels": kernels, "described": g.describe(),
+           "layer_ms": layer_ms, "images": (1 if strips is not None else net.n * size) * args.steps, "e2e": None,
+           "scaling": "strong" if strips is not None else "weak"}
+
+    if with_e2e:
+        # ---- end to end: pinned host input in, result out, every step ----
+        D.barrier()
+        torch.cuda.synchronize(dev)
+        # Two device input buffers and a copy stream, as a serving loop would run it: the batch of
+        # step i+1 crosses PCIe while step i computes.  Every step's input still comes from pinned
+        # host memory inside the timed region, and every step's result goes back to the host.
+        x_bufs = [x_dev, torch.empty_like(x_dev)]
+        copy_stream = torch.cuda.Stream(dev)
+        copied = [torch.cuda.Event() for _ in range(args.steps)]
+        consumed = [torch.cuda.Event() for _ in range(args.steps)]
+        e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2.record(stream)
+        copy_stream.wait_stream(stream)
+        for i in range(args.steps):
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(consumed[i - 2])       # the buffer's previous batch has been read
+                x_bufs[i % 2].copy_(x_host, non_blocking=True)
+                copied[i].record(copy_stream)
+            stream.wait_event(copied[i])
+            out = g.forward(x_bufs[i % 2])
+            consumed[i].record(stream)
+            out_host.copy_(out, non_blocking=True)
+        e3.record(stream)
+        torch.cuda.synchronize(dev)
+        ms_e2e = D.max_over_ranks(e2.elapsed_time(e3), dev)
+        B.iconv_check(stream.cuda_stream)
+        res["e2e"] = {"value": res["images"] / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel()),
+                      "d2h_bytes_per_step": int(out_host.numel() * out_host.element_size()),
+                      "overlap": "the input copy of step i+1 runs under the compute of step i (two device buffers, one copy stream)"}
+    g.close()
+    del g
+    torch.cuda.empty_cache()
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -180,23 +439,23 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--per-layer", action="store_true", help="print the per-layer table to stderr")
+    ap.add_argument("--no-extras", action="store_true", help="skip the VDSR leg and the element-wise kernels (profiler captures)")
+    ap.add_argument("--per-layer", action="store_true", help="also print the per-layer table to stderr")
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    ap.add_argument("--row-shard", action="store_true",
+                    help="one picture (vrcnn_hd, vdsr_hd) with its rows sharded over the ranks instead of one batch per rank")
     ap.add_argument("--batch", type=int, default=0,
-                    help="images per GPU; 0 = the full workload (256). Smaller batches are for profiler "
-                         "captures only and are named in config.workload")
+                    help="images per GPU; 0 = the full workload. Smaller batches are for profiler captures only and are "
+                         "named in config.workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         return run_reference(args)
 
-    import numpy as np
     import torch
 
-    from paper_2006_11735_b200 import binding as B          # raises if the CUDA library is missing
+    from paper_2006_11735_b200 import binding as B          # noqa: F401  (raises if the CUDA library is missing)
     from paper_2006_11735_b200 import dist as D
-    from paper_2006_11735_b200.network import Network, load_params, net_input
-    from workloads import networks as N
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
@@ -204,121 +463,37 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     D.init("nccl")
+    if args.row_shard and args.workload not in ("vrcnn_hd", "vdsr_hd"):
+        raise SystemExit("--row-shard applies to the single-picture workloads (vrcnn_hd, vdsr_hd)")
 
-    metric, full_name = WORKLOADS[args.workload]
-    full = N.by_name(args.workload)
-    net = N.by_name(args.workload, n=args.batch) if args.batch > 0 else full   # the full batch per GPU (weak scaling)
-    workload = full_name if net.n == full.n else "%s with batch %d (reduced batch: profiling only)" % (full_name, net.n)
-    params = load_params(args.workload)
-    g = Network(net, params, device=dev)
-    x_host = torch.from_numpy(net_input(net)).pin_memory()
-    x_dev = x_host.to(dev, non_blocking=True)
-    t_out = net.tensors[net.output]
-    logits_host = torch.empty((net.n, t_out.h, t_out.w, t_out.c),
-                              dtype=torch.int32 if t_out.dtype == "i32" else torch.uint8).pin_memory()
-    stream = torch.cuda.current_stream(dev)
-    kernels = g.kernels()
-    described = g.describe()
-    macs = g.conv_macs()
-    abytes = g.algorithmic_bytes()
-
-    for _ in range(args.warmup):
-        g.forward(x_dev)
-    B.iconv_check(stream.cuda_stream)
-
-    # ---- device-resident timing: exactly K steps between two events ----
-    D.barrier()
-    torch.cuda.synchronize(dev)
-    sampler = ClockSampler(local_rank)
-    time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    all_marks = []
-    t_wall0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        marks = []
-        g.forward(x_dev, marks=marks)
-        all_marks.append(marks)
-    e1.record(stream)
-    torch.cuda.synchronize(dev)
-    D.barrier()
-    t_wall1 = time.time()
-    clocks = sampler.stop(t_wall0, t_wall1)
-    ms_local = e0.elapsed_time(e1)
-    ms = D.max_over_ranks(ms_local, dev)
-    B.iconv_check(stream.cuda_stream)
-    # the stem is two launches (repack + GEMM), every other step one
-    launches = (len(g.steps) + sum(1 for k in kernels.values() if k == "stem")) * args.steps
-
-    # per-kernel-family time inside the timed region
-    fam_ms, fam_macs, fam_bytes, layer_ms = {}, {}, {}, {}
-    for marks in all_marks:
-        for (_, prev), (name, ev) in zip(marks[:-1], marks[1:]):
-            dt = prev.elapsed_time(ev)
-            fam = kernels.get(name, "pool")
-            fam_ms[fam] = fam_ms.get(fam, 0.0) + dt
-            fam_macs[fam] = fam_macs.get(fam, 0) + macs.get(name, 0)
-            fam_bytes[fam] = fam_bytes.get(fam, 0) + abytes.get(name, 0)
-            layer_ms[name] = layer_ms.get(name, 0.0) + dt / args.steps
-    int8_peak, hbm_peak, peak_kind = measured_peaks()
-    issue_tops, issue_cycles = probe_mma_rate(256, 100000)             # outside every timed region
-    umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
-    umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
-    traffic = None
-    if args.workload in DRAM_TRAFFIC and net.n == full.n:
-        import hashlib
-        src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2006_11735_b200", "csrc", "kernel_umma.cu")
-        with open(src, "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest() == DRAM_TRAFFIC[args.workload][1]:
-                traffic = DRAM_TRAFFIC[args.workload][0]
-    roofline = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "tensor", "achieved": umma_tops, "peak": int8_peak,
-                "unit": "TOP/s", "frac": umma_tops / int8_peak, "traffic": traffic, "peak_kind": peak_kind + " 2 x bf16 sustained",
-                "launches": umma_launches, "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
-                "frac_of_nominal_4500": umma_tops / NOMINAL_INT8_TOPS,
-                "issue_rate_peak": issue_tops, "frac_of_issue_rate_peak": umma_tops / issue_tops,
-                "time_share": {k: v / sum(fam_ms.values()) for k, v in fam_ms.items()}}
-    # the same launches against the memory roofline: most layers of this workload are bound by it
-    umma_gbs = fam_bytes.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e9
-    roofline_hbm = {"kernel": "umma_conv_kernel + umma_window_kernel", "bound": "hbm", "achieved": umma_gbs, "peak": hbm_peak,
-                    "unit": "GB/s", "frac": umma_gbs / hbm_peak, "traffic": traffic,
-                    "algorithmic_bytes_per_launch": fam_bytes.get("umma", 0) / max(1, umma_launches), "peak_kind": peak_kind + " copy bandwidth",
-                    "algorithmic_bytes_per_step": int(sum(abytes.values())),
-                    "whole_step_gbs": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9}
-
-    # ---- end to end: pinned host input in, logits out, every step ----
-    D.barrier()
-    torch.cuda.synchronize(dev)
-    # Two device input buffers and a copy stream, as a serving loop would run it: the batch of
-    # step i+1 crosses PCIe while step i computes.  Every step's input still comes from pinned
-    # host memory inside the timed region, and every step's result goes back to the host.
-    x_bufs = [x_dev, torch.empty_like(x_dev)]
-    copy_stream = torch.cuda.Stream(dev)
-    copied = [torch.cuda.Event() for _ in range(args.steps)]
-    consumed = [torch.cuda.Event() for _ in range(args.steps)]
-    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2.record(stream)
-    copy_stream.wait_stream(stream)
-    for i in range(args.steps):
-        with torch.cuda.stream(copy_stream):
-            if i >= 2:
-                copy_stream.wait_event(consumed[i - 2])       # the buffer's previous batch has been read
-            x_bufs[i % 2].copy_(x_host, non_blocking=True)
-            copied[i].record(copy_stream)
-        stream.wait_event(copied[i])
-        out = g.forward(x_bufs[i % 2])
-        consumed[i].record(stream)
-        logits_host.copy_(out, non_blocking=True)
-    e3.record(stream)
-    torch.cuda.synchronize(dev)
-    ms_e2e = D.max_over_ranks(e2.elapsed_time(e3), dev)
-    B.iconv_check(stream.cuda_stream)
+    r = bench_network(args.workload, args, dev, local_rank, rank, size)
+    ms, net = r["ms"], r["net"]
+    extras = rank == 0 and size == 1 and not args.no_extras and args.batch == 0 and args.workload == "resnet50"
+    vdsr = elementwise = None
+    if extras:
+        v = bench_network("vdsr", args, dev, local_rank, rank, size)
+        vdsr = {"metric": v["metric"], "value": v["images"] / (v["ms"] * 1e-3), "unit": UNIT, "ms_per_step": v["ms"] / args.steps,
+                "workload": v["workload"], "clocks": v["clocks"], "e2e": v["e2e"], "roofline": v["roofline"], "roofline_hbm": v["roofline_hbm"],
+                "int8_tops_whole_step": 2.0 * sum(v["macs"].values()) / (v["ms"] / args.steps * 1e-3) / 1e12, "per_layer": v["per_layer"]}
+        _, _, hbm_peak, peak_kind = measured_peaks()
+        elementwise = elementwise_kernels(dev, hbm_peak, peak_kind)
+        # the repacked stem (repack kernel + GEMM) as one step of the timed forward
+        stem_ms = r["layer_ms"].get("stem")
+        if stem_ms and r["kernels"].get("stem") == "stem":
+            t = net.tensors
+            scratch = net.n * (t["stem"].h + 3) * (t["stem"].w + 3) * 16
+            nbytes = net.n * t["x0"].h * t["x0"].w * 3 + 2 * scratch + net.n * t["stem"].h * t["stem"].w * t["stem"].c
+            elementwise["stem_repack_kernel + umma_window_kernel (7x7/2 stem)"] = {
+                "bound": "hbm", "achieved": nbytes / (stem_ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                "frac": nbytes / (stem_ms * 1e-3) / 1e9 / hbm_peak, "ms": stem_ms, "algorithmic_bytes": int(nbytes),
+                "peak_kind": peak_kind + " copy bandwidth", "traffic": None,
+                "note": "image in, repacked copy written and read once, activations out"}
 
     if args.per_layer and rank == 0:
-        for op in net.ops:
-            m = macs.get(op.name, 0)
-            t = layer_ms.get(op.name, 0.0)
-            sys.stderr.write("%-14s %-6s %8.4f ms %8.1f TOP/s  %s\n" % (op.name, kernels.get(op.name, "pool"), t,
-                                                                          2.0 * m / max(t, 1e-9) / 1e9, described.get(op.name, "")))
+        for row in r["per_layer"]:
+            sys.stderr.write("%-14s %-6s %8.4f ms %8.1f TOP/s %8.1f GB/s  %5.1f %% int8  %5.1f %% hbm  %-6s %s\n" % (
+                row["layer"], row["kernel"], row["ms"], row["tops"] or 0.0, row["gbs"] or 0.0, row["pct_int8_peak"] or 0.0,
+                row["pct_hbm_peak"] or 0.0, row["bound"], r["described"].get(row["layer"], "")))
 
     cpu = None
     if rank == 0 and size == 1 and not args.no_cpu_baseline and args.workload == "resnet50":
@@ -328,22 +503,19 @@ def main():
                "sample": "%d images of the same batch, one forward, %.1f s" % (n_s, dt)}
 
     if rank == 0:
-        total_images = net.n * size * args.steps
-        line = {"metric": metric, "value": total_images / (ms * 1e-3), "unit": UNIT, "n_gpus": size,
+        abytes, macs = r["abytes"], r["macs"]
+        line = {"metric": r["metric"], "value": r["images"] / (ms * 1e-3), "unit": UNIT, "n_gpus": size,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-                "config": {"workload": workload, "global_batch": net.n * size, "parallelism": "dp%d" % size,
+                "scaling": r["scaling"], "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+                "config": {"workload": r["workload"], "global_batch": net.n * size if r["scaling"] == "weak" else net.n,
+                           "parallelism": ("dp%d" if r["scaling"] == "weak" else "rows%d") % size,
                            "l2": "per-step algorithmic traffic (%.1f GB) far exceeds the 126 MB L2" % (sum(abytes.values()) / 1e9),
                            "timing_note": "the timed region carries one CUDA event per layer (the per-kernel durations of "
                                           "`roofline`); the end-to-end loop carries none, which is worth 1-2 %",
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
-                "clocks": clocks,
-                "e2e": {"value": total_images / (ms_e2e * 1e-3), "unit": UNIT,
-                        "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(logits_host.numel() * logits_host.element_size()),
-                        "overlap": "the input copy of step i+1 runs under the compute of step i (two device buffers, one copy stream)"},
-                "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "cpu_baseline": cpu}
+                "clocks": r["clocks"], "e2e": r["e2e"], "gpu_launches": r["launches"], "roofline": r["roofline"],
+                "roofline_hbm": r["roofline_hbm"], "cpu_baseline": cpu, "per_layer": r["per_layer"], "elementwise": elementwise, "vdsr": vdsr}
         print(json.dumps(line))
-    g.close()
     D.finish()
 
 

@@ -175,10 +175,109 @@ __global__ void __launch_bounds__(256) add_requant_kernel(const __grid_constant_
     }
 }
 
+// The usual case in 32-bit arithmetic: 8-bit operands, an 8-bit result, and bounds (checked on the
+// host from the descriptor alone) under which every product and sum below stays inside int32:
+//   a' = (A * mul_a + ca) >> sh_a   with ca = 2^(sh_a-1) - a_zero * mul_a   (the zero point folded in)
+//   b' likewise,  Y = a' + b',  clamp, V = (Y * mul + 2^(shift-1)) >> shift, zero point, saturation.
+// Sixteen elements per thread and step, 16-byte accesses, two steps in flight per thread.
+struct AddFast {
+    int mul_a, ca, sh_a, mul_b, cb, sh_b;
+    int y_lo, y_hi;          // BReLU's clamp, or the (unreachable) bounds of Y when there is none
+    int mul, half, shift, out_zero, out_lo, out_hi;
+    unsigned xor_a, xor_b;   // 0x80808080 turns int8 bytes into offset-binary (the offset rides in ca / cb)
+    int out_signed;
+};
+
+__device__ __forceinline__ void add_fast16(const AddFast &f, uint4 ta, uint4 tb, uint4 &o)
+{
+    const unsigned wa[4] = {ta.x ^ f.xor_a, ta.y ^ f.xor_a, ta.z ^ f.xor_a, ta.w ^ f.xor_a};
+    const unsigned wb[4] = {tb.x ^ f.xor_b, tb.y ^ f.xor_b, tb.z ^ f.xor_b, tb.w ^ f.xor_b};
+    int V[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const int av = (int)__byte_perm(wa[k >> 2], 0, 0x4440 + (k & 3));
+        const int bv = (int)__byte_perm(wb[k >> 2], 0, 0x4440 + (k & 3));
+        int y = ((av * f.mul_a + f.ca) >> f.sh_a) + ((bv * f.mul_b + f.cb) >> f.sh_b);
+        y = min(max(y, f.y_lo), f.y_hi);
+        const int v = ((y * f.mul + f.half) >> f.shift) + f.out_zero;
+        V[k] = min(max(v, f.out_lo), f.out_hi);
+    }
+    unsigned wds[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        wds[k] = (V[4 * k] & 0xff) | ((V[4 * k + 1] & 0xff) << 8) | ((V[4 * k + 2] & 0xff) << 16) | ((unsigned)(V[4 * k + 3] & 0xff) << 24);
+    o = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+}
+
+__global__ void __launch_bounds__(256) add_requant_fast_kernel(const __grid_constant__ AddFast f, const uint4 *__restrict__ A,
+                                                               const uint4 *__restrict__ B, uint4 *__restrict__ out, long long groups)
+{
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; g + nthreads < groups; g += 2 * nthreads) {
+        const uint4 a0 = __ldcs(A + g), b0 = __ldcs(B + g), a1 = __ldcs(A + g + nthreads), b1 = __ldcs(B + g + nthreads);
+        uint4 o0, o1;
+        add_fast16(f, a0, b0, o0);
+        add_fast16(f, a1, b1, o1);
+        __stcs(out + g, o0);
+        __stcs(out + g + nthreads, o1);
+    }
+    if (g < groups) {
+        uint4 o0;
+        add_fast16(f, __ldcs(A + g), __ldcs(B + g), o0);
+        __stcs(out + g, o0);
+    }
+}
+
+// Fills `f` and returns true when the 32-bit form is exact for every possible operand value.
+static bool add_fast_plan(const iadd_desc &d, AddFast &f)
+{
+    const auto eight = [](int t) { return t == ICONV_U8 || t == ICONV_S8; };
+    if (!eight(d.a_dtype) || !eight(d.b_dtype) || !eight(d.out_dtype)) return false;
+    if (d.sh_a > 30 || d.sh_b > 30 || d.shift > 30) return false;
+    const long long LIM = 1ll << 31;
+    // stored byte as an unsigned number sv in [0, 255]; value = sv - z with z = zero (u8) or zero + 128 (offset-binary int8)
+    const long long za = d.a_zero + (d.a_dtype == ICONV_S8 ? 128 : 0), zb = d.b_zero + (d.b_dtype == ICONV_S8 ? 128 : 0);
+    const long long half_a = d.sh_a ? 1ll << (d.sh_a - 1) : 0, half_b = d.sh_b ? 1ll << (d.sh_b - 1) : 0, half = d.shift ? 1ll << (d.shift - 1) : 0;
+    const long long ca = half_a - za * d.mul_a, cb = half_b - zb * d.mul_b;
+    const auto mag = [](long long v) { return v < 0 ? -v : v; };
+    if (mag(ca) + 255ll * d.mul_a >= LIM || mag(cb) + 255ll * d.mul_b >= LIM) return false;
+    const long long a_lo = ca >> d.sh_a, a_hi = (255ll * d.mul_a + ca) >> d.sh_a, b_lo = cb >> d.sh_b, b_hi = (255ll * d.mul_b + cb) >> d.sh_b;
+    long long y_lo = a_lo + b_lo, y_hi = a_hi + b_hi;
+    if (d.brelu) { y_lo = 0; y_hi = d.h_i; }
+    if (mag(y_lo) >= LIM || mag(y_hi) >= LIM) return false;
+    if (mag(y_lo) * d.mul + half >= LIM || mag(y_hi) * d.mul + half >= LIM) return false;
+    if (mag((long long)d.out_zero) >= (1ll << 30)) return false;
+    f.mul_a = d.mul_a; f.ca = (int)ca; f.sh_a = d.sh_a; f.mul_b = d.mul_b; f.cb = (int)cb; f.sh_b = d.sh_b;
+    f.y_lo = (int)y_lo; f.y_hi = (int)y_hi;
+    f.mul = d.mul; f.half = (int)half; f.shift = d.shift; f.out_zero = d.out_zero; f.out_lo = d.out_lo; f.out_hi = d.out_hi;
+    f.xor_a = d.a_dtype == ICONV_S8 ? 0x80808080u : 0u; f.xor_b = d.b_dtype == ICONV_S8 ? 0x80808080u : 0u;
+    f.out_signed = d.out_dtype == ICONV_S8;
+    return true;
+}
+
 int launch_add_requant(const iadd_desc &d, const void *a, const void *b, void *out, cudaStream_t stream)
 {
     if (d.n_elems == 0) return ICONV_OK;
     const int vec_ok = ((uintptr_t)a % 16 == 0) && ((uintptr_t)b % 16 == 0) && ((uintptr_t)out % 16 == 0);
+    AddFast f;
+    if (vec_ok && d.n_elems >= 16 && add_fast_plan(d, f)) {
+        const long long groups = d.n_elems / 16;
+        long long fblocks = (groups + 511) / 512;                 // two groups per thread and round
+        if (fblocks > 148ll * 16) fblocks = 148ll * 16;           // a whole number of waves: 8 resident blocks of 256 threads per SM
+        if (fblocks < 1) fblocks = 1;
+        add_requant_fast_kernel<<<(unsigned)fblocks, 256, 0, stream>>>(f, (const uint4 *)a, (const uint4 *)b, (uint4 *)out, groups);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        const long long done = groups * 16;
+        if (done == d.n_elems) return ICONV_OK;
+        // the ragged tail (fewer than 16 elements) through the general kernel
+        iadd_desc t = d;
+        t.n_elems = d.n_elems - done;
+        const size_t ea = 1, eo = 1;
+        add_requant_kernel<<<1, 32, 0, stream>>>(t, (const uint8_t *)a + done * ea, (const uint8_t *)b + done * ea, (uint8_t *)out + done * eo, 0);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        return ICONV_OK;
+    }
     long long blocks = (d.n_elems / 16 + 255) / 256 + 1;
     if (blocks > 148ll * 32) blocks = 148ll * 32;
     add_requant_kernel<<<(unsigned)blocks, 256, 0, stream>>>(d, a, b, out, vec_ok);

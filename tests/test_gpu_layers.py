@@ -148,6 +148,34 @@ def test_iadd_requant_matches_oracle(n_elems, a_dtype, b_dtype, out_dtype):
     assert np.array_equal(out.get(), want) if n_elems else True
 
 
+@pytest.mark.parametrize("trial", range(12))
+def test_iadd_requant_8bit_forms_with_random_descriptors(trial):
+    """8-bit operands and results take a 32-bit kernel when the descriptor's bounds allow it and the
+    64-bit one otherwise; both must give the oracle's bytes for any multipliers, shifts and zeros."""
+    rng = np.random.default_rng(500 + trial)
+    n_elems = int(rng.integers(1, 70000))
+    a_dtype, b_dtype = [B.U8, B.S8][trial % 2], [B.U8, B.S8][(trial // 2) % 2]
+    out_dtype = [B.U8, B.S8][(trial // 4) % 2]
+    big = trial >= 8                   # multipliers that push the products beyond 32 bits: the general kernel
+    A = rng.integers(0, 256, size=n_elems, dtype=np.uint8).view(np.int8 if a_dtype == B.S8 else np.uint8)
+    Bv = rng.integers(0, 256, size=n_elems, dtype=np.uint8).view(np.int8 if b_dtype == B.S8 else np.uint8)
+    lo, hi = (0, 255) if out_dtype == B.U8 else (-128, 127)
+    kw = dict(a_dtype=a_dtype, b_dtype=b_dtype, out_dtype=out_dtype, a_zero=int(rng.integers(-5, 140)), b_zero=int(rng.integers(-5, 140)),
+              mul_a=int(rng.integers(1, 2 ** 30 if big else 500000)), sh_a=int(rng.integers(20 if big else 0, 31 if big else 12)),
+              mul_b=int(rng.integers(1, 3000)), sh_b=int(rng.integers(0, 12)), brelu=trial % 3 != 0, h_i=int(rng.integers(1, 300000)),
+              mul=int(rng.integers(1, 400)), shift=int(rng.integers(0, 22)), out_zero=int(rng.integers(-20, 140)),
+              out_lo=lo + int(rng.integers(0, 5)), out_hi=hi - int(rng.integers(0, 5)))
+    want, ovf = L.add_requant(A, Bv, **kw)
+    if ovf:
+        pytest.skip("the drawn descriptor overflows int32 in Y")
+    out = Fenced((n_elems,), np.uint8 if out_dtype == B.U8 else np.int8)
+    ad, bd = dev(A), dev(Bv)
+    B.iadd_requant(ad.data_ptr(), bd.data_ptr(), out.ptr, torch.cuda.current_stream().cuda_stream, n_elems=n_elems, **kw)
+    torch.cuda.synchronize()
+    got = out.get()
+    assert np.array_equal(got, want), "%d mismatches" % (got != want).sum()
+
+
 def test_pooling_matches_oracle():
     rng = np.random.default_rng(3)
     for (n, h, w, c, k, s, p) in [(2, 16, 14, 64, 3, 2, 1), (1, 9, 9, 16, 3, 2, 1), (3, 7, 8, 32, 2, 2, 0),
