@@ -69,13 +69,13 @@ def measured_peaks():
 
 def tensor_roofline(tops: float, clocks: dict, issue_tops: float) -> dict:
     """Fractions of every int8 peak in use, and which measured one applies to this run: the burst
-    figure when the SM clock held (within 5 % of its maximum, no power cap), else the sustained one."""
+    figure when the median SM clock under load stayed within 5 % of its maximum (the condition that
+    figure was measured under), else the sustained one (measured at about 1.35 GHz under the power cap)."""
     burst, sustained, _, kind = measured_peaks()
-    held = bool(clocks.get("sm_mhz")) and bool(clocks.get("sm_max_mhz")) and clocks["sm_mhz"] >= 0.95 * clocks["sm_max_mhz"] \
-        and "sw_power_cap" not in clocks.get("reasons", [])
+    held = bool(clocks.get("sm_mhz")) and bool(clocks.get("sm_max_mhz")) and clocks["sm_mhz"] >= 0.95 * clocks["sm_max_mhz"]
     peak = burst if held else sustained
     return {"bound": "tensor", "achieved": tops, "peak": peak, "unit": "TOP/s", "frac": tops / peak,
-            "peak_kind": "%s 2 x bf16 %s (of %s)" % (kind, "burst: the SM clock held its maximum" if held else "sustained: clocks or power capped", kind),
+            "peak_kind": "%s 2 x bf16 %s (of %s)" % (kind, "burst: the median SM clock stayed within 5 % of its maximum" if held else "sustained: the SM clock fell under the power cap", kind),
             "frac_of_burst": tops / burst, "frac_of_sustained": tops / sustained, "peak_burst": burst, "peak_sustained": sustained,
             "frac_of_nominal_4500": tops / NOMINAL_INT8_TOPS, "issue_rate_peak": issue_tops,
             "frac_of_issue_rate_peak": tops / issue_tops if issue_tops else None}
@@ -195,22 +195,30 @@ def run_reference(args):
 
 
 def time_network(g, x_dev, steps, stream, sampler_index):
-    """K forwards between two events, one event per layer inside.  Returns (ms, marks, clocks)."""
+    """Exactly K forwards between two events (nothing else on the stream, so consecutive kernels
+    overlap their set-up with the tail of the one before, as in deployment), then a second pass of
+    up to 20 forwards with one event after every layer for the per-kernel durations (an event
+    between two kernels keeps the second from starting early, so that pass is a little slower and
+    is not the reported step time).  Returns (ms of the K steps, marks, steps of the marks pass, clocks)."""
     import torch
     sampler = ClockSampler(sampler_index)
     time.sleep(0.3)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    all_marks = []
     t0 = time.time()
     e0.record(stream)
     for _ in range(steps):
-        marks = []
-        g.forward(x_dev, marks=marks)
-        all_marks.append(marks)
+        g.forward(x_dev)
     e1.record(stream)
     torch.cuda.synchronize()
     t1 = time.time()
-    return e0.elapsed_time(e1), all_marks, sampler.stop(t0, t1)
+    clocks = sampler.stop(t0, t1)
+    all_marks = []
+    for _ in range(min(steps, 20)):
+        marks = []
+        g.forward(x_dev, marks=marks)
+        all_marks.append(marks)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1), all_marks, len(all_marks), clocks
 
 
 def layer_table(g, net, all_marks, steps, kernels, macs, abytes, int8_peak, hbm_peak):
@@ -359,7 +367,7 @@ def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
 
     D.barrier()
     torch.cuda.synchronize(dev)
-    ms_local, all_marks, clocks = time_network(g, x_dev, args.steps, stream, local_rank)
+    ms_local, all_marks, mark_steps, clocks = time_network(g, x_dev, args.steps, stream, local_rank)
     D.barrier()
     ms = D.max_over_ranks(ms_local, dev)
     B.iconv_check(stream.cuda_stream)
@@ -369,7 +377,7 @@ def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
     burst, sustained, hbm_peak, peak_kind = measured_peaks()
     fam_ms, fam_macs, fam_bytes = family_sums(all_marks, kernels, macs, abytes)
     issue_tops, _ = probe_mma_rate(256, 100000)             # outside every timed region
-    umma_launches = sum(1 for k in kernels.values() if k == "umma") * args.steps
+    umma_launches = sum(1 for k in kernels.values() if k == "umma") * mark_steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
     traffic = None
     if name in DRAM_TRAFFIC and net.n == full.n:
@@ -388,7 +396,7 @@ def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
                     "algorithmic_bytes_per_step": int(sum(abytes.values())),
                     "whole_step_gbs": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9,
                     "whole_step_frac": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9 / hbm_peak}
-    table, layer_ms = layer_table(g, net, all_marks, args.steps, kernels, macs, abytes, roofline["peak"], hbm_peak)
+    table, layer_ms = layer_table(g, net, all_marks, mark_steps, kernels, macs, abytes, roofline["peak"], hbm_peak)
 
     res = {"metric": metric, "workload": workload, "net": net, "ms": ms, "clocks": clocks, "launches": launches, "roofline": roofline,
            "roofline_hbm": roofline_hbm, "per_layer": table, "macs": macs, "abytes": abytes, "kernels": kernels, "described": g.describe(),
@@ -510,8 +518,8 @@ def main():
                 "config": {"workload": r["workload"], "global_batch": net.n * size if r["scaling"] == "weak" else net.n,
                            "parallelism": ("dp%d" if r["scaling"] == "weak" else "rows%d") % size,
                            "l2": "per-step algorithmic traffic (%.1f GB) far exceeds the 126 MB L2" % (sum(abytes.values()) / 1e9),
-                           "timing_note": "the timed region carries one CUDA event per layer (the per-kernel durations of "
-                                          "`roofline`); the end-to-end loop carries none, which is worth 1-2 %",
+                           "timing_note": "value: exactly K forwards between two CUDA events; the per-kernel durations of `roofline`, "
+                                          "`roofline_hbm` and `per_layer` come from a second pass with one event after every layer",
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
                 "clocks": r["clocks"], "e2e": r["e2e"], "gpu_launches": r["launches"], "roofline": r["roofline"],
                 "roofline_hbm": r["roofline_hbm"], "cpu_baseline": cpu, "per_layer": r["per_layer"], "elementwise": elementwise, "vdsr": vdsr}

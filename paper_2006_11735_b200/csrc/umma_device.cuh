@@ -242,6 +242,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// Programmatic dependent launch.  The kernels are launched with programmatic stream serialisation:
+// the next kernel of the stream may be scheduled while this one still runs (its CTAs take the SMs
+// this kernel's CTAs leave, and run their set-up -- barriers, TMEM, the resident filter bank --
+// under the tail of this kernel).  grid_dep_wait blocks until every kernel before this one in the
+// stream has completed and its writes are visible: every role executes it before it first touches
+// a tensor another kernel may have written (activations, skip); plan-owned constants may be read
+// before.  grid_dep_launch tells the scheduler that the kernel after this one may be scheduled.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -630,6 +640,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         mbar_init(smem_u32(&sh->drain), 1);
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        grid_dep_launch();
     }
     if (warp == MMA_WARP) tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
     tc_fence_before();
@@ -660,6 +671,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                     ki * u.kc, nt * u.block_n);
                 b_issued = 1;
             }
+            grid_dep_wait();                        // the activations may come from the kernel before this one
             int stage = 0, slot = 0, turn = warp;   // turn: iterations until this producer's next one
             uint32_t parity = 0;
             bool ok = true;
@@ -848,6 +860,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // outputs in its own two swizzled shared-memory pieces and writes them with its own
         // TMA stores (which also clip the ragged last tile and the channels beyond c_out), so
         // no cross-warp barrier exists that a warp which gave up could strand.
+        grid_dep_wait();                            // the skip operand may come from the kernel before this one
         const int ew = warp - EPI_WARP0;
         const int quad = warp & 3;
         const int slot = ew >> 2;
@@ -1104,6 +1117,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         mbar_init(smem_u32(&sh->drain), 2);          // one arrival per MMA issuer
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        grid_dep_launch();
     }
     if (warp == MMA_WARP) tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
     tc_fence_before();
@@ -1122,6 +1136,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             for (int tap = 0; tap < u.taps; ++tap)
                 tma_load_2d(smem_u32(b_res + (size_t)tap * u.b_tile_bytes), &tmap_w, bf, tap * u.kc, 0);
             b_issued = 1;
+            grid_dep_wait();                        // the activations may come from the kernel before this one
             int stage = 0;
             uint32_t parity = 0;
             const uint32_t tx = (uint32_t)(u.kc * u.win_bw * u.win_bh);
@@ -1227,6 +1242,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         __syncwarp();
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps) {
         // ---------------------------------------------------------------- epilogue
+        grid_dep_wait();                            // the skip operand may come from the kernel before this one
         const int ew = warp - EPI_WARP0;
         const int quad = warp & 3;
         const int slot = ew >> 2;

@@ -17,6 +17,23 @@ struct UmmaLaunch {
     const UmmaArgs *u;
 };
 
+// Launch with programmatic stream serialisation (see grid_dep_wait in umma_device.cuh).
+template <typename... KArgs, typename... Args>
+cudaError_t umma_launch_pdl(void (*kernel)(KArgs...), const UmmaLaunch &l, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(l.grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = l.smem;
+    cfg.stream = l.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // im2col kernel: epi = EPI_* (EPI_NARROW excluded), issue = 0 / 1 / 2
 cudaError_t umma_conv_launch(int epi, int issue, const UmmaLaunch &l);
 cudaError_t umma_conv_opt_in(int epi);

@@ -9,10 +9,9 @@ namespace iconv {
 cudaError_t ICONV_CAT(umma_conv_launch_, ICONV_INST_EPI)(int issue, const UmmaLaunch &l)
 {
     constexpr int E = ICONV_INST_EPI;
-    if (issue == 1) umma_conv_kernel<E, 1><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
-    else if (issue == 2) umma_conv_kernel<E, 2><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
-    else umma_conv_kernel<E, 0><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
-    return cudaGetLastError();
+    if (issue == 1) return umma_launch_pdl(umma_conv_kernel<E, 1>, l, *l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
+    if (issue == 2) return umma_launch_pdl(umma_conv_kernel<E, 2>, l, *l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
+    return umma_launch_pdl(umma_conv_kernel<E, 0>, l, *l.tmap_x, *l.tmap_w, *l.tmap_out, *l.tmap_skip, *l.a, *l.u);
 }
 
 cudaError_t ICONV_CAT(umma_conv_opt_in_, ICONV_INST_EPI)()

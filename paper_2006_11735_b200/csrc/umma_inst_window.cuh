@@ -7,7 +7,7 @@ namespace iconv {
 
 #define ICONV_CAT2(a, b) a##b
 #define ICONV_CAT(a, b) ICONV_CAT2(a, b)
-#define ICONV_WIN_GO(KH, KW, KJ) umma_window_kernel<E, KH, KW, KJ><<<l.grid, NUM_THREADS, l.smem, l.stream>>>(*l.tmap_x, *l.tmap_w, *l.a, *l.u)
+#define ICONV_WIN_GO(KH, KW, KJ) return umma_launch_pdl(umma_window_kernel<E, KH, KW, KJ>, l, *l.tmap_x, *l.tmap_w, *l.a, *l.u)
 #define ICONV_WIN_ATTR(KH, KW, KJ) if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_window_kernel<E, KH, KW, KJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM)
 
 cudaError_t ICONV_CAT(umma_window_launch_, ICONV_INST_EPI)(int kh, int kw, int kj, int pair16, const UmmaLaunch &l)
@@ -20,7 +20,6 @@ cudaError_t ICONV_CAT(umma_window_launch_, ICONV_INST_EPI)(int kh, int kw, int k
     else if (ALL && kh == 4 && kw == 4 && kj == 1 && pair16) ICONV_WIN_GO(ALL ? 4 : 0, ALL ? 2 : 0, ALL ? 1 : 0);
     else if (ALL && kh == 4 && kw == 4 && kj == 1) ICONV_WIN_GO(ALL ? 4 : 0, ALL ? 4 : 0, ALL ? 1 : 0);
     else ICONV_WIN_GO(0, 0, 0);
-    return cudaGetLastError();
 }
 
 cudaError_t ICONV_CAT(umma_window_opt_in_, ICONV_INST_EPI)()
