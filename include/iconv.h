@@ -161,6 +161,30 @@ ICONV_API int iconv_forward(const iconv_plan_t *plan, const void *x, const void 
                   void *workspace, void *cuda_stream);
 
 /*
+ * Two consecutive layers in one kernel (Section 3.1: the output V_i of a layer is the input of the
+ * next; Section 4.1 for the first layer's skip): `first` is a block-closing 1x1 convolution with an
+ * 8-bit skip, `second` the 1x1 convolution that reads exactly first's output slice.  The first
+ * layer's output tile is staged in shared memory on its way to HBM and serves from there as the
+ * second layer's operand, so the wide tensor is written once and the second layer never reads it
+ * back.  Both outputs are bit-identical to iconv_forward of the two layers one after the other.
+ * Taken: both 1x1, stride 1, unpadded, the same pixel grid; 8-bit unsigned activations; first.c_in
+ * 64 or 128, first.c_out a multiple of 128 up to 512, second.c_out 64 or 128; per-layer mul / shift
+ * / h_i whose clamp-free 32-bit epilogue forms the plan can prove (BReLU on, u8 saturation,
+ * skip_shift = 8); both filter banks resident in shared memory.  Anything else returns
+ * ICONV_ERR_UNSUPPORTED with the reason in iconv_last_error(): run the layers apart.
+ * iconv_plan_chain copies what the descriptors point to (host pointers, as iconv_plan) and
+ * allocates the two layers' parameters with cudaMalloc.  iconv_forward_chain: x, skip, out as in
+ * iconv_forward of `first`; out2 DEVICE, the second layer's output tensor (n*h*w*second.out_c_total
+ * bytes, slice [out_c_offset, +c_out) written); all 16-byte aligned; asynchronous on cuda_stream;
+ * no workspace.
+ */
+typedef struct iconv_chain_s iconv_chain_t;
+ICONV_API int iconv_plan_chain(const iconv_desc *first, const iconv_desc *second, iconv_chain_t **chain_out);
+ICONV_API int iconv_chain_destroy(iconv_chain_t *chain);
+ICONV_API int iconv_forward_chain(const iconv_chain_t *chain, const void *x, const void *skip, void *out, void *out2,
+                        void *cuda_stream);
+
+/*
  * Device-side waits (mbarrier phases) are bounded.  A kernel whose wait runs out records
  * a code (1-7) in a per-device status word and returns early.  iconv_check synchronises the
  * stream, reads and clears the word of the current device and returns ICONV_ERR_TIMEOUT if a

@@ -16,7 +16,8 @@ DTYPE_CODE = {"u8": U8, "s8": S8, "i32": I32, "u8_raw128": U8_RAW128}
 KERNEL_NAME = {KERNEL_DIRECT: "direct", KERNEL_UMMA: "umma", KERNEL_THIN: "thin", KERNEL_STEM: "stem"}
 
 EXPORTS = ("iconv_plan", "iconv_plan_destroy", "iconv_plan_kernel", "iconv_plan_describe", "iconv_workspace_bytes", "iconv_forward",
-           "iconv_check", "iconv_selftest_wait_timeout", "iconv_device_initialised",
+           "iconv_check", "iconv_selftest_wait_timeout", "iconv_device_initialised", "iconv_plan_chain", "iconv_chain_destroy",
+           "iconv_forward_chain",
            "iadd_requant", "ipool_max", "ipool_avg_requant", "iq_weight_delta", "iq_quantize_weights",
            "iq_mul_shift", "iq_brelu_params", "iq_skip_sync", "iq_sigma_bound", "iq_bn_fold", "iconcat_plan",
            "iconv_stem_forward_static", "iconv_last_error")
@@ -67,6 +68,9 @@ def _load():
     lib.iconv_plan_describe.argtypes = [vp, C.c_char_p, C.c_size_t]
     lib.iconv_workspace_bytes.argtypes = [vp]
     lib.iconv_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.iconv_plan_chain.argtypes = [P(iconv_desc), P(iconv_desc), P(vp)]
+    lib.iconv_chain_destroy.argtypes = [vp]
+    lib.iconv_forward_chain.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.iconv_selftest_wait_timeout.argtypes = [i32, i64, vp]
     lib.iconv_device_initialised.argtypes = [i32]
     lib.iconv_check.argtypes = [vp]
@@ -106,14 +110,12 @@ def _i32(a):
     return np.ascontiguousarray(np.atleast_1d(np.asarray(a)), dtype=np.int32)
 
 
-def iconv_plan(*, n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, in_dtype=U8, in_c_total=None, in_c_offset=0,
+def _make_desc(*, n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, in_dtype=U8, in_c_total=None, in_c_offset=0,
                out_dtype=U8, out_c_total=None, out_c_offset=0, brelu=1, out_lo=0, out_hi=255, out_zero=0,
                skip_dtype=-1, skip_c_total=0, skip_c_offset=0, skip_mul=1, skip_shift=0, kernel=KERNEL_AUTO,
                weights, bias, mul=None, shift=None, h_i=None, proj=None):
-    """Plan one layer; returns an opaque handle (int).  Arrays are host numpy arrays.
-    proj: optional fused projection skip, a dict with ``weights`` [c_out][k][k][c_in], ``bias``,
-    ``h``, ``w``, ``c_total``, ``c_offset``, ``stride``, ``pad`` of the projection's input; the
-    forward's skip tensor is then that input and ``skip_dtype`` its storage type."""
+    """The C descriptor of one layer and the host arrays it points to (which must outlive the call
+    that reads it)."""
     weights = np.ascontiguousarray(weights, dtype=np.int8)
     assert weights.shape == (c_out, kh, kw, c_in), weights.shape
     bias = _i32(bias)
@@ -142,9 +144,38 @@ def iconv_plan(*, n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, in_dtype=U8, in
         d.proj_stride, d.proj_pad = proj.get("stride", 1), proj.get("pad", 0)
         d.proj_weights, d.proj_bias = pw.ctypes.data, pb.ctypes.data
         keep += [pw, pb]
+    return d, keep
+
+
+def iconv_plan(**kw):
+    """Plan one layer; returns an opaque handle (int).  Arrays are host numpy arrays.
+    proj: optional fused projection skip, a dict with ``weights`` [c_out][k][k][c_in], ``bias``,
+    ``h``, ``w``, ``c_total``, ``c_offset``, ``stride``, ``pad`` of the projection's input; the
+    forward's skip tensor is then that input and ``skip_dtype`` its storage type."""
+    d, keep = _make_desc(**kw)
     plan = C.c_void_p()
     _check(lib.iconv_plan(C.byref(d), C.byref(plan)))
+    del keep
     return plan.value
+
+
+def iconv_plan_chain(first: dict, second: dict):
+    """Plan two consecutive 1x1 layers as one kernel (``iconv_plan``'s keyword arguments for each);
+    raises IconvError(ERR_UNSUPPORTED) when the pair does not qualify."""
+    d1, k1 = _make_desc(**first)
+    d2, k2 = _make_desc(**second)
+    chain = C.c_void_p()
+    _check(lib.iconv_plan_chain(C.byref(d1), C.byref(d2), C.byref(chain)))
+    del k1, k2
+    return chain.value
+
+
+def iconv_chain_destroy(chain):
+    _check(lib.iconv_chain_destroy(chain))
+
+
+def iconv_forward_chain(chain, x_ptr, skip_ptr, out_ptr, out2_ptr, stream=0):
+    _check(lib.iconv_forward_chain(chain, x_ptr, skip_ptr, out_ptr, out2_ptr, stream))
 
 
 def iconv_plan_destroy(plan):

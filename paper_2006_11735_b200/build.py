@@ -13,7 +13,7 @@ OBJ_DIR = os.path.join(_HERE, "_build")
 PROBE_SRC = os.path.join(_HERE, "bench_probe", "probe_mma.cu")
 PROBE_LIB = os.path.join(_HERE, "libiconv_probe.so")
 SOURCES = ["iconv_api.cu", "plan.cu", "kernels_direct.cu", "kernel_thin.cu", "kernel_umma.cu", "kernel_stem.cu",
-           "kernel_calib.cu", "planner.cpp"] + ["umma_inst_conv%d.cu" % e for e in range(8)] + \
+           "kernel_calib.cu", "kernel_chain.cu", "planner.cpp"] + ["umma_inst_conv%d.cu" % e for e in range(8)] + \
           ["umma_inst_window%d.cu" % e for e in (2, 3, 4, 5, 8)]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-diag-suppress", "128", "-Xcompiler", "-fPIC",
          "-Xcompiler", "-fvisibility=hidden", "-I", INCLUDE, "-I", CSRC]

@@ -750,6 +750,22 @@ int encode_launch_maps(const iconv_plan_t *p, const void *x, const void *skip, v
     return ICONV_OK;
 }
 
+int umma_encode_2d(CUtensorMap *map, const void *base, long long inner, long long rows, long long row_stride, int box_inner, int box_rows, int swizzle)
+{
+    const int rc = load_driver_entry_points();
+    if (rc != ICONV_OK) return rc;
+    const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_stride};
+    const cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapSwizzle sw = swizzle == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                  : swizzle == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (2-D map) failed with %d", (int)r); return ICONV_ERR_UNSUPPORTED; }
+    return ICONV_OK;
+}
+
 // ICONV_OK when every descriptor of a launch on these addresses can be encoded (nothing is enqueued).
 int umma_check_maps(const iconv_plan_t *p, const void *x, void *out)
 {

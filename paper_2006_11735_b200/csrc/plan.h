@@ -55,6 +55,10 @@ bool umma_narrow(const iconv_desc &d);      // an 8-bit output too narrow or una
 int umma_setup(iconv_plan_t *p);
 int umma_init_once();                        // driver entry points, shared-memory opt-in of the current device; allocates nothing
 int umma_device_ready(int device);           // the device's SM count once umma_init_once ran on it, else -1
+// 2-D tiled TMA map over uint8 rows: `inner` bytes per row of which a box takes box_inner, `rows` rows `row_stride`
+// bytes apart of which a box takes box_rows; swizzle span in bytes (32, 64, 128; 0 none)
+int umma_encode_2d(CUtensorMap *map, const void *base, long long inner, long long rows, long long row_stride, int box_inner, int box_rows, int swizzle);
+int umma_chain_opt_in();                     // shared-memory opt-in of the two-layer kernel on the current device
 int umma_check_maps(const iconv_plan_t *p, const void *x, void *out);   // can every TMA descriptor of a launch be encoded?
 int umma_geometry(iconv_plan_t *p);           // host-only tile / pipeline / epilogue geometry
 int umma_encode_weight_map(iconv_plan_t *p);  // TMA map over p->w_packed
