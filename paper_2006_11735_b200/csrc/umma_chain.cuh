@@ -155,8 +155,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const uint32_t w2_hi = (uint32_t)(((unsigned long long)(1024 >> 4) << 32 | (1ull << 46) | (2ull << 61)) >> 32);
             // GEMM 2 of tile tt: four K = 32 chunks of the staged tile against the second bank's rows for
             // the tile's 128 input channels, into the accumulator of the tile's pixel tile
-            auto second = [&](int tt) -> bool {
-                const int ss = tt / c.n_tiles, nn = tt - ss * c.n_tiles;
+            int ps = 0, pn = 0;                      // pixel tile and N tile of the tile before the current one
+            auto second = [&](int tt, int ss, int nn) -> bool {
                 if (!mbar_wait(smem_u32(&sh->a2_full[tt & 1]), (uint32_t)((tt >> 1) & 1), &sh->abort_flag)) { chain_give_up(sh, c.status, 3); return false; }
                 if (nn == 0 && !mbar_wait(smem_u32(&sh->d2_empty[ss & 1]), (uint32_t)(((ss >> 1) & 1) ^ 1), &sh->abort_flag)) {
                     chain_give_up(sh, c.status, 2);
@@ -173,13 +173,14 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 if (nn == c.n_tiles - 1) umma_commit(smem_u32(&sh->d2_full[ss & 1]));
                 return true;
             };
+            int s = 0, nt = 0, st = 0;
+            uint32_t a1_parity = 0;
             for (int t = 0; t < T && ok; ++t) {
-                const int s = t / c.n_tiles, nt = t - s * c.n_tiles, st = s % c.stages;
                 if (!mbar_wait(smem_u32(&sh->acc1_empty[t & 1]), (uint32_t)(((t >> 1) & 1) ^ 1), &sh->abort_flag)) {
                     chain_give_up(sh, c.status, 2);
                     break;
                 }
-                if (nt == 0 && !mbar_wait(smem_u32(&sh->a1_full[st]), (uint32_t)((s / c.stages) & 1), &sh->abort_flag)) {
+                if (nt == 0 && !mbar_wait(smem_u32(&sh->a1_full[st]), a1_parity, &sh->abort_flag)) {
                     chain_give_up(sh, c.status, 3);
                     break;
                 }
@@ -189,9 +190,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 for (int j = 0; j < kj1; ++j) umma_i8_split(d1, a_lo + 2u * (uint32_t)j, b_lo + 2u * (uint32_t)j, c.desc_hi1, c.idesc1, (uint32_t)(j != 0));
                 umma_commit(smem_u32(&sh->acc1_full[t & 1]));
                 if (nt == c.n_tiles - 1) umma_commit(smem_u32(&sh->a1_empty[st]));
-                if (t > 0) ok = second(t - 1);
+                if (t > 0) ok = second(t - 1, ps, pn);
+                ps = s; pn = nt;
+                if (++nt == c.n_tiles) { nt = 0; ++s; if (++st == c.stages) { st = 0; a1_parity ^= 1u; } }
             }
-            if (ok && T > 0) second(T - 1);
+            if (ok && T > 0) second(T - 1, ps, pn);
         }
         __syncwarp();
     } else if (warp >= EPI_WARP0) {
@@ -211,15 +214,17 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         bool ok = true;
 
         // skip pieces (32 pixels x 32 bytes) through a ring, requested `ring - 1` tiles ahead
-        int pf = 0;                                 // next tile to request
+        // (no divisions in the per-tile paths: pixel-tile and N-tile counters advance by themselves)
+        int pf = 0, pf_nt = 0, pf_m = (int)blockIdx.x * BLOCK_M + quad * 32;      // next tile to request: index, N tile, first pixel row
+        const int m_step = (int)gridDim.x * BLOCK_M, col0 = part * 32;
         auto request_skip = [&](int ring_slot) {
             if (pf >= T) return;
-            const int s = pf / c.n_tiles, nt = pf - s * c.n_tiles;
             const uint32_t bar = skip_bar0 + 8u * (uint32_t)ring_slot;
             mbar_expect_tx(bar, 1024u);
-            tma_load_2d(sbuf + (uint32_t)(ring_slot * 1024), &tmap_skip, bar, nt * 128 + part * 32, ((int)blockIdx.x + s * (int)gridDim.x) * BLOCK_M + quad * 32);
+            tma_load_2d(sbuf + (uint32_t)(ring_slot * 1024), &tmap_skip, bar, pf_nt * 128 + col0, pf_m);
             ++skip_issued;
             ++pf;
+            if (++pf_nt == c.n_tiles) { pf_nt = 0; pf_m += m_step; }
         };
         if (lane == 0)
             for (int r = 0; r < c.skip_ring; ++r) request_skip(r);
@@ -256,9 +261,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             return true;
         };
 
+        int s = 0, nt = 0, m0 = (int)blockIdx.x * BLOCK_M + quad * 32;
         for (int t = 0; t < T && ok; ++t) {
-            const int s = t / c.n_tiles, nt = t - s * c.n_tiles;
-            const int m0 = ((int)blockIdx.x + s * (int)gridDim.x) * BLOCK_M + quad * 32;
             if (!mbar_wait_warp(smem_u32(&sh->acc1_full[t & 1]), (uint32_t)((t >> 1) & 1), &sh->abort_flag, lane)) {
                 chain_give_up(sh, c.status, 4);
                 break;
@@ -324,6 +328,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             // the second layer's outputs of the pixel tile before this one: its last GEMM 2 was issued
             // behind this tile's GEMM 1
             if (nt == 0 && s > 0) ok = second(s - 1);
+            if (++nt == c.n_tiles) { nt = 0; ++s; m0 += m_step; }
         }
         if (ok && n_super > 0) second(n_super - 1);
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");

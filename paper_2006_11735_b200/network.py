@@ -28,15 +28,21 @@ class Network:
     """Plans every layer once; ``forward`` enqueues the whole network on the current stream."""
 
     def __init__(self, net: Net, params: dict, n=None, device="cuda:0", kernel=B.KERNEL_AUTO, fuse_projection=True,
-                 merge_branches=True):
+                 merge_branches=True, fuse_chain=True):
         """fuse_projection: run a projection skip (a "raw" convolution whose int32 output only feeds
         the next layer's skip) inside that layer's kernel; its int32 tensor is then never written.
         merge_branches: plan two convolutions that read the same tensor and write neighbouring
         channel ranges of the same concatenation (a variable-filter-size block) as one layer: the
         smaller filter sits zero-padded in the middle of the larger one, every channel keeps its
-        own bias, h_i, mul and shift.  The sums only gain zero terms, so the bytes are the same."""
+        own bias, h_i, mul and shift.  The sums only gain zero terms, so the bytes are the same.
+        fuse_chain: run a block-closing 1x1 layer with an 8-bit identity skip and the 1x1 layer that
+        reads its output as ONE kernel where the library takes the pair (``iconv_plan_chain``): the
+        wide tensor is still written (later layers read it as their skip) but not read back by the
+        next layer, and one launch goes."""
         self.net, self.n, self.device = net, net.n if n is None else n, torch.device(device)
         self.plans, self.steps, self.tensors = {}, [], {}
+        self.chains = {}         # name of a closing layer -> chain handle; self.chained: second op name -> closing layer
+        self.chained = {}
         self.fused = {}          # name of a fused projection op -> name of the layer that absorbed it
         self.merged = {}         # name of a branch convolution -> name of the sibling whose plan runs both
         self._pending = {}
@@ -59,7 +65,7 @@ class Network:
                     self.merged[b.name] = a.name
         for op in net.ops:
             src, dst = net.tensors[op.src], net.tensors[op.dst]
-            if op.name in self.merged:
+            if op.name in self.merged or op.name in self.chained:
                 continue
             if op.name in partner:
                 self.plans[op.name] = self._plan_merged(op, partner[op.name], params, kernel)
@@ -103,9 +109,47 @@ class Network:
                     self.tensors.pop(fused["op"].dst, None)        # the projection's int32 output is never written
                     self.steps.append(("conv", op, fused["op"].src))
                     continue
+                nxt = self._chain_partner(op, kernel) if fuse_chain else None
+                if nxt is not None:
+                    try:
+                        self.chains[op.name] = B.iconv_plan_chain(kw, self._conv_kwargs(nxt, params, kernel))
+                        self.chained[nxt.name] = op.name
+                        self.steps.append(("chain", op, nxt))
+                        continue
+                    except B.IconvError as e:
+                        if e.status != B.ERR_UNSUPPORTED:
+                            raise
                 self.plans[op.name] = B.iconv_plan(**kw)
                 self.steps.append(("conv", op, None))
         self._alloc_workspace()
+
+    def _chain_partner(self, op, kernel):
+        """The layer to run in the same kernel as the closing layer `op`, or None: the next
+        operation, a plain 1x1 layer (no skip, 8-bit output) that reads op's whole output."""
+        if kernel not in (B.KERNEL_AUTO, B.KERNEL_UMMA) or op.k != 1 or not op.skip or op.skip_dtype != "u8" or op.role != "act":
+            return None
+        ops = self.net.ops
+        i = ops.index(op)
+        if i + 1 >= len(ops):
+            return None
+        nxt = ops[i + 1]
+        if not isinstance(nxt, Conv) or nxt.src != op.dst or nxt.k != 1 or nxt.stride != 1 or nxt.skip or nxt.role != "act":
+            return None
+        if nxt.c_in != op.c_out or nxt.in_c_offset != op.out_c_offset:
+            return None
+        return nxt
+
+    def _conv_kwargs(self, op, params, kernel) -> dict:
+        """iconv_plan's keyword arguments of a plain layer (8-bit output, no skip)."""
+        net = self.net
+        src, dst = net.tensors[op.src], net.tensors[op.dst]
+        p = params[op.name]
+        w_f = gen.weights_f(net.seed, op.layer, op.c_out, op.k, op.k, op.c_in)
+        return dict(n=self.n, h=src.h, w=src.w, c_in=op.c_in, c_out=op.c_out, kh=op.k, kw=op.k, stride=op.stride, pad=op.pad,
+                    in_dtype=B.DTYPE_CODE[op.in_dtype], in_c_total=src.c, in_c_offset=op.in_c_offset, out_c_total=dst.c,
+                    out_c_offset=op.out_c_offset, weights=B.iq_quantize_weights(w_f, p["delta"]),
+                    bias=gen.bias_i32(net.seed, op.layer, op.c_out), kernel=kernel, out_dtype=B.U8, brelu=p["brelu"],
+                    mul=p["mul"], shift=p["shift"], h_i=p["h_i"], out_lo=p["out_lo"], out_hi=p["out_hi"], out_zero=p["out_zero"])
 
     def _alloc_workspace(self):
         """One buffer of the largest workspace any plan asks for: the layers run one after another
@@ -162,10 +206,14 @@ class Network:
         return True
 
     def kernels(self) -> dict:
-        return {k: B.KERNEL_NAME[B.iconv_plan_kernel(p)] for k, p in self.plans.items()}
+        out = {k: B.KERNEL_NAME[B.iconv_plan_kernel(p)] for k, p in self.plans.items()}
+        out.update({k: "umma" for k in self.chains})
+        return out
 
     def describe(self) -> dict:
-        return {k: B.iconv_plan_describe(p) for k, p in self.plans.items()}
+        out = {k: B.iconv_plan_describe(p) for k, p in self.plans.items()}
+        out.update({k: "umma chain: this layer and %s in one kernel" % [b for b, a in self.chained.items() if a == k][0] for k in self.chains})
+        return out
 
     def conv_macs(self) -> dict:
         """True multiply-accumulates per forward of every convolution (M * N * K)."""
@@ -174,6 +222,7 @@ class Network:
             dst = self.net.tensors[op.dst]
             name = self.fused.get(op.name, op.name)          # a fused projection counts with the layer that runs it
             name = self.merged.get(name, name)               # and so does a merged sibling branch
+            name = self.chained.get(name, name)              # and the second layer of a two-layer kernel
             out[name] = out.get(name, 0) + self.n * dst.h * dst.w * op.c_out * op.c_in * op.k * op.k
         return out
 
@@ -189,7 +238,10 @@ class Network:
                 out[op.name] = self.n * (src.h * src.w * src.c + dst.h * dst.w * dst.c)
                 continue
             b = self.n * src.h * src.w * op.c_in + op.c_out * op.c_in * op.k * op.k + 4 * op.c_out
-            if op.name in self.fused:
+            if op.name in self.chained:                      # its input never comes back from memory
+                name = self.chained[op.name]
+                b += self.n * dst.h * dst.w * op.c_out * esz[dst.dtype] - self.n * src.h * src.w * op.c_in
+            elif op.name in self.fused:
                 name = self.fused[op.name]
             elif op.name in self.merged:                     # shares its sibling's input read
                 name = self.merged[op.name]
@@ -218,7 +270,10 @@ class Network:
             marks.append((None, ev))
         for kind, op, p in self.steps:
             src = self.net.tensors[op.src]
-            if kind == "conv":
+            if kind == "chain":
+                B.iconv_forward_chain(self.chains[op.name], T[op.src].data_ptr(), T[op.skip].data_ptr(), T[op.dst].data_ptr(),
+                                      T[p.dst].data_ptr(), stream)
+            elif kind == "conv":
                 skip_name = p if p is not None else op.skip       # a fused projection reads its own input
                 B.iconv_forward(self.plans[op.name], T[op.src].data_ptr(),
                                 T[skip_name].data_ptr() if skip_name else None, T[op.dst].data_ptr(), self._ws_ptr, stream)
@@ -237,7 +292,9 @@ class Network:
     def close(self):
         for p in self.plans.values():
             B.iconv_plan_destroy(p)
-        self.plans = {}
+        for c in self.chains.values():
+            B.iconv_chain_destroy(c)
+        self.plans, self.chains = {}, {}
 
     def __del__(self):
         try:
