@@ -50,7 +50,7 @@ struct ChainArgs {
 struct ChainShared {
     unsigned long long skip_full[EPI_WARPS_MAX][SKIP_RING];
     unsigned long long a1_full[CHAIN_STAGES_MAX], a1_empty[CHAIN_STAGES_MAX];
-    unsigned long long acc1_full[2], acc1_empty[2];
+    unsigned long long acc1_full[2];
     unsigned long long a2_full[2], a2_empty[2];
     unsigned long long d2_full[2], d2_empty[2];
     unsigned long long w_full, drain;
@@ -93,7 +93,6 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh->acc1_full[b]), 1);
-            mbar_init(smem_u32(&sh->acc1_empty[b]), EPI_WARPS_MAX);
             mbar_init(smem_u32(&sh->a2_full[b]), EPI_WARPS_MAX);
             mbar_init(smem_u32(&sh->a2_empty[b]), 1);
             mbar_init(smem_u32(&sh->d2_full[b]), 1);
@@ -176,10 +175,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             int s = 0, nt = 0, st = 0;
             uint32_t a1_parity = 0;
             for (int t = 0; t < T && ok; ++t) {
-                if (!mbar_wait(smem_u32(&sh->acc1_empty[t & 1]), (uint32_t)(((t >> 1) & 1) ^ 1), &sh->abort_flag)) {
-                    chain_give_up(sh, c.status, 2);
-                    break;
-                }
+                // (accumulator buffer t & 1 is free: the second GEMM of tile t - 2, issued in the round before this
+                // one, waited until every epilogue warp had staged that tile, i.e. had read the buffer)
                 if (nt == 0 && !mbar_wait(smem_u32(&sh->a1_full[st]), a1_parity, &sh->abort_flag)) {
                     chain_give_up(sh, c.status, 3);
                     break;
@@ -262,14 +259,18 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         };
 
         int s = 0, nt = 0, m0 = (int)blockIdx.x * BLOCK_M + quad * 32;
+        const uint32_t acc1_full0 = smem_u32(&sh->acc1_full[0]), a2_full0 = smem_u32(&sh->a2_full[0]), a2_empty0 = smem_u32(&sh->a2_empty[0]);
+        const uint32_t a2_base = smem_u32(a2) + (uint32_t)(part * 4096 + quad * 1024);
+        const uint32_t t_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * 32);
         for (int t = 0; t < T && ok; ++t) {
-            if (!mbar_wait_warp(smem_u32(&sh->acc1_full[t & 1]), (uint32_t)((t >> 1) & 1), &sh->abort_flag, lane)) {
+            const uint32_t par = (uint32_t)(t & 1), par8 = par << 3, phase = (uint32_t)((t >> 1) & 1);
+            if (!mbar_wait_warp(acc1_full0 + par8, phase, &sh->abort_flag, lane)) {
                 chain_give_up(sh, c.status, 4);
                 break;
             }
             tc_fence_after();
             // the staging buffer: GEMM 2 of the tile two back has read it, and so has this warp's own store
-            if (!mbar_wait_warp(smem_u32(&sh->a2_empty[t & 1]), (uint32_t)(((t >> 1) & 1) ^ 1), &sh->abort_flag, lane)) {
+            if (!mbar_wait_warp(a2_empty0 + par8, phase ^ 1u, &sh->abort_flag, lane)) {
                 chain_give_up(sh, c.status, 4);
                 break;
             }
@@ -282,10 +283,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 break;
             }
             if (lane == 0) ++skip_taken;
-            const uint32_t ob = smem_u32(a2) + (uint32_t)((t & 1) * 16384 + part * 4096 + quad * 1024);
+            const uint32_t ob = a2_base + par * 16384u;
             const uint32_t ob_row = ob + row_off, sk_row = sbuf + (uint32_t)(ring * 1024) + row_off;
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((t & 1) * 128 + part * 32);
-            const int n0 = nt * 128 + part * 32;
+            const uint32_t t_row = t_base + par * 128u;
+            const int n0 = nt * 128 + col0;
 #pragma unroll
             for (int g = 0; g < 2; ++g) {
                 const uint32_t goff = (uint32_t)(g << 4) ^ row_swz16;
@@ -316,8 +317,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(smem_u32(&sh->acc1_empty[t & 1]));
-                mbar_arrive(smem_u32(&sh->a2_full[t & 1]));
+                mbar_arrive(a2_full0 + par8);      // also tells the issuer that this warp has read the accumulator buffer
                 asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                              ::"l"(&tmap_out), "r"(ob), "r"(n0), "r"(m0)
                              : "memory");
