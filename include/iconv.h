@@ -76,9 +76,10 @@ typedef enum {
                                   image; stride-1 filters over a single-channel image): a repack of the
                                   image into the caller's workspace (iconv_workspace_bytes), then the
                                   tensor-core kernel on the repacked tensor */
-    ICONV_KERNEL_UMMA_IM2COL = 5  /* the tensor-core kernel with im2col staging even where the plan
-                                  would load one input patch per tile (stride-1 filters); reported
-                                  as ICONV_KERNEL_UMMA by iconv_plan_kernel */
+    ICONV_KERNEL_UMMA_IM2COL = 5  /* the tensor-core kernel in its plainest form: im2col staging even where the
+                                  plan would load one input patch per tile (stride-1 filters), and single
+                                  CTAs even where it would run CTA pairs (long reductions); reported as
+                                  ICONV_KERNEL_UMMA by iconv_plan_kernel */
 } iconv_kernel;
 
 /*

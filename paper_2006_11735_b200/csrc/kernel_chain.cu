@@ -137,6 +137,7 @@ extern "C" int iconv_forward_chain(const iconv_chain_t *c, const void *x, const 
     l.grid = (unsigned)(a.m_tiles < sms ? a.m_tiles : sms);
     l.smem = c->smem;
     l.stream = (cudaStream_t)cuda_stream;
+    l.cluster = 1;
     ICONV_CUDA_TRY(umma_launch_pdl(umma_chain_kernel, l, tmap_x, c->tmap_w1, c->tmap_w2, tmap_out, tmap_skip, a));
     return ICONV_OK;
 }

@@ -496,6 +496,7 @@ int umma_geometry(iconv_plan_t *p)
             p->epi_warps = ew;
             p->skip_ring = ring;
             p->epi_warp_bytes = warp_bytes;
+            p->pipe_room = room;
             for (int kg = k_iters < 8 ? k_iters : 8; kg >= 1; --kg)
                 if (kg * slot <= 48 * 1024 && room / (kg * slot) >= 3) { p->kg = kg; break; }
             p->stages = room / (p->kg * slot);
@@ -618,7 +619,7 @@ int umma_encode_weight_map(iconv_plan_t *p)
     const size_t k_pad = (size_t)plan_taps(p) * p->c_in_pad + (size_t)p->proj_iters * p->kc;
     const cuuint64_t dims[2] = {(cuuint64_t)k_pad, (cuuint64_t)p->c_out_pad};
     const cuuint64_t strides[1] = {(cuuint64_t)k_pad};
-    const cuuint32_t box[2] = {(cuuint32_t)p->kc, (cuuint32_t)p->block_n};
+    const cuuint32_t box[2] = {(cuuint32_t)p->kc, (cuuint32_t)(p->pair ? p->block_n / 2 : p->block_n)};    // pairs: each CTA loads half of a B tile
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = g_encode_tiled(&p->tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, p->w_packed, dims, strides, box, estr,
                                       CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p->kc), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -690,6 +691,25 @@ int umma_setup(iconv_plan_t *p)
     if (p->window) {
         CUtensorMap probe2;     // the tiled patch map must be encodable as well
         if (encode_patch_map(p, p->w_packed, &probe2) != ICONV_OK) p->window = 0;
+    }
+    // Long reductions (one 128-byte k-iteration per stage, the B tile riding in the stage) run on CTA
+    // pairs: per k-iteration a CTA then pulls its 128 pixel rows and HALF of the B tile through its own
+    // L2 port (32 KB instead of 48 for 256 output channels), which is what bounds these layers, and the
+    // stages are deeper.  Not with a forced single-CTA form, a fused projection or per-channel reads.
+    p->pair = 0;
+    if (!p->window && d.kernel != ICONV_KERNEL_UMMA_IM2COL && p->kc == 128 && p->kg == 1 && !p->resident_b && !d.proj_weights &&
+        p->block_n % 32 == 0 && (p->epi == EPI_FAST || p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE) &&
+        (long long)d.n * p->h_out * p->w_out > 2 * BLOCK_M) {
+        const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
+        const int slot = BLOCK_M * p->kc + b_tile / 2;
+        int st = p->pipe_room / slot;
+        if (st > MAX_STAGES) st = MAX_STAGES;
+        if (st >= 3) {
+            p->pair = 1;
+            p->stages = st;
+            rc = umma_encode_weight_map(p);
+            if (rc != ICONV_OK) return rc;
+        }
     }
     if (p->group_uniform && !p->window) {
         // the im2col kernel reads per-channel parameters channel by channel
@@ -812,7 +832,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.slot_a_bytes = BLOCK_M * p->kc;
     u.b_tile_bytes = (p->block_n * p->kc + 1023) / 1024 * 1024;
     u.resident_b = p->resident_b;
-    u.slot_bytes = u.slot_a_bytes + (p->resident_b ? 0 : u.b_tile_bytes);
+    u.slot_bytes = u.slot_a_bytes + (p->resident_b ? 0 : (p->pair ? u.b_tile_bytes / 2 : u.b_tile_bytes));
     u.stage_bytes = u.kg * u.slot_bytes;
     u.producers = p->stages * p->kg < NUM_PRODUCERS ? p->stages * p->kg : NUM_PRODUCERS;
     u.nbuf = p->nbuf;
@@ -830,7 +850,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.skip_ring = p->skip_ring;
     // instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, N/8, M/16
     u.idesc = (2u << 4) | ((d.in_dtype == ICONV_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(p->block_n >> 3) << 17) |
-              ((unsigned)(BLOCK_M >> 4) << 24);
+              ((unsigned)((p->pair ? 2 * BLOCK_M : BLOCK_M) >> 4) << 24);      // pairs: one instruction spans both CTAs' rows (M = 256)
     u.idesc_p = (u.idesc & ~(7u << 7)) | ((d.skip_dtype == ICONV_S8 ? 1u : 0u) << 7);
     // matrix descriptor, upper half: stride between 8-row groups (8 * KC bytes, in 16-byte
     // units), descriptor version 1, swizzle mode (128B = 2, 64B = 4, 32B = 6)
@@ -868,21 +888,23 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
         const unsigned wgrid = (unsigned)(u.m_tiles < sms ? u.m_tiles : sms);
         const size_t wsmem = 1024 + (size_t)u.stages * u.stage_bytes + (size_t)u.b_tile_bytes * u.taps + sizeof(Shared);
         if (wsmem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
-        const UmmaLaunch l = {wgrid, wsmem, stream, &tmap_x, &p->tmap_w, &tmap_out, &tmap_skip, &a, &u};
+        const UmmaLaunch l = {wgrid, wsmem, stream, &tmap_x, &p->tmap_w, &tmap_out, &tmap_skip, &a, &u, 1};
         const int wepi = (p->epi == EPI_FAST || p->epi == EPI_NARROW || p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE_SKIP8) ? p->epi : EPI_SAFE;
         ICONV_CUDA_TRY(umma_window_launch(wepi, d.kh, d.kw, p->kc >> 5, p->pair16, l));
         return ICONV_OK;
     }
+    if (p->pair) u.m_tiles = (u.m_tiles + 1) / 2;                // pixel-tile pairs
     const long long tiles = (long long)u.m_tiles * u.n_tiles;
-    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    if (p->pair) grid = 2u * (unsigned)(tiles < sms / 2 ? tiles : sms / 2);     // clusters of two CTAs
     const size_t smem = 1024 + (size_t)u.stages * u.stage_bytes +
                         (p->resident_b ? (size_t)u.b_tile_bytes * (u.p_iters + u.taps * u.cchunks) * u.n_tiles : 0) + sizeof(Shared) + 1024 +
                         (size_t)p->epi_warps * p->epi_warp_bytes;
     if (smem > (size_t)MAX_SMEM) { set_error("tensor-core path: shared-memory plan exceeds the limit"); return ICONV_ERR_UNSUPPORTED; }
     const int kj_l = p->kc >> 5;
-    const int issue = (kj_l == 4 && p->kg == 1 && !p->resident_b) ? 1
+    const int issue = p->pair ? 3 : (kj_l == 4 && p->kg == 1 && !p->resident_b) ? 1
                       : (kj_l == 4 && p->resident_b && u.p_iters + u.taps * u.cchunks <= p->kg && u.p_iters == 0) ? 2 : 0;
-    const UmmaLaunch l = {grid, smem, stream, &tmap_x, &p->tmap_w, &tmap_out, &tmap_skip, &a, &u};
+    const UmmaLaunch l = {grid, smem, stream, &tmap_x, &p->tmap_w, &tmap_out, &tmap_skip, &a, &u, p->pair ? 2 : 1};
     ICONV_CUDA_TRY(umma_conv_launch(p->epi >= EPI_WIDE && p->epi <= EPI_PROJ ? p->epi : EPI_WIDE, issue, l));
     return ICONV_OK;
 }

@@ -33,6 +33,8 @@ struct iconv_plan_s {
     int q_mul = 1, q_shift = 0, q_h = 0; // per-layer Eq. 4 / BReLU scalars
     int epi_warp_bytes = 8192;           // staging memory per epilogue warp (im2col kernel)
     int skip_ring = 3;                   // staged 8-bit skip pieces per epilogue warp (2 or 3)
+    int pair = 0;                        // long reductions on CTA pairs (tcgen05 cta_group::2): 256-pixel tiles, each CTA holds half of every B tile
+    int pipe_room = 0;                   // shared memory left to the pipeline stages (bytes)
     int group_uniform = 0;               // per-channel parameters equal within every 16-channel group
     int pair16 = 0;                      // internal (stem): 16-channel positions read in pairs, two taps per K step
     // stem path: the plan of the GEMM that follows the repack, and the size of the repacked image,

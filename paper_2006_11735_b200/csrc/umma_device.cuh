@@ -252,6 +252,70 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- CTA pairs (tcgen05 cta_group::2): two CTAs of a cluster work on one 256-row tile.  Each loads
+// its own 128 rows of A and its own half of the B tile; one thread of the even ("leader") CTA issues
+// the MMAs, which read both CTAs' shared memory and write both CTAs' TMEM.  No load is multicast.
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;      // a shared::cluster address with this mask applied names the same offset in the leader CTA
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
+// loads whose completion is counted on the LEADER CTA's barrier (bar already masked)
+__device__ __forceinline__ void tma_load_im2col_4d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h, int n,
+                                                        unsigned short off_w, unsigned short off_h)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar)      // arrive on the barrier at this offset in the leader CTA
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// one arrival on the barrier at this offset in BOTH CTAs once every MMA issued so far is done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -340,6 +404,7 @@ struct IssueRing {
 // `rounds` pipeline stages of one 128-byte k-iteration each into the accumulator at d_tmem:
 // wait for the stage, four MMAs (A at a_lo, B right behind it in the stage), commit the stage.
 // Straight-line apart from the loop itself; returns false when a wait gave up.
+template <bool PAIR_>
 __device__ __forceinline__ bool issue_rounds(IssueRing &g, uint32_t d_tmem, uint32_t idesc, int rounds, int stages, uint32_t a_lo0,
                                              uint32_t stage_step, uint32_t slot_a_step, uint32_t desc_hi32, uint32_t full0,
                                              uint32_t empty0, volatile int *abort_flag)
@@ -347,9 +412,17 @@ __device__ __forceinline__ bool issue_rounds(IssueRing &g, uint32_t d_tmem, uint
     uint32_t acc = 0;
     for (int ki = 0; ki < rounds; ++ki) {
         if (!mbar_test_wait(g.full_bar, g.parity) && !mbar_wait(g.full_bar, g.parity, abort_flag)) return false;
-        umma_slot<4>(d_tmem, g.a_lo, g.a_lo + slot_a_step, desc_hi32, idesc, acc);
+        if (PAIR_) {
+            // one instruction covers both CTAs' 128 rows; the stage is released in both CTAs
+            umma_i8_pair(d_tmem, g.a_lo, g.a_lo + slot_a_step, desc_hi32, idesc, acc);
+#pragma unroll
+            for (int j = 1; j < 4; ++j) umma_i8_pair(d_tmem, g.a_lo + 2u * j, g.a_lo + slot_a_step + 2u * j, desc_hi32, idesc, 1u);
+            umma_commit_pair(g.empty_bar);
+        } else {
+            umma_slot<4>(d_tmem, g.a_lo, g.a_lo + slot_a_step, desc_hi32, idesc, acc);
+            umma_commit(g.empty_bar);
+        }
         acc = 1;
-        umma_commit(g.empty_bar);
         const bool wrap = ++g.stage == stages;
         g.stage = wrap ? 0 : g.stage;
         g.parity ^= wrap ? 1u : 0u;
@@ -614,6 +687,11 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                  const __grid_constant__ ConvArgs a, const __grid_constant__ UmmaArgs u)
 {
     constexpr bool SKIP8 = (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8);
+    // ISSUE 3: the long-reduction path on CTA pairs.  A "tile" is then 256 pixels x block_n: this CTA's
+    // pixel tile is 2 * (tile / n_tiles) + rank, u.m_tiles counts pixel-tile pairs, the grid is walked pair by pair.
+    constexpr bool PAIR = ISSUE == 3;
+    const uint32_t rank = PAIR ? cluster_rank() : 0u;
+    const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, tile_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
     // tiles need the alignment of the widest swizzle pattern (8 rows x 128 bytes)
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -633,7 +711,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         for (int b = 0; b < u.nbuf; ++b) {
             mbar_init(smem_u32(&sh->tmem_full[b]), 1);
-            mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)(4 * u.cs));
+            mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)((PAIR ? 8 : 4) * u.cs));     // pairs: both CTAs' epilogue warps arrive at the leader
         }
         for (int w = 0; w < EPI_WARPS_MAX * SKIP_RING; ++w) mbar_init(smem_u32(&sh->skip_full[0][0]) + 8u * (uint32_t)w, 1);
         mbar_init(smem_u32(&sh->b_full), 1);
@@ -642,9 +720,13 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         grid_dep_launch();
     }
-    if (warp == MMA_WARP) tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
+    if (warp == MMA_WARP) {
+        if (PAIR) tmem_alloc_pair(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
+        else tmem_alloc(smem_u32(&sh->tmem_base), (uint32_t)u.tmem_cols);
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();            // the peer's barriers exist before anything arrives at them
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
 
@@ -661,7 +743,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // wait cannot tell a barrier that is two phases behind from one that is done, and a
         // producer that skips P iterations only knows the consumer's progress up to its own
         // previous iteration.
-        if (lane == 0 && warp < u.producers && (int)blockIdx.x < num_tiles) {
+        if (lane == 0 && warp < u.producers && tile0 < num_tiles) {
             if (u.resident_b && warp == 0) {
                 const uint32_t bf = smem_u32(&sh->b_full);
                 mbar_expect_tx(bf, (uint32_t)(u.block_n * u.kc * k_iters * u.n_tiles));
@@ -676,10 +758,14 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             uint32_t parity = 0;
             bool ok = true;
             const int hw = a.h_out * a.w_out;
-            const uint32_t tx = (uint32_t)(BLOCK_M * u.kc + (u.resident_b ? 0 : u.block_n * u.kc));
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
-                const int n_tile = tile - m_tile * u.n_tiles;
+            // (pairs: every CTA brings its own pixel rows and its own half of the B tile; the bytes of both
+            // CTAs are counted on the leader's barrier, which the leader arms)
+            const uint32_t tx = PAIR ? (uint32_t)(2 * (BLOCK_M * u.kc + (u.block_n >> 1) * u.kc))
+                                     : (uint32_t)(BLOCK_M * u.kc + (u.resident_b ? 0 : u.block_n * u.kc));
+            for (int tile = tile0; tile < num_tiles && ok; tile += tile_stride) {
+                const int m_unit = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
+                const int n_tile = tile - m_unit * u.n_tiles;
+                const int m_tile = PAIR ? 2 * m_unit + (int)rank : m_unit;
                 const unsigned m0 = (unsigned)m_tile * BLOCK_M;
                 const int img = (int)fast_div(m0, u.div_hw_mul, u.div_hw_shr);
                 const unsigned rem = m0 - (unsigned)img * (unsigned)hw;
@@ -730,10 +816,16 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                             }
                             const uint32_t full = smem_u32(&sh->full[stage]);
                             const uint32_t sa = smem_u32(tiles + (size_t)stage * u.stage_bytes + (size_t)slot * u.slot_bytes);
+                            if (PAIR) {
+                                if (rank == 0) mbar_expect_tx(full, tx);
+                                tma_load_im2col_4d_pair(sa, &tmap_x, full & PEER_MASK, cc * u.kc, cw, ch, img, (unsigned short)s, (unsigned short)r);
+                                tma_load_2d_pair(sa + u.slot_a_bytes, &tmap_w, full & PEER_MASK, kx, n_tile * u.block_n + (int)rank * (u.block_n >> 1));
+                            } else {
                             mbar_expect_tx(full, tx);
                             tma_load_im2col_4d(sa, &tmap_x, full, cc * u.kc, cw, ch, img, (unsigned short)s,
                                                (unsigned short)r);
                             if (!u.resident_b) tma_load_2d(sa + u.slot_a_bytes, &tmap_w, full, kx, n_tile * u.block_n);
+                            }
                             // a tile's last stage may be short: stand in for its missing slots
                             if (tile_end)
                                 for (int e = slot + 1; e < u.kg; ++e) mbar_arrive(full);
@@ -754,7 +846,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         __syncwarp();
     } else if (warp == MMA_WARP) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0 && (int)blockIdx.x < num_tiles) {
+        if (lane == 0 && tile0 < num_tiles && (!PAIR || rank == 0)) {
             int t = 0, stage = 0;
             uint32_t parity = 0;
             bool ok = true;
@@ -768,9 +860,9 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const uint32_t stage_step = (uint32_t)u.stage_bytes >> 4, slot_step = (uint32_t)u.slot_bytes >> 4;
             const uint32_t slot_a_step = (uint32_t)u.slot_a_bytes >> 4;
             const uint32_t b_step = (uint32_t)(u.resident_b ? u.b_tile_bytes : u.slot_bytes) >> 4;
-            constexpr bool simple = ISSUE == 1, one_round = ISSUE == 2;
+            constexpr bool simple = ISSUE == 1 || ISSUE == 3, one_round = ISSUE == 2;
             const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+            for (int tile = tile0; tile < num_tiles && ok; tile += tile_stride, ++t) {
                 const int buf = t & (u.nbuf - 1);
                 if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
                     give_up(sh, u.status, 2);
@@ -816,16 +908,16 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ring.a_lo = a_lo0 + (uint32_t)stage * stage_step;
                     ring.full_bar = full0 + 8u * (uint32_t)stage; ring.empty_bar = empty0 + 8u * (uint32_t)stage;
                     if (EPI == EPI_PROJ && u.p_iters) {
-                        ok = issue_rounds(ring, d_tmem + (uint32_t)u.block_n, u.idesc_p, u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
-                                          desc_hi32, full0, empty0, &sh->abort_flag);
-                        if (ok) ok = issue_rounds(ring, d_tmem, u.idesc, k_iters - u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
-                                                  desc_hi32, full0, empty0, &sh->abort_flag);
+                        ok = issue_rounds<PAIR>(ring, d_tmem + (uint32_t)u.block_n, u.idesc_p, u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
+                                                desc_hi32, full0, empty0, &sh->abort_flag);
+                        if (ok) ok = issue_rounds<PAIR>(ring, d_tmem, u.idesc, k_iters - u.p_iters, u.stages, a_lo0, stage_step, slot_a_step,
+                                                        desc_hi32, full0, empty0, &sh->abort_flag);
                     } else {
-                        ok = issue_rounds(ring, d_tmem, u.idesc, k_iters, u.stages, a_lo0, stage_step, slot_a_step, desc_hi32, full0, empty0,
-                                          &sh->abort_flag);
+                        ok = issue_rounds<PAIR>(ring, d_tmem, u.idesc, k_iters, u.stages, a_lo0, stage_step, slot_a_step, desc_hi32, full0, empty0,
+                                                &sh->abort_flag);
                     }
                     stage = ring.stage; parity = ring.parity;
-                    if (ok) umma_commit(smem_u32(&sh->tmem_full[buf]));
+                    if (ok) { if (PAIR) umma_commit_pair(smem_u32(&sh->tmem_full[buf])); else umma_commit(smem_u32(&sh->tmem_full[buf])); }
                     else give_up(sh, u.status, 3);
                     continue;
                 }
@@ -879,7 +971,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int swz_shift = pb == 128 ? 0 : (pb == 64 ? 1 : 2);
         const unsigned row_off = (unsigned)lane * (unsigned)pb;
         const unsigned row_swz16 = pb >= 32 ? ((((unsigned)lane >> swz_shift) & (unsigned)(pb / 16 - 1)) << 4) : 0u;   // XOR mask of the row's 16-byte chunks
-        const int tile_step = u.bi * (int)gridDim.x;
+        const int tile_step = u.bi * tile_stride;
         const EpiScalars es = epi_scalars(a, u);
         int pieces = 0;
         bool ok = true;
@@ -888,14 +980,14 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // SKIP_RING buffers: the load of a piece is issued when the piece SKIP_RING places before it has
         // been consumed, i.e. two pieces of epilogue work ahead of its use, which covers the DRAM latency.
         // (pf_tile, pf_pc): the next piece to request; lane 0 only.
-        int pf_tile = (int)blockIdx.x + turn * (int)gridDim.x, pf_pc = 0;
+        int pf_tile = tile0 + turn * tile_stride, pf_pc = 0;
         auto request_skip_piece = [&](int ring_slot) {
             if (pf_tile >= num_tiles) return;
             const int mt = (int)fast_div((unsigned)pf_tile, u.div_nt_mul, u.div_nt_shr);
             const uint32_t bar = skip_bar0 + 8u * (uint32_t)ring_slot;
             mbar_expect_tx(bar, (uint32_t)piece_smem);
             tma_load_2d(sbuf + (uint32_t)(ring_slot * piece_smem), &tmap_skip, bar, (pf_tile - mt * u.n_tiles) * u.block_n + col_lo + pf_pc,
-                        mt * BLOCK_M + quad * 32);
+                        (PAIR ? 2 * mt + (int)rank : mt) * BLOCK_M + quad * 32);
             ++skip_issued;
             pf_pc += pcols;
             if (pf_pc >= ncols) { pf_pc = 0; pf_tile += tile_step; }
@@ -906,9 +998,10 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         int ring = 0;
         uint32_t ring_parity = 0;
 
-        for (int t = turn, tile = blockIdx.x + turn * gridDim.x; tile < num_tiles && ok; t += u.bi, tile += tile_step) {
-            const int m_tile = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
-            const int n_tile = tile - m_tile * u.n_tiles;
+        for (int t = turn, tile = tile0 + turn * tile_stride; tile < num_tiles && ok; t += u.bi, tile += tile_step) {
+            const int m_unit = (int)fast_div((unsigned)tile, u.div_nt_mul, u.div_nt_shr);
+            const int n_tile = tile - m_unit * u.n_tiles;
+            const int m_tile = PAIR ? 2 * m_unit + (int)rank : m_unit;
             const int buf = t & (u.nbuf - 1);
             const int n0 = n_tile * u.block_n + col_lo;                // first channel of this warp
             if (!mbar_wait_warp(smem_u32(&sh->tmem_full[buf]), (uint32_t)((t >> u.lg_nbuf) & 1), &sh->abort_flag, lane)) {
@@ -998,7 +1091,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
+            if (lane == 0) { if (PAIR) mbar_arrive_leader(smem_u32(&sh->tmem_empty[buf])); else mbar_arrive(smem_u32(&sh->tmem_empty[buf])); }
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         __syncwarp();
@@ -1020,8 +1113,8 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const long long t0 = clock64();
             while (clock64() - t0 < 2000000) {}
         }
-        if (warp == MMA_WARP && lane == 0) {
-            umma_commit(smem_u32(&sh->drain));
+        if (warp == MMA_WARP && lane == 0 && (!PAIR || rank == 0)) {
+            if (PAIR) umma_commit_pair(smem_u32(&sh->drain)); else umma_commit(smem_u32(&sh->drain));
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }
         if (warp >= EPI_WARP0 && warp < EPI_WARP0 + u.epi_warps && lane == 0)
@@ -1029,9 +1122,13 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 mbar_wait(smem_u32(&sh->skip_full[warp - EPI_WARP0][j % u.skip_ring]), (uint32_t)((j / u.skip_ring) & 1), &never);
         __syncthreads();
     }
+    // pairs: neither CTA may leave (or give back its TMEM) while the other can still reach its shared memory
+    // or have MMAs in flight that write its TMEM
+    if (PAIR) cluster_sync_all();
     if (warp == MMA_WARP) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, (uint32_t)u.tmem_cols);
+        if (PAIR) tmem_dealloc_pair(tmem_base, (uint32_t)u.tmem_cols);
+        else tmem_dealloc(tmem_base, (uint32_t)u.tmem_cols);
     }
 }
 

@@ -15,6 +15,7 @@ struct UmmaLaunch {
     const CUtensorMap *tmap_x, *tmap_w, *tmap_out, *tmap_skip;
     const ConvArgs *a;
     const UmmaArgs *u;
+    int cluster;                    // CTAs per cluster: 2 for the CTA-pair form, else 1
 };
 
 // Launch with programmatic stream serialisation (see grid_dep_wait in umma_device.cuh).
@@ -26,15 +27,22 @@ cudaError_t umma_launch_pdl(void (*kernel)(KArgs...), const UmmaLaunch &l, Args.
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = l.smem;
     cfg.stream = l.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (l.cluster > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)l.cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-// im2col kernel: epi = EPI_* (EPI_NARROW excluded), issue = 0 / 1 / 2
+// im2col kernel: epi = EPI_* (EPI_NARROW excluded), issue = 0 / 1 / 2, or 3 (CTA pairs; EPI_FAST, EPI_FAST_SKIP8, EPI_SAFE only)
 cudaError_t umma_conv_launch(int epi, int issue, const UmmaLaunch &l);
 cudaError_t umma_conv_opt_in(int epi);
 // window kernel: kh, kw, kj as planned (the instance with compile-time sizes where one exists)
