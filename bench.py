@@ -45,11 +45,12 @@ WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"
              "vrcnn": ("VRCNN int8 images/sec", "vrcnn_16x512x512x1"),
              "vrcnn_hd": ("VRCNN int8 images/sec", "vrcnn_1x1600x2560x1"),
              "vdsr_hd": ("VDSR int8 images/sec", "vdsr_1x1080x1920x1")}
-# DRAM bytes (read + written) per launch of the dominant kernel instance, from an ncu capture of a
-# few launches of that instance (two one-pass counters): {workload: (bytes per launch, kernel
-# instance, sha256 of csrc/umma_device.cuh the counters were taken on)}.  A changed kernel
+# DRAM bytes (read + written) per launch of the dominant kernel, from an ncu capture of that
+# kernel's launches in one forward (two one-pass counters): {workload: (bytes per launch, kernel,
+# sha256 of the kernel's source the counters were taken on, that source file)}.  A changed kernel
 # reports null until the counters are taken again.
-DRAM_TRAFFIC = {}
+DRAM_TRAFFIC = {"resnet50": (46467249, "umma_conv_kernel (cta pairs)", "619aefc133978185ede5f133027ec6598846ad101637da49033137d8330985fa",
+                             "umma_device.cuh")}
 NOMINAL_INT8_TOPS = 4500.0      # NVIDIA's dense INT8 figure for B200 (context only)
 INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
 
@@ -257,7 +258,7 @@ def family_sums(all_marks, kernels, macs, abytes):
     return fam_ms, fam_macs, fam_bytes
 
 
-def elementwise_kernels(dev, hbm_peak, peak_kind):
+def elementwise_kernels(dev, hbm_peak, peak_kind, iters_default=10):
     """The bandwidth-bound kernels, each timed alone through the C ABI on tensors of the paper's
     shapes: CUDA events around every call, a 256 MB write between calls so that nothing is served
     from L2.  Algorithmic bytes = every input and output once."""
@@ -269,7 +270,8 @@ def elementwise_kernels(dev, hbm_peak, peak_kind):
     rng = np.random.default_rng(7)
     out = {}
 
-    def timed(name, nbytes, fn, iters=10):
+    def timed(name, nbytes, fn, iters=None):
+        iters = iters or iters_default
         for _ in range(3):
             fn()
         ms = 0.0
@@ -321,7 +323,7 @@ def elementwise_kernels(dev, hbm_peak, peak_kind):
     B.iconv_plan_destroy(plan)
     # the n-sigma bound of a 256 MB int32 feature map: four passes over the data
     y = torch.randint(-200000, 200000, (64 << 20,), dtype=torch.int32, device=dev)
-    timed("select_hist_kernel (iq_sigma_bound, 4 passes)", 4 * y.numel() * 4, lambda: B.iq_sigma_bound(y.data_ptr(), y.numel(), 0.0015, st.cuda_stream), iters=5)
+    timed("select_hist_kernel (iq_sigma_bound, 4 passes)", 4 * y.numel() * 4, lambda: B.iq_sigma_bound(y.data_ptr(), y.numel(), 0.0015, st.cuda_stream), iters=max(1, iters_default // 2))
     del y, flush
     torch.cuda.empty_cache()
     return out
@@ -379,12 +381,7 @@ def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
     issue_tops, _ = probe_mma_rate(256, 100000)             # outside every timed region
     umma_launches = sum(1 for k in kernels.values() if k == "umma") * mark_steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
-    traffic = None
-    if name in DRAM_TRAFFIC and net.n == full.n:
-        import hashlib
-        with open(os.path.join(ROOT, "paper_2006_11735_b200", "csrc", "umma_device.cuh"), "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest() == DRAM_TRAFFIC[name][2]:
-                traffic = DRAM_TRAFFIC[name][0]
+    traffic = None     # the aggregate over several kernels has no single capture behind it: see roofline_dominant
     roofline = tensor_roofline(umma_tops, clocks, issue_tops)
     roofline.update({"kernel": "umma_conv_kernel + umma_window_kernel", "traffic": traffic, "launches": umma_launches,
                      "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
@@ -397,8 +394,35 @@ def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
                     "whole_step_gbs": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9,
                     "whole_step_frac": sum(abytes.values()) / (ms / args.steps * 1e-3) / 1e9 / hbm_peak}
     table, layer_ms = layer_table(g, net, all_marks, mark_steps, kernels, macs, abytes, roofline["peak"], hbm_peak)
+    # the kernel with the largest share of the step, by itself against the roofline that binds it
+    groups = {}
+    for row in table:
+        desc = g.describe().get(row["layer"], "")
+        kname = ("umma_chain_kernel" if "chain" in desc else "umma_window_kernel" if "window" in desc else
+                 "umma_conv_kernel (cta pairs)" if "cta pairs" in desc else "umma_conv_kernel" if row["kernel"] == "umma" else row["kernel"])
+        gr = groups.setdefault(kname, {"ms": 0.0, "bytes": 0, "ops": 0.0, "launches": 0})
+        gr["ms"] += row["ms"]; gr["bytes"] += abytes.get(row["layer"], 0); gr["ops"] += 2.0 * macs.get(row["layer"], 0); gr["launches"] += 1
+    dom = max(groups, key=lambda k: groups[k]["ms"])
+    gd = groups[dom]
+    t_tensor, t_hbm = gd["ops"] / (roofline["peak"] * 1e12) * 1e3, gd["bytes"] / (hbm_peak * 1e9) * 1e3
+    dom_traffic = None
+    if name in DRAM_TRAFFIC and net.n == full.n and DRAM_TRAFFIC[name][1] == dom:
+        import hashlib
+        with open(os.path.join(ROOT, "paper_2006_11735_b200", "csrc", DRAM_TRAFFIC[name][3]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() == DRAM_TRAFFIC[name][2]:
+                dom_traffic = DRAM_TRAFFIC[name][0]
+    if t_hbm >= t_tensor:
+        dominant = {"kernel": dom, "bound": "hbm", "achieved": gd["bytes"] / (gd["ms"] * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                    "frac": t_hbm / gd["ms"], "traffic": dom_traffic, "peak_kind": peak_kind + " copy bandwidth"}
+    else:
+        dominant = {"kernel": dom, "bound": "tensor", "achieved": gd["ops"] / (gd["ms"] * 1e-3) / 1e12, "peak": roofline["peak"], "unit": "TOP/s",
+                    "frac": t_tensor / gd["ms"], "traffic": dom_traffic, "peak_kind": roofline["peak_kind"]}
+    dominant.update({"launches_per_step": gd["launches"], "avg_launch_ms": gd["ms"] / gd["launches"],
+                     "algorithmic_bytes_per_launch": gd["bytes"] / gd["launches"], "share_of_step": gd["ms"] / sum(v["ms"] for v in groups.values()),
+                     "shares": {k: round(v["ms"] / sum(x["ms"] for x in groups.values()), 4) for k, v in groups.items()}})
 
     res = {"metric": metric, "workload": workload, "net": net, "ms": ms, "clocks": clocks, "launches": launches, "roofline": roofline,
+           "roofline_dominant": dominant,
            "roofline_hbm": roofline_hbm, "per_layer": table, "macs": macs, "abytes": abytes, "kernels": kernels, "described": g.describe(),
            "layer_ms": layer_ms, "images": (1 if strips is not None else net.n * size) * args.steps, "e2e": None,
            "scaling": "strong" if strips is not None else "weak"}
@@ -448,6 +472,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the VDSR leg and the element-wise kernels (profiler captures)")
+    ap.add_argument("--elementwise-iters", type=int, default=10, help="timed calls per element-wise kernel (1 for profiler captures)")
     ap.add_argument("--per-layer", action="store_true", help="also print the per-layer table to stderr")
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--row-shard", action="store_true",
@@ -482,9 +507,10 @@ def main():
         v = bench_network("vdsr", args, dev, local_rank, rank, size)
         vdsr = {"metric": v["metric"], "value": v["images"] / (v["ms"] * 1e-3), "unit": UNIT, "ms_per_step": v["ms"] / args.steps,
                 "workload": v["workload"], "clocks": v["clocks"], "e2e": v["e2e"], "roofline": v["roofline"], "roofline_hbm": v["roofline_hbm"],
+                "roofline_dominant": v["roofline_dominant"],
                 "int8_tops_whole_step": 2.0 * sum(v["macs"].values()) / (v["ms"] / args.steps * 1e-3) / 1e12, "per_layer": v["per_layer"]}
         _, _, hbm_peak, peak_kind = measured_peaks()
-        elementwise = elementwise_kernels(dev, hbm_peak, peak_kind)
+        elementwise = elementwise_kernels(dev, hbm_peak, peak_kind, args.elementwise_iters)
         # the repacked stem (repack kernel + GEMM) as one step of the timed forward
         stem_ms = r["layer_ms"].get("stem")
         if stem_ms and r["kernels"].get("stem") == "stem":
@@ -522,7 +548,7 @@ def main():
                                           "`roofline_hbm` and `per_layer` come from a second pass with one event after every layer",
                            "int8_tops_whole_step": 2.0 * sum(macs.values()) / (ms / args.steps * 1e-3) / 1e12},
                 "clocks": r["clocks"], "e2e": r["e2e"], "gpu_launches": r["launches"], "roofline": r["roofline"],
-                "roofline_hbm": r["roofline_hbm"], "cpu_baseline": cpu, "per_layer": r["per_layer"], "elementwise": elementwise, "vdsr": vdsr}
+                "roofline_hbm": r["roofline_hbm"], "roofline_dominant": r["roofline_dominant"], "cpu_baseline": cpu, "per_layer": r["per_layer"], "elementwise": elementwise, "vdsr": vdsr}
         print(json.dumps(line))
     D.finish()
 
