@@ -698,7 +698,7 @@ int umma_setup(iconv_plan_t *p)
     // stages are deeper.  Not with a forced single-CTA form, a fused projection or per-channel reads.
     p->pair = 0;
     if (!p->window && d.kernel != ICONV_KERNEL_UMMA_IM2COL && p->kc == 128 && p->kg == 1 && !p->resident_b && !d.proj_weights &&
-        p->block_n % 32 == 0 && (p->epi == EPI_FAST || p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE) &&
+        p->block_n % 32 == 0 && (p->epi == EPI_FAST || p->epi == EPI_FAST_SKIP8 || p->epi == EPI_SAFE || p->epi == EPI_SAFE_SKIP8) &&
         (long long)d.n * p->h_out * p->w_out > 2 * BLOCK_M) {
         const int b_tile = (p->block_n * p->kc + 1023) / 1024 * 1024;
         const int slot = BLOCK_M * p->kc + b_tile / 2;

@@ -42,7 +42,7 @@ cudaError_t umma_launch_pdl(void (*kernel)(KArgs...), const UmmaLaunch &l, Args.
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-// im2col kernel: epi = EPI_* (EPI_NARROW excluded), issue = 0 / 1 / 2, or 3 (CTA pairs; EPI_FAST, EPI_FAST_SKIP8, EPI_SAFE only)
+// im2col kernel: epi = EPI_* (EPI_NARROW excluded), issue = 0 / 1 / 2, or 3 (CTA pairs; the 8-bit-output forms without a fused projection: EPI_FAST, EPI_FAST_SKIP8, EPI_SAFE, EPI_SAFE_SKIP8)
 cudaError_t umma_conv_launch(int epi, int issue, const UmmaLaunch &l);
 cudaError_t umma_conv_opt_in(int epi);
 // window kernel: kh, kw, kj as planned (the instance with compile-time sizes where one exists)

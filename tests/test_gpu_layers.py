@@ -217,6 +217,44 @@ UMMA_SHAPES = [
 ]
 
 
+PAIR_SHAPES = [
+    # long reductions the plan runs on CTA pairs (256-pixel tiles, each CTA loads half of every B tile);
+    # n, h, w, c_in, c_out, k, stride, pad
+    (2, 14, 14, 256, 256, 3, 1, 1),     # stage-3 3x3: 18 k-iterations, 4 pixel tiles = 2 pairs
+    (6, 14, 14, 256, 256, 3, 2, 1),     # stride 2: 294 pixels = 3 pixel tiles, the last pair's second CTA has none
+    (3, 14, 14, 1024, 256, 1, 1, 0),    # 5 pixel tiles: the last pair's second CTA has no real pixel at all
+    (2, 15, 15, 512, 512, 1, 1, 0),     # two N tiles of 256, 450 pixels
+    (40, 14, 14, 1024, 128, 1, 1, 0),   # N = 128 (64 rows of B per CTA), 62 pixel tiles
+    (8, 7, 7, 512, 512, 3, 1, 1),       # stage-4 3x3 on 7 x 7 maps, 392 pixels
+    (150, 14, 14, 256, 256, 3, 1, 1),   # 230 pixel tiles: more pairs than SM pairs, ragged schedule
+]
+
+
+@pytest.mark.parametrize("shape", PAIR_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("skip", [None, B.U8], ids=["plain", "skip8"])
+def test_cta_pair_form_matches_oracle(shape, skip):
+    n, h, w, c_in, c_out, k, stride, pad = shape
+    if n > 100 and skip is not None:
+        pytest.skip("the large case runs once")
+    X, W, b, mul, shift, h_i = _layer(sum(shape) + 7, n, h, w, c_in, c_out, k)
+    kw = dict(stride=stride, pad=pad)
+    if skip is not None:
+        ho, wo = (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
+        S = np.random.default_rng(3).integers(0, 256, size=(n, ho, wo, c_out), dtype=np.uint8)
+        kw.update(skip=S, skip_dtype=skip, skip_mul=int(h_i[0]) // 2, skip_shift=8)
+    want = oracle_conv(X, W, b, mul, shift, h_i, **kw)
+    text = []
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, kernel=B.KERNEL_UMMA, describe=text, **kw)
+    assert fam == B.KERNEL_UMMA and "cta pairs" in text[0], text[0]
+    bad = np.argwhere(got != want)
+    assert bad.shape[0] == 0, "%d mismatches, first at %s" % (bad.shape[0], bad[:1])
+    assert 0.02 < (want == 0).mean() < 0.98
+    # the single-CTA form of the same layer
+    text = []
+    got1, _ = gpu_conv(X, W, b, mul, shift, h_i, kernel=B.KERNEL_UMMA_IM2COL, describe=text, **kw)
+    assert "cta pairs" not in text[0] and np.array_equal(got1, want)
+
+
 WINDOW_SHAPES = [
     # stride-1 filters the plan runs in window mode (one patch load per tile); n, h, w, c_in, c_out, k, stride, pad
     (2, 5, 256, 64, 64, 3, 1, 1),       # VDSR rows: two 128-pixel strips per row
