@@ -81,7 +81,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     uint8_t *skp = a2 + 2 * 16384;                          // [16 warps][ring][32 pixels][32 bytes]
     ChainShared *sh = (ChainShared *)(skp + (size_t)EPI_WARPS_MAX * c.skip_ring * 1024);
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);    // the same value in every lane, and known to the compiler as such: per-warp addresses and coordinates live in uniform registers
     const int lane = threadIdx.x & 31;
     const int n_super = (int)blockIdx.x < c.m_tiles ? (c.m_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     const int T = n_super * c.n_tiles;                      // tiles of this CTA
@@ -275,7 +275,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 break;
             }
             if (t >= 2) {
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                if (elect_one()) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 __syncwarp();
             }
             if (!mbar_wait_warp(skip_bar0 + 8u * (uint32_t)ring, ring_parity, &sh->abort_flag, lane)) {
@@ -316,7 +316,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) {
+            if (elect_one()) {
                 mbar_arrive(a2_full0 + par8);      // also tells the issuer that this warp has read the accumulator buffer
                 asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                              ::"l"(&tmap_out), "r"(ob), "r"(n0), "r"(m0)

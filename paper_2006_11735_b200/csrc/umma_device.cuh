@@ -252,6 +252,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// One lane of the (fully active) warp, the lowest: the form the compiler recognises as "a single thread", so that what
+// the lane does (TMA issue, barrier arrivals) is issued from uniform registers.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t p;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(p));
+    return p != 0;
+}
+
 // ---- CTA pairs (tcgen05 cta_group::2): two CTAs of a cluster work on one 256-row tile.  Each loads
 // its own 128 rows of A and its own half of the B tile; one thread of the even ("leader") CTA issues
 // the MMAs, which read both CTAs' shared memory and write both CTAs' TMEM.  No load is multicast.
@@ -700,7 +709,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     Shared *sh = (Shared *)(b_res + (u.resident_b ? (size_t)u.b_tile_bytes * k_iters * u.n_tiles : 0));
     uint8_t *epi_smem = (uint8_t *)(((uintptr_t)(sh + 1) + 1023) & ~(uintptr_t)1023);
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);    // the same value in every lane, and known to the compiler as such: per-warp addresses and coordinates live in uniform registers
     const int lane = threadIdx.x & 31;
     const int num_tiles = u.m_tiles * u.n_tiles;
 
@@ -1023,7 +1032,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const uint32_t t_piece = t_row + (uint32_t)pc;
                 // the store issued two pieces ago must have finished reading this buffer
                 if (pieces >= 2) {
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    if (elect_one()) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                 }
                 if (SKIP8) {
@@ -1080,7 +1089,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 // one SKIP_RING places on
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) {
+                if (elect_one()) {
                     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                                  ::"l"(&tmap_out), "r"(ob), "r"(n0 + pc), "r"(m_tile * BLOCK_M + quad * 32)
                                  : "memory");
@@ -1197,7 +1206,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *b_res = tiles + (size_t)u.stages * u.stage_bytes;
     Shared *sh = (Shared *)(b_res + (size_t)u.b_tile_bytes * u.taps);
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);    // the same value in every lane, and known to the compiler as such: per-warp addresses and coordinates live in uniform registers
     const int lane = threadIdx.x & 31;
     const int num_tiles = u.m_tiles;
 
