@@ -144,6 +144,21 @@ def probe_mma_rate(block_n: int = 256, iters: int = 100000):
     return tops.value, cyc.value
 
 
+def probe_mma_rate_rows(block_n: int, row_bytes: int, a_group_stride: int, iters: int = 50000):
+    """The same probe with operand rows of row_bytes (32 / 64 / 128, the swizzle width) and A's 8-row groups
+    a_group_stride bytes apart: the operand forms of narrow layers and of the window kernel's block tiling."""
+    import ctypes as C
+    from paper_2006_11735_b200 import build as lib_build
+    lib = C.CDLL(lib_build.PROBE_LIB)
+    lib.probe_mma_rate_rows.argtypes = [C.c_int32] * 4 + [C.POINTER(C.c_double)] * 2
+    lib.probe_mma_rate_rows.restype = C.c_int
+    tops, cyc = C.c_double(), C.c_double()
+    rc = lib.probe_mma_rate_rows(block_n, row_bytes, a_group_stride, iters, C.byref(tops), C.byref(cyc))
+    if rc != 0:
+        raise RuntimeError("probe_mma_rate_rows failed with status %d" % rc)
+    return tops.value, cyc.value
+
+
 def oracle_images_per_s(n_images: int, repeats: int = 1, first: int = 0):
     """Times the CPU oracle, as it stands, on n_images of the workload (forward only)."""
     from oracle import networks as ON
@@ -379,10 +394,14 @@ def bench_network(name, args, dev, local_rank, rank, size, with_e2e=True):
     burst, sustained, hbm_peak, peak_kind = measured_peaks()
     fam_ms, fam_macs, fam_bytes = family_sums(all_marks, kernels, macs, abytes)
     issue_tops, _ = probe_mma_rate(256, 100000)             # outside every timed region
+    issue64_tops, issue64_cycles = probe_mma_rate_rows(64, 64, 512, 50000)
     umma_launches = sum(1 for k in kernels.values() if k == "umma") * mark_steps
     umma_tops = 2.0 * fam_macs.get("umma", 0) / (fam_ms.get("umma", 1e-9) * 1e-3) / 1e12
     traffic = None     # the aggregate over several kernels has no single capture behind it: see roofline_dominant
     roofline = tensor_roofline(umma_tops, clocks, issue_tops)
+    # what a stream of N = 64 instructions reaches (layers with at most 64 output channels): an instruction with
+    # N <= 64 occupies the pipe about as long as one with N = 128
+    roofline.update({"issue_rate_peak_n64": issue64_tops, "cycles_per_instruction_n64": issue64_cycles})
     roofline.update({"kernel": "umma_conv_kernel + umma_window_kernel", "traffic": traffic, "launches": umma_launches,
                      "avg_launch_ms": fam_ms.get("umma", 0.0) / max(1, umma_launches),
                      "time_share": {k: v / sum(fam_ms.values()) for k, v in fam_ms.items()}})

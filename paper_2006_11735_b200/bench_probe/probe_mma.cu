@@ -22,7 +22,7 @@ struct ProbeResult {
     int pad;
 };
 
-__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int iters, ProbeResult *res)
+__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int row_bytes, int a_group_stride, int iters, ProbeResult *res)
 {
     extern __shared__ uint8_t probe_raw[];
     uint8_t *tiles = (uint8_t *)(((uintptr_t)probe_raw + 1023) & ~(uintptr_t)1023);   // A: 16 KB, B: 32 KB
@@ -43,14 +43,19 @@ __global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int iters, Prob
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tb = tmem_base;
     if (threadIdx.x == 0) {
-        // K-major tiles with 128-byte rows and the 128-byte swizzle, as the convolution kernel stages them
-        const unsigned long long hi = ((unsigned long long)((8 * 128) >> 4) << 32) | (1ull << 46) | (2ull << 61);
-        const unsigned long long da = hi | (unsigned long long)((probe_smem_u32(tiles) & 0x3FFFFu) >> 4) | (1ull << 16);
-        const unsigned long long db = hi | (unsigned long long)((probe_smem_u32(tiles + 16384) & 0x3FFFFu) >> 4) | (1ull << 16);
+        // K-major tiles with rows of row_bytes (128, 64 or 32) and the swizzle of that width, as the
+        // convolution kernels stage them; A's 8-row groups a_group_stride bytes apart (8 * row_bytes for
+        // a dense tile, a patch line in the window kernel's block tiling)
+        const unsigned long long layout = row_bytes == 128 ? 2ull : (row_bytes == 64 ? 4ull : 6ull);
+        const unsigned long long hi_a = ((unsigned long long)(a_group_stride >> 4) << 32) | (1ull << 46) | (layout << 61);
+        const unsigned long long hi_b = ((unsigned long long)((8 * row_bytes) >> 4) << 32) | (1ull << 46) | (layout << 61);
+        const unsigned long long da = hi_a | (unsigned long long)((probe_smem_u32(tiles) & 0x3FFFFu) >> 4) | (1ull << 16);
+        const unsigned long long db = hi_b | (unsigned long long)((probe_smem_u32(tiles + 16384) & 0x3FFFFu) >> 4) | (1ull << 16);
         const uint32_t idesc = (2u << 4) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((128u >> 4) << 24);   // u8 x s8 -> s32
+        const unsigned slices = (unsigned)(row_bytes >> 5);
         const long long t0 = clock64();
         for (int i = 0; i < iters; ++i) {
-            const unsigned long long k = 2ull * (unsigned)(i & 3);    // walk the four 32-byte K slices of a row
+            const unsigned long long k = 2ull * ((unsigned)i & (slices - 1));    // walk the 32-byte K slices of a row
             asm volatile(
                 "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
@@ -87,7 +92,27 @@ using namespace iconv_probe;
 // time of the launch) and the slowest SM's cycles per instruction to the HOST pointers.
 // Synchronous; allocates a few KB on the current device.  Returns 0, -1 (bad argument),
 // -6 (a CUDA call failed) or -7 (the bounded wait for the last instruction ran out).
+//
+// probe_mma_rate_rows: the same with operand rows of row_bytes (32, 64 or 128: the swizzle width) and
+// A's 8-row groups a_group_stride bytes apart (a multiple of 16, at least 8 * row_bytes, the 16 groups
+// within 16 KB), the forms the convolution kernels use for narrow layers and for block tiling.
+static int probe_run(int32_t block_n, int32_t row_bytes, int32_t a_group_stride, int32_t iters, double *tops, double *cycles_per_mma);
+
 extern "C" __attribute__((visibility("default"))) int probe_mma_rate(int32_t block_n, int32_t iters, double *tops, double *cycles_per_mma)
+{
+    return probe_run(block_n, 128, 1024, iters, tops, cycles_per_mma);
+}
+
+extern "C" __attribute__((visibility("default"))) int probe_mma_rate_rows(int32_t block_n, int32_t row_bytes, int32_t a_group_stride, int32_t iters,
+                                                                          double *tops, double *cycles_per_mma)
+{
+    if ((row_bytes != 32 && row_bytes != 64 && row_bytes != 128) || a_group_stride % 16 || a_group_stride < 8 * row_bytes ||
+        15 * a_group_stride + 8 * row_bytes > 16384)
+        return -1;
+    return probe_run(block_n, row_bytes, a_group_stride, iters, tops, cycles_per_mma);
+}
+
+static int probe_run(int32_t block_n, int32_t row_bytes, int32_t a_group_stride, int32_t iters, double *tops, double *cycles_per_mma)
 {
     if (!tops || !cycles_per_mma || iters < 1 || iters > (1 << 22) || block_n < 16 || block_n > 256 || block_n % 16) return -1;
     int dev = 0, sms = 0;
@@ -102,7 +127,7 @@ extern "C" __attribute__((visibility("default"))) int probe_mma_rate(int32_t blo
     if (err == cudaSuccess) err = cudaEventCreate(&e1);
     for (int rep = 0; rep < 2 && err == cudaSuccess; ++rep) {      // the first launch warms up
         if (err == cudaSuccess) err = cudaEventRecord(e0, 0);
-        mma_rate_kernel<<<sms, 128, smem, 0>>>(block_n, iters, d_res);
+        mma_rate_kernel<<<sms, 128, smem, 0>>>(block_n, row_bytes, a_group_stride, iters, d_res);
         if (err == cudaSuccess) err = cudaGetLastError();
         if (err == cudaSuccess) err = cudaEventRecord(e1, 0);
         if (err == cudaSuccess) err = cudaEventSynchronize(e1);

@@ -603,9 +603,14 @@ void window_plan(iconv_plan_t *p)
     p->win_vw = vw; p->win_bw = bw; p->win_bh = bh; p->win_full_width = full_width; p->win_blocks = blocks; p->win_tpi = (int)tpi;
     p->win_patch_bytes = (int)patch;
     p->win_stages = (int)(room / patch < 6 ? room / patch : 6);
-    // sixteen epilogue warps: no staging memory is needed here
+    // Sixteen epilogue warps (no staging memory is needed here), and twice as many accumulator buffers
+    // as tiles in flight wherever the 512 TMEM columns allow it: a buffer belongs to one group of warps,
+    // so with as many tiles in flight as buffers the MMAs of a group's next tile could only start once
+    // its epilogue had ended, and the two never overlapped.
     const int slots = 4;
-    p->bi = slots < p->nbuf ? slots : p->nbuf;
+    p->win_nbuf = p->block_n <= 64 ? 8 : p->nbuf;
+    p->bi = p->win_nbuf / 2 < slots ? p->win_nbuf / 2 : slots;
+    if (p->bi < 1) p->bi = 1;
     p->cs = slots / p->bi;
     while (p->cs > 1 && p->block_n < 32 * p->cs) p->cs /= 2;
     p->half_n = p->cs > 1 ? (p->block_n / p->cs + 15) / 16 * 16 : p->block_n;
@@ -835,11 +840,11 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     u.slot_bytes = u.slot_a_bytes + (p->resident_b ? 0 : (p->pair ? u.b_tile_bytes / 2 : u.b_tile_bytes));
     u.stage_bytes = u.kg * u.slot_bytes;
     u.producers = p->stages * p->kg < NUM_PRODUCERS ? p->stages * p->kg : NUM_PRODUCERS;
-    u.nbuf = p->nbuf;
-    u.lg_nbuf = p->nbuf == 4 ? 2 : 1;
+    u.nbuf = p->window ? p->win_nbuf : p->nbuf;
+    u.lg_nbuf = u.nbuf == 8 ? 3 : u.nbuf == 4 ? 2 : 1;
     int cols = 32;
     u.acc_cols = p->block_n * (p->proj_iters ? 2 : 1);
-    while (cols < p->nbuf * u.acc_cols) cols *= 2;
+    while (cols < u.nbuf * u.acc_cols) cols *= 2;
     u.tmem_cols = cols;
     u.epi_warps = p->epi_warps;
     u.cs = p->cs;

@@ -50,7 +50,7 @@ constexpr int SKIP_RING = 3;              // staged skip pieces per epilogue war
 constexpr int EPI_WARP_SMEM = 8192;       // per epilogue warp: two output pieces of up to 4 KB together (int32 outputs)
 constexpr int EPI_WARP_SMEM_SMALL = 4096; // ... when the output is 8-bit (pieces of 2 KB) and no 8-bit skip is staged
 constexpr int MAX_STAGES = 12;
-constexpr int MAX_TMEM_BUFS = 4;
+constexpr int MAX_TMEM_BUFS = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds at the boost clock
 constexpr int MAX_SMEM = 227 * 1024;
 constexpr int RESIDENT_B_MAX = 80 * 1024;
@@ -79,7 +79,7 @@ struct UmmaArgs {
     int stages, kg;                 // pipeline stages; k-iterations (slots) per stage
     int slot_a_bytes, slot_bytes, stage_bytes, b_tile_bytes, resident_b;
     int producers;                  // active TMA warps: min(NUM_PRODUCERS, stages * kg)
-    int tmem_cols, nbuf, lg_nbuf;   // accumulator buffers (2 or 4)
+    int tmem_cols, nbuf, lg_nbuf;   // accumulator buffers (2 or 4; window mode up to 8)
     int epi_warps, cs, bi;          // epilogue warps, column split per tile, tiles in flight
     int part_n;                     // columns one epilogue warp handles per tile
     int piece_bytes;                // row width of one staged output piece (16 ... 128 bytes)
@@ -1141,13 +1141,13 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
 }
 
-// Window-mode epilogue of one warp and tile: groups of 16 columns from TMEM (the first one
-// already requested into accA), each through the layer's epilogue and out with one 16-byte
-// store per pixel.  NG: the number of groups when known at compile time (0: `ngroups`).
+// Window-mode epilogue of one warp and tile: groups of 16 columns from TMEM (one register block,
+// load and wait in one step: a second block with the next group in flight measured no faster),
+// each through the layer's epilogue and out with one 16-byte store per pixel.  NG: the number of groups when known at compile time (0: `ngroups`).
 // GU: per-channel parameters that are uniform per group (fetched group by group).
 template <int EPI, int NG, bool GU>
 __device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, uint8_t *ocol, const uint8_t *scol, bool valid, int col_lo,
-                                              int ngroups, int *accA, int *accB, const EpiScalars &es, const ConvArgs &a, const UmmaArgs &u)
+                                              int ngroups, int *accA, const EpiScalars &es, const ConvArgs &a, const UmmaArgs &u)
 {
     constexpr bool SKIP8 = (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8);    // scol: this pixel's 8-bit skip row, read directly
     const int ng = NG ? NG : ngroups;
@@ -1164,11 +1164,10 @@ __device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, u
             for (int g = 0; g < 4; ++g) ca[g] = __ldg(cap + 4 * gcur + g);
             uint4 sk = make_uint4(0, 0, 0, 0);
             if (SKIP8 && valid && co0 < a.c_out) sk = __ldg((const uint4 *)(scol + (gcur << 4)));
-            tmem_ld_wait();
-            if (gcur + 1 < ng) tmem_ld16(t_row + (uint32_t)((gcur + 1) << 4), hf ? accA : accB);
+            tmem_ld16_sync(t_row + (uint32_t)(gcur << 4), accA);
             int V[16];
-            if (GU) epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, sk, group_scalars(es, u, co0), a, u);
-            else epilogue16<EPI>(hf ? accB : accA, accA, V, ca, co0, 0, false, sk, es, a, u);
+            if (GU) epilogue16<EPI>(accA, accA, V, ca, co0, 0, false, sk, group_scalars(es, u, co0), a, u);
+            else epilogue16<EPI>(accA, accA, V, ca, co0, 0, false, sk, es, a, u);
             uint4 o;
             if (EPI == EPI_FAST || EPI == EPI_FAST_SKIP8 || a.out_dtype == ICONV_U8) {
                 o.x = pack4_sat<false>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<false>(V[4], V[5], V[6], V[7]);
@@ -1382,9 +1381,9 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * u.block_n + col_lo);
             const int ngroups = ncols >> 4;
-            int accA[16], accB[16];
-            tmem_ld16(t_row, accA);
+            int accA[16];
             if (EPI == EPI_NARROW) {
+                tmem_ld16(t_row, accA);
                 // a handful of channels per pixel (the regression networks' last layer): the general
                 // 64-bit epilogue channel by channel, the skip read and the output written byte-wise
                 const long long mpix = ((long long)img * a.h_out + y) * a.w_out + xq;
@@ -1415,12 +1414,12 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 if (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8)
                     scol = (const uint8_t *)a.skip + (((long long)img * a.h_out + y) * a.w_out + xq) * a.skip_c_total + a.skip_c_offset + col_lo;
                 // the usual widths get straight-line code: every offset an immediate, no loop control
-                if (es.group_uniform) window_groups<EPI, 0, true>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 4) window_groups<EPI, 4, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 3) window_groups<EPI, 3, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 2) window_groups<EPI, 2, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else if (ngroups == 1) window_groups<EPI, 1, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
-                else window_groups<EPI, 0, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, accB, es, a, u);
+                if (es.group_uniform) window_groups<EPI, 0, true>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, es, a, u);
+                else if (ngroups == 4) window_groups<EPI, 4, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, es, a, u);
+                else if (ngroups == 3) window_groups<EPI, 3, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, es, a, u);
+                else if (ngroups == 2) window_groups<EPI, 2, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, es, a, u);
+                else if (ngroups == 1) window_groups<EPI, 1, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, es, a, u);
+                else window_groups<EPI, 0, false>(t_row, cap, ocol, scol, valid, col_lo, ngroups, accA, es, a, u);
             }
             tc_fence_before();
             __syncwarp();

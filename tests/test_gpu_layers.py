@@ -413,6 +413,12 @@ def test_mma_issue_rate_probe_reports_a_plausible_peak():
     assert 1000.0 < tops < 10000.0
     with pytest.raises(RuntimeError):
         bench.probe_mma_rate(100, 10)
+    # 64-byte rows with the block tiling's group stride, 64 columns: half the work per instruction at
+    # about the same duration
+    tops64, cycles64 = bench.probe_mma_rate_rows(64, 64, 640, 20000)
+    assert 30.0 <= cycles64 <= 200.0 and tops64 < tops
+    with pytest.raises(RuntimeError):
+        bench.probe_mma_rate_rows(64, 48, 512, 10)
 
 
 THIN_SHAPES = [
