@@ -609,6 +609,18 @@ void window_plan(iconv_plan_t *p)
     // its epilogue had ended, and the two never overlapped.
     const int slots = 4;
     p->win_nbuf = p->block_n <= 64 ? 8 : p->nbuf;
+    // MMA-issuing warps: three with six stages and eight accumulator buffers, else two with an even number of
+    // stages.  The issuers take the tiles in turn and wait on barriers by phase parity, which tells a phase only
+    // from its neighbours: a stage's fills must all pass through one issuer (issuers divide stages), and an
+    // issuer must never be a whole round of accumulator buffers ahead of the others (stages <= buffers, or
+    // issuers divide buffers).
+    if (p->win_stages >= 6 && p->win_nbuf >= 8) {
+        p->win_stages = 6;
+        p->win_issuers = 3;
+    } else {
+        p->win_stages = p->win_stages / 2 * 2;
+        p->win_issuers = 2;
+    }
     p->bi = p->win_nbuf / 2 < slots ? p->win_nbuf / 2 : slots;
     if (p->bi < 1) p->bi = 1;
     p->cs = slots / p->bi;
@@ -815,6 +827,7 @@ int launch_umma(const iconv_plan_t *p, const ConvArgs &a, cudaStream_t stream)
     UmmaArgs u;
     u.win_vw = p->win_vw; u.win_bw = p->win_bw; u.win_bh = p->win_bh; u.win_full_width = p->win_full_width; u.win_tpi = p->win_tpi;
     u.win_blocks = p->win_blocks;
+    u.win_issuers = p->win_issuers;
     find_divisor((unsigned)(p->win_tpi > 0 ? p->win_tpi : 1), u.div_tpi_mul, u.div_tpi_shr);
     find_divisor((unsigned)(p->win_vw > 0 ? p->win_vw : 1), u.div_vw_mul, u.div_vw_shr);
     u.m_total = (long long)d.n * p->h_out * p->w_out;

@@ -23,7 +23,7 @@ struct iconv_plan_s {
     int half_n = 0, piece_bytes = 0;   // columns per epilogue warp and staged piece width
     int proj_c_in_pad = 0, proj_iters = 0, proj32 = 0;   // fused projection: padded channels, k-iterations, 32-bit rescale proven
     // window mode of the tensor-core kernel (stride-1 filters: one patch load per tile)
-    int window = 0, win_vw = 0, win_bw = 0, win_bh = 0, win_full_width = 0, win_blocks = 0, win_tpi = 0, win_patch_bytes = 0, win_stages = 0, win_nbuf = 0;
+    int window = 0, win_vw = 0, win_bw = 0, win_bh = 0, win_full_width = 0, win_blocks = 0, win_tpi = 0, win_patch_bytes = 0, win_stages = 0, win_nbuf = 0, win_issuers = 2;
     int thin_narrow = 0;     // thin kernels: BReLU + Eq. 4 provably fit 32 bits
     int kg = 1;              // k-iterations grouped behind one pair of pipeline barriers
     int nbuf = 2;            // TMEM accumulator buffers

@@ -43,6 +43,8 @@ constexpr int EPI_WARPS_MAX = 16;
 constexpr int NUM_PRODUCERS = 3;          // TMA warps: one thread issues a load per 300-400 cycles, the unit takes three times that
 constexpr int MMA_WARP = NUM_PRODUCERS;
 constexpr int MMA_WARP2 = 1;           // window mode (one TMA warp): a second MMA issuer
+constexpr int MMA_WARP3 = 2;           // ... and a third
+constexpr int WIN_ISSUERS = 3;
 constexpr int EPI_WARP0 = 4;              // first epilogue warp (a multiple of 4: warp % 4 is its TMEM lane quadrant)
 constexpr int NUM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS_MAX);
 constexpr int FAST_SKIP_SHIFT = 8;         // the skip shift the clamp-free epilogue forms are compiled for (what iq_skip_sync yields unless the skip is scaled down a lot)
@@ -101,6 +103,7 @@ struct UmmaArgs {
     int win_vw, win_bw, win_bh, win_full_width, win_tpi;    // virtual row width, patch width / height, mode, tiles per image
     int win_tap_step;               // patch positions between two horizontal taps (2 with paired taps)
     int win_blocks;                 // 1: tiles are blocks of 8 x 16 output pixels (win_vw = blocks per image row)
+    int win_issuers;                // MMA-issuing warps (2 or 3): a divisor of the number of stages, see window_plan
     unsigned desc_hi_a;             // upper descriptor word of the A operand in block mode (8-row groups one patch line apart)
     unsigned div_tpi_mul, div_tpi_shr, div_vw_mul, div_vw_shr;
     // exact division of a tile index by n_tiles and of a pixel index by w_out and by
@@ -1219,7 +1222,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             mbar_init(smem_u32(&sh->tmem_empty[b]), (uint32_t)(4 * u.cs));
         }
         mbar_init(smem_u32(&sh->b_full), 1);
-        mbar_init(smem_u32(&sh->drain), 2);          // one arrival per MMA issuer
+        mbar_init(smem_u32(&sh->drain), WIN_ISSUERS);          // one arrival per MMA issuer
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         grid_dep_launch();
@@ -1272,18 +1275,25 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
         }
         __syncwarp();
-    } else if (warp == MMA_WARP || warp == MMA_WARP2) {
+    } else if (warp == MMA_WARP || warp == MMA_WARP2 || warp == MMA_WARP3) {
         // ---------------------------------------------------------------- MMA issuers
-        // Two threads issue alternate tiles.  Between two tiles an issuer spends several hundred
+        // Three warps issue the tiles in turn.  Between two tiles an issuer spends several hundred
         // cycles on its barrier round (two commits, two waits), longer than the tensor pipe's
-        // queue covers; with two issuers one thread's round hides behind the other's MMAs.
+        // queue covers; one issuer's round hides behind the others' MMAs.
         // Tiles are independent (own accumulator buffer, own patch), so no order is needed
-        // between the two instruction streams, and each thread's commits cover its own MMAs.
-        const int which = warp == MMA_WARP ? 0 : 1;
-        if (lane == 0 && (int)blockIdx.x + which * (int)gridDim.x < num_tiles) {
+        // between the instruction streams, and each issuer's commits cover its own MMAs.
+        // The whole warp walks the tiles and waits (warp-uniform control flow: addresses and descriptors
+        // are then computed in uniform registers, which is where the MMA instruction takes them from);
+        // one elected lane issues.  With the loop inside a single-lane branch every operand of every MMA
+        // had to be moved over from a vector register, and the lone thread could not keep the pipe fed.
+        // A stage's fills all go through the same issuer (the number of issuers divides the number of
+        // stages): a parity wait tells a phase only from its neighbours, so the thread that waits for a
+        // stage's next fill must be the one that consumed the fill before.
+        const int which = warp == MMA_WARP ? 0 : warp == MMA_WARP2 ? 1 : 2;
+        if (which < u.win_issuers && (int)blockIdx.x + which * (int)gridDim.x < num_tiles) {
             int t = which, stage = which % u.stages;
             uint32_t parity = (uint32_t)((which / u.stages) & 1);
-            bool ok = mbar_wait(smem_u32(&sh->b_full), 0, &sh->abort_flag);
+            bool ok = mbar_wait_warp(smem_u32(&sh->b_full), 0, &sh->abort_flag, lane);
             if (!ok) give_up(sh, u.status, 6);
             const int kj = u.kc >> 5;
             const uint32_t desc_hi32 = (uint32_t)(u.desc_hi >> 32);
@@ -1294,7 +1304,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const uint32_t b_step = (uint32_t)u.b_tile_bytes >> 4;
             const uint32_t line_step = (uint32_t)u.win_bw * row_step;
             const uint32_t tap_step = (uint32_t)u.win_tap_step * row_step;
-            for (int tile = blockIdx.x + which * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x, t += 2) {
+            for (int tile = blockIdx.x + which * gridDim.x; tile < num_tiles && ok; tile += u.win_issuers * gridDim.x, t += u.win_issuers) {
                 const int buf = t & (u.nbuf - 1);
                 uint32_t off0 = 0;
                 if (u.win_full_width) {
@@ -1302,19 +1312,20 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     const unsigned i0 = (unsigned)(tile - img * u.win_tpi) * BLOCK_M;
                     off0 = i0 - fast_div(i0, u.div_vw_mul, u.div_vw_shr) * (unsigned)u.win_vw;
                 }
-                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
+                if (!mbar_wait_warp(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag, lane)) {
                     give_up(sh, u.status, 2);
                     break;
                 }
                 tc_fence_after();
-                if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
+                if (!mbar_wait_warp(smem_u32(&sh->full[stage]), parity, &sh->abort_flag, lane)) {
                     give_up(sh, u.status, 3);
                     break;
                 }
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * u.block_n);
                 uint32_t a_line = a_lo0 + (uint32_t)stage * stage_step + off0 * row_step;
                 uint32_t b_lo = b_lo0;
-                if (KH) {
+                if (!elect_one()) {
+                } else if (KH) {
 #pragma unroll
                     for (int r = 0; r < (KH ? KH : 1); ++r) {
 #pragma unroll
@@ -1338,9 +1349,11 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         a_line += line_step;
                     }
                 }
-                umma_commit(smem_u32(&sh->empty[stage]));
-                umma_commit(smem_u32(&sh->tmem_full[buf]));
-                stage += 2;
+                if (elect_one()) {
+                    umma_commit(smem_u32(&sh->empty[stage]));
+                    umma_commit(smem_u32(&sh->tmem_full[buf]));
+                }
+                stage += u.win_issuers;
                 if (stage >= u.stages) { stage -= u.stages; parity ^= 1u; }
             }
         }
@@ -1438,7 +1451,7 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const long long t0 = clock64();
             while (clock64() - t0 < 2000000) {}
         }
-        if ((warp == MMA_WARP || warp == MMA_WARP2) && lane == 0) {
+        if ((warp == MMA_WARP || warp == MMA_WARP2 || warp == MMA_WARP3) && lane == 0) {
             umma_commit(smem_u32(&sh->drain));
             mbar_wait(smem_u32(&sh->drain), 0, &never);
         }

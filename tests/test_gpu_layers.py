@@ -582,3 +582,25 @@ def test_window_mode_with_identity_skip_matches_oracle(shape, skip_dtype, varian
         bad = np.argwhere(got != want)
         assert bad.shape[0] == 0, "%s: %d mismatches, first at %s: got %s want %s" % (
             text[0], bad.shape[0], bad[0], got[tuple(bad[0])], want[tuple(bad[0])])
+
+
+MANY_TILE_SHAPES = [
+    # enough tiles that every MMA-issuing warp of a CTA takes several and the stage and accumulator rings wrap
+    # many times: n, h, w, c_in, c_out, text the plan must show
+    (96, 28, 28, 128, 128, "stages=2"),         # tiles across image rows, two stages (a large filter bank): two issuers
+    (6, 256, 256, 64, 64, "stages=6"),          # six stages, eight accumulator buffers: three issuers
+    (40, 56, 56, 64, 64, "window(blocks)"),     # ragged blocks at the bottom of every image
+]
+
+
+@pytest.mark.parametrize("shape", MANY_TILE_SHAPES, ids=lambda s: "x".join(map(str, s[:5])))
+def test_window_mode_with_many_tiles_per_cta_matches_oracle(shape):
+    """The issuing warps take a CTA's tiles in turn and wait by phase parity; every stage's fills must stay with
+    one of them.  Several hundred to several thousand tiles on the GPU's CTAs, against the oracle."""
+    n, h, w, c_in, c_out, expect = shape
+    X, W, b, mul, shift, h_i = _layer(sum(shape[:5]) + 37, n, h, w, c_in, c_out, 3)
+    want = oracle_conv(X, W, b, mul, shift, h_i, pad=1)
+    text = []
+    got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, kernel=B.KERNEL_UMMA, describe=text)
+    assert fam == B.KERNEL_UMMA and "window" in text[0] and expect in text[0], text
+    assert np.array_equal(got, want)
