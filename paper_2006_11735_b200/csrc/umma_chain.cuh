@@ -140,8 +140,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         __syncwarp();
     } else if (warp == MMA_WARP) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0 && T > 0) {
-            bool ok = mbar_wait(smem_u32(&sh->w_full), 0, &sh->abort_flag);
+        // (the whole warp walks the tiles and waits, so that addresses and descriptors are computed in uniform
+        // registers, where the MMA instruction takes them from; one elected lane issues)
+        if (T > 0) {
+            bool ok = mbar_wait_warp(smem_u32(&sh->w_full), 0, &sh->abort_flag, lane);
             if (!ok) chain_give_up(sh, c.status, 6);
             const int kj1 = c.k1 >> 5;
             const uint32_t a1_lo0 = ((smem_u32(a1) & 0x3FFFFu) >> 4) | (1u << 16);
@@ -156,8 +158,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             // the tile's 128 input channels, into the accumulator of the tile's pixel tile
             int ps = 0, pn = 0;                      // pixel tile and N tile of the tile before the current one
             auto second = [&](int tt, int ss, int nn) -> bool {
-                if (!mbar_wait(smem_u32(&sh->a2_full[tt & 1]), (uint32_t)((tt >> 1) & 1), &sh->abort_flag)) { chain_give_up(sh, c.status, 3); return false; }
-                if (nn == 0 && !mbar_wait(smem_u32(&sh->d2_empty[ss & 1]), (uint32_t)(((ss >> 1) & 1) ^ 1), &sh->abort_flag)) {
+                if (!mbar_wait_warp(smem_u32(&sh->a2_full[tt & 1]), (uint32_t)((tt >> 1) & 1), &sh->abort_flag, lane)) { chain_give_up(sh, c.status, 3); return false; }
+                if (nn == 0 && !mbar_wait_warp(smem_u32(&sh->d2_empty[ss & 1]), (uint32_t)(((ss >> 1) & 1) ^ 1), &sh->abort_flag, lane)) {
                     chain_give_up(sh, c.status, 2);
                     return false;
                 }
@@ -165,11 +167,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const uint32_t d2 = tmem_base + 256u + (uint32_t)((ss & 1) * 128);
                 const uint32_t a_lo = a2_lo0 + (uint32_t)((tt & 1) * (16384 >> 4));
                 const uint32_t b_lo = w2_lo0 + (uint32_t)(nn * (w2_tile >> 4));
+                if (elect_one()) {
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch)
-                    umma_i8_split2(d2, a_lo + (uint32_t)(ch * (4096 >> 4)), a2_hi, b_lo + 2u * (uint32_t)ch, w2_hi, c.idesc2, (uint32_t)(nn != 0 || ch != 0));
-                umma_commit(smem_u32(&sh->a2_empty[tt & 1]));
-                if (nn == c.n_tiles - 1) umma_commit(smem_u32(&sh->d2_full[ss & 1]));
+                    for (int ch = 0; ch < 4; ++ch)
+                        umma_i8_split2(d2, a_lo + (uint32_t)(ch * (4096 >> 4)), a2_hi, b_lo + 2u * (uint32_t)ch, w2_hi, c.idesc2, (uint32_t)(nn != 0 || ch != 0));
+                    umma_commit(smem_u32(&sh->a2_empty[tt & 1]));
+                    if (nn == c.n_tiles - 1) umma_commit(smem_u32(&sh->d2_full[ss & 1]));
+                }
                 return true;
             };
             int s = 0, nt = 0, st = 0;
@@ -177,16 +181,18 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             for (int t = 0; t < T && ok; ++t) {
                 // (accumulator buffer t & 1 is free: the second GEMM of tile t - 2, issued in the round before this
                 // one, waited until every epilogue warp had staged that tile, i.e. had read the buffer)
-                if (nt == 0 && !mbar_wait(smem_u32(&sh->a1_full[st]), a1_parity, &sh->abort_flag)) {
+                if (nt == 0 && !mbar_wait_warp(smem_u32(&sh->a1_full[st]), a1_parity, &sh->abort_flag, lane)) {
                     chain_give_up(sh, c.status, 3);
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d1 = tmem_base + (uint32_t)((t & 1) * 128);
                 const uint32_t a_lo = a1_lo0 + (uint32_t)(st * (a1_bytes >> 4)), b_lo = w1_lo0 + (uint32_t)(nt * (w1_tile >> 4));
-                for (int j = 0; j < kj1; ++j) umma_i8_split(d1, a_lo + 2u * (uint32_t)j, b_lo + 2u * (uint32_t)j, c.desc_hi1, c.idesc1, (uint32_t)(j != 0));
-                umma_commit(smem_u32(&sh->acc1_full[t & 1]));
-                if (nt == c.n_tiles - 1) umma_commit(smem_u32(&sh->a1_empty[st]));
+                if (elect_one()) {
+                    for (int j = 0; j < kj1; ++j) umma_i8_split(d1, a_lo + 2u * (uint32_t)j, b_lo + 2u * (uint32_t)j, c.desc_hi1, c.idesc1, (uint32_t)(j != 0));
+                    umma_commit(smem_u32(&sh->acc1_full[t & 1]));
+                    if (nt == c.n_tiles - 1) umma_commit(smem_u32(&sh->a1_empty[st]));
+                }
                 if (t > 0) ok = second(t - 1, ps, pn);
                 ps = s; pn = nt;
                 if (++nt == c.n_tiles) { nt = 0; ++s; if (++st == c.stages) { st = 0; a1_parity ^= 1u; } }

@@ -415,7 +415,8 @@ struct IssueRing {
 };
 // `rounds` pipeline stages of one 128-byte k-iteration each into the accumulator at d_tmem:
 // wait for the stage, four MMAs (A at a_lo, B right behind it in the stage), commit the stage.
-// Straight-line apart from the loop itself; returns false when a wait gave up.
+// Run by the whole issuing warp (the ring position is warp-uniform and lives in uniform registers,
+// where the MMA takes its operands from); one elected lane issues.  Returns false when a wait gave up.
 template <bool PAIR_>
 __device__ __forceinline__ bool issue_rounds(IssueRing &g, uint32_t d_tmem, uint32_t idesc, int rounds, int stages, uint32_t a_lo0,
                                              uint32_t stage_step, uint32_t slot_a_step, uint32_t desc_hi32, uint32_t full0,
@@ -423,8 +424,9 @@ __device__ __forceinline__ bool issue_rounds(IssueRing &g, uint32_t d_tmem, uint
 {
     uint32_t acc = 0;
     for (int ki = 0; ki < rounds; ++ki) {
-        if (!mbar_test_wait(g.full_bar, g.parity) && !mbar_wait(g.full_bar, g.parity, abort_flag)) return false;
-        if (PAIR_) {
+        if (!mbar_wait_warp(g.full_bar, g.parity, abort_flag, 0)) return false;
+        if (!elect_one()) {
+        } else if (PAIR_) {
             // one instruction covers both CTAs' 128 rows; the stage is released in both CTAs
             umma_i8_pair(d_tmem, g.a_lo, g.a_lo + slot_a_step, desc_hi32, idesc, acc);
 #pragma unroll
@@ -702,7 +704,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // ISSUE 3: the long-reduction path on CTA pairs.  A "tile" is then 256 pixels x block_n: this CTA's
     // pixel tile is 2 * (tile / n_tiles) + rank, u.m_tiles counts pixel-tile pairs, the grid is walked pair by pair.
     constexpr bool PAIR = ISSUE == 3;
-    const uint32_t rank = PAIR ? cluster_rank() : 0u;
+    const uint32_t rank = PAIR ? __shfl_sync(0xffffffffu, cluster_rank(), 0) : 0u;    // (known to the compiler as warp-uniform)
     const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, tile_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
     // tiles need the alignment of the widest swizzle pattern (8 rows x 128 bytes)
@@ -858,11 +860,15 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         __syncwarp();
     } else if (warp == MMA_WARP) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0 && tile0 < num_tiles && (!PAIR || rank == 0)) {
+        // The whole warp walks the tiles and waits (warp-uniform control flow: ring positions and
+        // descriptors are computed in uniform registers, where the MMA instruction takes them from);
+        // one elected lane issues.  (The TMA producers stay single-lane loops: the same change
+        // measured no different there.)
+        if (tile0 < num_tiles && (!PAIR || rank == 0)) {
             int t = 0, stage = 0;
             uint32_t parity = 0;
             bool ok = true;
-            if (u.resident_b && !mbar_wait(smem_u32(&sh->b_full), 0, &sh->abort_flag)) {
+            if (u.resident_b && !mbar_wait_warp(smem_u32(&sh->b_full), 0, &sh->abort_flag, lane)) {
                 give_up(sh, u.status, 6);
                 ok = false;
             }
@@ -876,7 +882,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
             for (int tile = tile0; tile < num_tiles && ok; tile += tile_stride, ++t) {
                 const int buf = t & (u.nbuf - 1);
-                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag)) {
+                if (!mbar_wait_warp(smem_u32(&sh->tmem_empty[buf]), (uint32_t)(((t >> u.lg_nbuf) & 1) ^ 1), &sh->abort_flag, lane)) {
                     give_up(sh, u.status, 2);
                     break;
                 }
@@ -891,19 +897,21 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     // The short reductions (the whole tile in one stage, the filter bank resident): one
                     // wait, the tile's MMAs, two commits, with as few branches as the lone thread can do with.
                     const uint32_t full_bar = full0 + 8u * (uint32_t)stage;
-                    if (!mbar_test_wait(full_bar, parity) && !mbar_wait(full_bar, parity, &sh->abort_flag)) {
+                    if (!mbar_wait_warp(full_bar, parity, &sh->abort_flag, lane)) {
                         give_up(sh, u.status, 3);
                         break;
                     }
-                    uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step, b_lo = sb;
-                    umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, 0u);
-                    for (int e = 1; e < k_iters; ++e) {
-                        a_lo += slot_step;
-                        b_lo += b_step;
-                        umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, 1u);
+                    if (elect_one()) {
+                        uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step, b_lo = sb;
+                        umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, 0u);
+                        for (int e = 1; e < k_iters; ++e) {
+                            a_lo += slot_step;
+                            b_lo += b_step;
+                            umma_slot<4>(d_tmem, a_lo, b_lo, desc_hi32, u.idesc, 1u);
+                        }
+                        umma_commit(empty0 + 8u * (uint32_t)stage);
+                        umma_commit(smem_u32(&sh->tmem_full[buf]));
                     }
-                    umma_commit(empty0 + 8u * (uint32_t)stage);
-                    umma_commit(smem_u32(&sh->tmem_full[buf]));
                     const bool wrap = ++stage == u.stages;
                     stage = wrap ? 0 : stage;
                     parity ^= wrap ? 1u : 0u;
@@ -929,12 +937,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                                 &sh->abort_flag);
                     }
                     stage = ring.stage; parity = ring.parity;
-                    if (ok) { if (PAIR) umma_commit_pair(smem_u32(&sh->tmem_full[buf])); else umma_commit(smem_u32(&sh->tmem_full[buf])); }
-                    else give_up(sh, u.status, 3);
+                    if (!ok) give_up(sh, u.status, 3);
+                    else if (elect_one()) { if (PAIR) umma_commit_pair(smem_u32(&sh->tmem_full[buf])); else umma_commit(smem_u32(&sh->tmem_full[buf])); }
                     continue;
                 }
                 for (int ki = 0; ISSUE == 0 && ki < k_iters;) {
-                    if (!mbar_wait(smem_u32(&sh->full[stage]), parity, &sh->abort_flag)) {
+                    if (!mbar_wait_warp(smem_u32(&sh->full[stage]), parity, &sh->abort_flag, lane)) {
                         give_up(sh, u.status, 3);
                         ok = false;
                         break;
@@ -943,15 +951,17 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_step;
                     uint32_t b_lo = u.resident_b ? sb : a_lo + slot_a_step;
                     const int in_stage = min(u.kg, k_iters - ki);
-                    if (kj == 4) umma_stage<4>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
-                    else if (kj == 2) umma_stage<2>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
-                    else umma_stage<1>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
+                    if (elect_one()) {
+                        if (kj == 4) umma_stage<4>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
+                        else if (kj == 2) umma_stage<2>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
+                        else umma_stage<1>(d_tmem, (uint32_t)u.block_n, a_lo, b_lo, slot_step, b_step, desc_hi32, u.idesc, u.idesc_p, ki, in_stage, EPI == EPI_PROJ ? u.p_iters : 0);
+                        umma_commit(smem_u32(&sh->empty[stage]));   // frees the stage when these MMAs are done
+                    }
                     ki += in_stage;
                     if (u.resident_b) sb = b_lo + (uint32_t)in_stage * b_step;
-                    umma_commit(smem_u32(&sh->empty[stage]));   // frees the stage when these MMAs are done
                     if (++stage == u.stages) { stage = 0; parity ^= 1u; }
                 }
-                if (ok) umma_commit(smem_u32(&sh->tmem_full[buf]));
+                if (ok && elect_one()) umma_commit(smem_u32(&sh->tmem_full[buf]));
             }
         }
         __syncwarp();
