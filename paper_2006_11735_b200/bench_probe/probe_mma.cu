@@ -53,13 +53,18 @@ __global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int row_bytes, 
         const unsigned long long db = hi_b | (unsigned long long)((probe_smem_u32(tiles + 16384) & 0x3FFFFu) >> 4) | (1ull << 16);
         const uint32_t idesc = (2u << 4) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((128u >> 4) << 24);   // u8 x s8 -> s32
         const unsigned slices = (unsigned)(row_bytes >> 5);
+        // four instructions per loop round, their K-slice offsets fixed before the loop: whatever the issuing
+        // thread executes between two instructions shows in the rate once the pipe's queue runs empty
+        unsigned long long koff[4];
+        for (int j = 0; j < 4; ++j) koff[j] = 2ull * ((unsigned)j & (slices - 1));    // walk the 32-byte K slices of a row
         const long long t0 = clock64();
-        for (int i = 0; i < iters; ++i) {
-            const unsigned long long k = 2ull * ((unsigned)i & (slices - 1));    // walk the 32-byte K slices of a row
-            asm volatile(
-                "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-                ::"r"(tb), "l"(da + k), "l"(db + k), "r"(idesc), "r"(i) : "memory");
+        for (int i = 0; i < iters; i += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                    "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                    ::"r"(tb), "l"(da + koff[j]), "l"(db + koff[j]), "r"(idesc), "r"(i + j) : "memory");
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(probe_smem_u32(&bar)) : "memory");
         int timed_out = 1;
@@ -90,6 +95,7 @@ using namespace iconv_probe;
 // u8 x s8 -> s32) when only the instruction stream limits it: one thread per SM issues `iters`
 // dependent instructions on operands in shared memory.  Writes whole-GPU TOP/s (2 * MACs / event
 // time of the launch) and the slowest SM's cycles per instruction to the HOST pointers.
+// `iters` is a multiple of 4 (the issue loop is unrolled four times).
 // Synchronous; allocates a few KB on the current device.  Returns 0, -1 (bad argument),
 // -6 (a CUDA call failed) or -7 (the bounded wait for the last instruction ran out).
 //
@@ -114,7 +120,7 @@ extern "C" __attribute__((visibility("default"))) int probe_mma_rate_rows(int32_
 
 static int probe_run(int32_t block_n, int32_t row_bytes, int32_t a_group_stride, int32_t iters, double *tops, double *cycles_per_mma)
 {
-    if (!tops || !cycles_per_mma || iters < 1 || iters > (1 << 22) || block_n < 16 || block_n > 256 || block_n % 16) return -1;
+    if (!tops || !cycles_per_mma || iters < 4 || iters % 4 || iters > (1 << 22) || block_n < 16 || block_n > 256 || block_n % 16) return -1;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -6;
     const size_t smem = 16384 + 32768 + 1024;
