@@ -471,6 +471,13 @@ __device__ __forceinline__ void tmem_ld16_sync(uint32_t taddr, int *r, uint4 dep
         : "r"(taddr), "r"(dep.x), "r"(dep.y), "r"(dep.z), "r"(dep.w)    // dep: values that must exist before the registers are reloaded
         : "memory");
 }
+// 32 bytes to a 32-byte-aligned global address in one store
+__device__ __forceinline__ void st_global_32(void *p, uint4 a, uint4 b)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x),
+                 "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // d = { sat8(v3), sat8(v2), sat8(v1), sat8(v0) } (v0 in the low byte), unsigned or signed saturation
@@ -1164,6 +1171,8 @@ __device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, u
 {
     constexpr bool SKIP8 = (EPI == EPI_FAST_SKIP8 || EPI == EPI_SAFE_SKIP8);    // scol: this pixel's 8-bit skip row, read directly
     const int ng = NG ? NG : ngroups;
+    const bool wide = (((uintptr_t)ocol) & 31u) == 0;      // this pixel's columns start on a 32-byte boundary
+    uint4 o_even = make_uint4(0, 0, 0, 0);
 #pragma unroll
     for (int gi = 0; gi < (NG ? NG : 16); gi += 2) {
         if (!NG && gi >= ng) break;
@@ -1189,7 +1198,19 @@ __device__ __forceinline__ void window_groups(uint32_t t_row, const int4 *cap, u
                 o.x = pack4_sat<true>(V[0], V[1], V[2], V[3]); o.y = pack4_sat<true>(V[4], V[5], V[6], V[7]);
                 o.z = pack4_sat<true>(V[8], V[9], V[10], V[11]); o.w = pack4_sat<true>(V[12], V[13], V[14], V[15]);
             }
-            if (valid && co0 < a.c_out) *(uint4 *)(ocol + (gcur << 4)) = o;
+            // Two groups of a pixel are 32 contiguous bytes: one 32-byte store writes a whole sector where two
+            // 16-byte stores wrote it in halves (with few MMAs per tile the epilogue's stores are the critical path:
+            // every 16-byte-per-lane store is 32 half-written sectors to the load/store unit).
+            if (hf == 0) {
+                o_even = o;
+                if ((!wide || gcur + 1 >= ng) && valid && co0 < a.c_out) *(uint4 *)(ocol + (gcur << 4)) = o;
+            } else if (!wide) {
+                if (valid && co0 < a.c_out) *(uint4 *)(ocol + (gcur << 4)) = o;
+            } else if (valid && co0 < a.c_out) {
+                st_global_32(ocol + ((gcur - 1) << 4), o_even, o);
+            } else if (valid && co0 - 16 < a.c_out) {
+                *(uint4 *)(ocol + ((gcur - 1) << 4)) = o_even;
+            }
         }
     }
 }
