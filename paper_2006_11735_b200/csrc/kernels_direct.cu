@@ -350,12 +350,66 @@ __global__ void __launch_bounds__(256) maxpool_3x3s2_kernel(const uint8_t *__res
     ((uint4 *)out)[e] = m;
 }
 
+// The same with 32 channels per thread (32-byte loads and one 32-byte store: half the memory
+// instructions, every store a whole sector), for channel counts that are multiples of 32 and
+// 32-byte aligned tensors.
+struct Bytes32 {
+    unsigned v[8];
+};
+__device__ __forceinline__ Bytes32 ld_global_32(const void *p)
+{
+    Bytes32 r;
+    asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+__global__ void __launch_bounds__(256) maxpool_3x3s2_wide_kernel(const uint8_t *__restrict__ x, uint8_t *__restrict__ out, unsigned total,
+                                                                 int h, int w, int cg, int h_out, int w_out)
+{
+    const unsigned e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const unsigned pix = e / (unsigned)cg;
+    const int g = (int)(e - pix * (unsigned)cg);
+    const unsigned row = pix / (unsigned)w_out;               // image * h_out + oh
+    const int ow = (int)(pix - row * (unsigned)w_out);
+    const unsigned in = row / (unsigned)h_out;
+    const int oh = (int)(row - in * (unsigned)h_out);
+    const uint8_t *base = x + ((size_t)in * h * w * cg + g) * 32;
+    Bytes32 v[9];
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int ih = min(max(2 * oh - 1 + r, 0), h - 1);
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            const int iw = min(max(2 * ow - 1 + s, 0), w - 1);
+            v[r * 3 + s] = ld_global_32(base + (size_t)(ih * w + iw) * cg * 32);
+        }
+    }
+    Bytes32 m = v[0];
+#pragma unroll
+    for (int t = 1; t < 9; ++t)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) m.v[k] = __vmaxu4(m.v[k], v[t].v[k]);
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(out + (size_t)e * 32), "r"(m.v[0]), "r"(m.v[1]), "r"(m.v[2]),
+                 "r"(m.v[3]), "r"(m.v[4]), "r"(m.v[5]), "r"(m.v[6]), "r"(m.v[7])
+                 : "memory");
+}
+
 int launch_maxpool(const void *x, void *out, int n, int h, int w, int c, int k, int stride, int pad,
                    cudaStream_t stream)
 {
     const int h_out = (h + 2 * pad - k) / stride + 1, w_out = (w + 2 * pad - k) / stride + 1;
     const long long total = (long long)n * h_out * w_out * (c / 16);
     if (total == 0) return ICONV_OK;
+    if (k == 3 && stride == 2 && pad == 1 && c % 32 == 0 && ((uintptr_t)x % 32) == 0 && ((uintptr_t)out % 32) == 0 && total < (1ll << 31) &&
+        (long long)n * h * w * (c / 16) < (1ll << 31)) {
+        const unsigned wide_total = (unsigned)(total / 2);
+        maxpool_3x3s2_wide_kernel<<<(wide_total + 255) / 256, 256, 0, stream>>>((const uint8_t *)x, (uint8_t *)out, wide_total, h, w, c / 32, h_out,
+                                                                                w_out);
+        ICONV_CUDA_TRY(cudaGetLastError());
+        return ICONV_OK;
+    }
     if (k == 3 && stride == 2 && pad == 1 && total < (1ll << 31) && (long long)n * h * w * (c / 16) < (1ll << 31)) {
         maxpool_3x3s2_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>((const uint8_t *)x, (uint8_t *)out, (unsigned)total, h, w,
                                                                                 c / 16, h_out, w_out);

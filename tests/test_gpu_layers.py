@@ -198,6 +198,21 @@ def test_pooling_matches_oracle():
         assert np.array_equal(out.get(), want)
 
 
+def test_maxpool_with_32_byte_accesses_matches_oracle():
+    """3x3/2 pooling over channel counts that are multiples of 32 on 32-byte aligned tensors takes the kernel
+    with 32-byte loads and stores; odd sizes, one-pixel images and several images."""
+    rng = np.random.default_rng(5)
+    for (n, h, w, c) in [(2, 16, 14, 64), (3, 7, 9, 32), (1, 1, 1, 96), (2, 112, 112, 64), (1, 5, 12, 128)]:
+        x = rng.integers(0, 256, size=(n, h, w, c), dtype=np.uint8)
+        want = L.maxpool(x, 3, 2, 1)
+        xd = dev(x)
+        out = torch.full(want.shape, 0x5A, dtype=torch.uint8, device="cuda")
+        assert xd.data_ptr() % 32 == 0 and out.data_ptr() % 32 == 0
+        B.ipool_max(xd.data_ptr(), out.data_ptr(), n, h, w, c, 3, 2, 1, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy(), want)
+
+
 UMMA_SHAPES = [
     # n, h, w, c_in, c_out, k, stride, pad
     (1, 32, 32, 64, 64, 3, 1, 1),       # configuration 1
