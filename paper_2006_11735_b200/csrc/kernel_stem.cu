@@ -28,37 +28,44 @@ namespace iconv {
 
 namespace {
 
-// One thread writes the 16 bytes of one position (n, Y, X) of T.
+// One thread writes the 16 bytes of one position (n, Y, X) of T.  The six input bytes of one image row
+// that a position holds (two pixels x three channels) are contiguous and start on an even address:
+// three 16-bit loads where both pixels are inside the image, byte loads at a ragged right edge.
 __global__ void __launch_bounds__(256)
 stem_repack_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ T, int n, int h, int w, int hp, int wp,
                    int raw128, int slack)
 {
-    const long long total = (long long)n * hp * wp;
-    for (long long pos = (long long)blockIdx.x * blockDim.x + threadIdx.x; pos < total;
-         pos += (long long)gridDim.x * blockDim.x) {
-        const int X = (int)(pos % wp);
-        const int Y = (int)((pos / wp) % hp);
-        const int img = (int)(pos / ((long long)wp * hp));
-        unsigned wds[4] = {0, 0, 0, 0};
+    const unsigned total = (unsigned)n * (unsigned)hp * (unsigned)wp;     // < 2^31 (checked by the caller)
+    const unsigned flip = raw128 ? 0x8080u : 0u;                           // raw - 128 as int8
+    for (unsigned pos = blockIdx.x * blockDim.x + threadIdx.x; pos < total; pos += gridDim.x * blockDim.x) {
+        const unsigned row = pos / (unsigned)wp;
+        const int X = (int)(pos - row * (unsigned)wp);
+        const unsigned img = row / (unsigned)hp;
+        const int Y = (int)(row - img * (unsigned)hp);
+        unsigned hw[6] = {0, 0, 0, 0, 0, 0};          // the twelve bytes as six 16-bit halves
+        const int iw = 2 * (X - 2);
 #pragma unroll
         for (int dy = 0; dy < 2; ++dy) {
             const int ih = 2 * (Y - 2) + dy;
-#pragma unroll
-            for (int dx = 0; dx < 2; ++dx) {
-                const int iw = 2 * (X - 2) + dx;
-                if (ih < 0 || ih >= h || iw < 0 || iw >= w) continue;    // zero padding
-                const uint8_t *p = in + (((long long)img * h + ih) * w + iw) * 3;
-#pragma unroll
-                for (int c = 0; c < 3; ++c) {
-                    const int k = (dy * 2 + dx) * 3 + c;
-                    unsigned v = p[c];
-                    if (raw128) v ^= 0x80u;                              // raw - 128 as int8
-                    wds[k >> 2] |= v << (8 * (k & 3));
+            if (ih < 0 || ih >= h || iw < 0 || iw >= w) continue;            // zero padding (iw is even: iw < 0 puts both pixels outside)
+            const uint8_t *p = in + (((size_t)img * h + ih) * w + iw) * 3;
+            if (iw + 1 < w && ((uintptr_t)p & 1) == 0) {
+                const unsigned short *q = (const unsigned short *)p;
+                hw[dy * 3] = (unsigned)__ldg(q) ^ flip;
+                hw[dy * 3 + 1] = (unsigned)__ldg(q + 1) ^ flip;
+                hw[dy * 3 + 2] = (unsigned)__ldg(q + 2) ^ flip;
+            } else {                          // rows of an odd width that start on an odd address, and their last pixel
+                const unsigned f = flip & 0xffu;
+                hw[dy * 3] = ((unsigned)p[0] ^ f) | (((unsigned)p[1] ^ f) << 8);
+                hw[dy * 3 + 1] = (unsigned)p[2] ^ f;
+                if (iw + 1 < w) {
+                    hw[dy * 3 + 1] |= ((unsigned)p[3] ^ f) << 8;
+                    hw[dy * 3 + 2] = ((unsigned)p[4] ^ f) | (((unsigned)p[5] ^ f) << 8);
                 }
             }
         }
-        *(uint4 *)(T + pos * 16) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
-        if (slack && pos == total - 1) *(uint4 *)(T + total * 16) = make_uint4(0, 0, 0, 0);   // the 16 bytes of slack behind T
+        *(uint4 *)(T + (size_t)pos * 16) = make_uint4(hw[0] | (hw[1] << 16), hw[2] | (hw[3] << 16), hw[4] | (hw[5] << 16), 0u);
+        if (slack && pos == total - 1) *(uint4 *)(T + (size_t)total * 16) = make_uint4(0, 0, 0, 0);   // the 16 bytes of slack behind T
     }
 }
 
@@ -210,6 +217,7 @@ int launch_stem(const iconv_plan_t *p, const ConvArgs &a, void *workspace, cudaS
     }
     const int hp = p->h_out + 3, wp = p->w_out + 3;
     const long long total = (long long)d.n * hp * wp;
+    if (total >= (1ll << 31)) { set_error("first-layer repack: more than 2^31 positions"); return ICONV_ERR_SHAPE; }
     long long blocks = (total + 255) / 256;
     if (blocks > 148ll * 32) blocks = 148ll * 32;
     stem_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t *)a.x, (uint8_t *)workspace, d.n, d.h, d.w,
