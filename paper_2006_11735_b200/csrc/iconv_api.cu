@@ -284,12 +284,13 @@ extern "C" int iconv_plan_describe(const iconv_plan_t *p, char *text, size_t siz
     }
     static const char *fam[] = {"auto", "direct", "umma", "thin", "stem", "umma"};
     if (p->kernel == ICONV_KERNEL_UMMA)
-        snprintf(text, size, "umma %s block_n=%d kc=%d stages=%d kg=%d resident_b=%d epi_warps=%d cs=%d bi=%d nbuf=%d epi=%d proj_iters=%d",
+        snprintf(text, size, "umma %s block_n=%d kc=%d stages=%d kg=%d resident_b=%d epi_warps=%d cs=%d bi=%d nbuf=%d epi=%d proj_iters=%d issuers=%d",
                  p->window ? (p->win_blocks ? "window(blocks)" : p->win_full_width ? "window(rows)" : "window(strips)") : p->pair ? "im2col(cta pairs)" : "im2col", p->block_n, p->kc,
                  p->window ? p->win_stages : p->stages, p->kg, p->window ? 1 : p->resident_b, p->epi_warps, p->cs, p->bi, p->window ? p->win_nbuf : p->nbuf, p->epi,
-                 p->proj_iters);
+                 p->proj_iters, p->window ? p->win_issuers : 1);
     else if (p->kernel == ICONV_KERNEL_STEM && p->inner)
-        snprintf(text, size, "stem -> umma block_n=%d kc=%d stages=%d kg=%d", p->inner->block_n, p->inner->kc, p->inner->stages, p->inner->kg);
+        snprintf(text, size, "stem -> umma block_n=%d kc=%d stages=%d kg=%d issuers=%d", p->inner->block_n, p->inner->kc,
+                 p->inner->window ? p->inner->win_stages : p->inner->stages, p->inner->kg, p->inner->window ? p->inner->win_issuers : 1);
     else
         snprintf(text, size, "%s", fam[p->kernel >= 0 && p->kernel <= 5 ? p->kernel : 0]);
     return ICONV_OK;

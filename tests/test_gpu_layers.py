@@ -618,4 +618,7 @@ def test_window_mode_with_many_tiles_per_cta_matches_oracle(shape):
     text = []
     got, fam = gpu_conv(X, W, b, mul, shift, h_i, pad=1, kernel=B.KERNEL_UMMA, describe=text)
     assert fam == B.KERNEL_UMMA and "window" in text[0] and expect in text[0], text
+    fields = dict(f.split("=") for f in text[0].split() if "=" in f)
+    stages, issuers, nbuf = int(fields["stages"]), int(fields["issuers"]), int(fields["nbuf"])
+    assert stages % issuers == 0 and (issuers == 2 or stages <= nbuf), text      # a stage's fills stay with one issuer
     assert np.array_equal(got, want)
