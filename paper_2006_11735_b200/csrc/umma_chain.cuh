@@ -86,6 +86,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int n_super = (int)blockIdx.x < c.m_tiles ? (c.m_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     const int T = n_super * c.n_tiles;                      // tiles of this CTA
 
+    if (threadIdx.x == 32) {
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w1);
+        prefetch_tensormap(&tmap_w2);
+        prefetch_tensormap(&tmap_out);
+        prefetch_tensormap(&tmap_skip);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < CHAIN_STAGES_MAX; ++s) {
             mbar_init(smem_u32(&sh->a1_full[s]), 1);

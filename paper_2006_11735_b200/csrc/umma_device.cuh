@@ -252,6 +252,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 // stream has completed and its writes are visible: every role executes it before it first touches
 // a tensor another kernel may have written (activations, skip); plan-owned constants may be read
 // before.  grid_dep_launch tells the scheduler that the kernel after this one may be scheduled.
+// Ask for a TMA descriptor ahead of its first use (the first copy otherwise waits for the descriptor fetch).
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -725,6 +730,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int lane = threadIdx.x & 31;
     const int num_tiles = u.m_tiles * u.n_tiles;
 
+    if (threadIdx.x == 32) {     // (a lane of a producer warp that has nothing else to do yet)
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
+        prefetch_tensormap(&tmap_out);
+        if (SKIP8 || EPI == EPI_PROJ) prefetch_tensormap(&tmap_skip);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < u.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), (uint32_t)u.kg);     // one arrival per slot
@@ -1243,6 +1254,10 @@ umma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const int lane = threadIdx.x & 31;
     const int num_tiles = u.m_tiles;
 
+    if (threadIdx.x == 32) {
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < u.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
