@@ -49,7 +49,7 @@ WORKLOADS = {"resnet50": ("ResNet-50 int8 images/sec", "resnet50_b256_224x224x3"
 # kernel's launches in one forward (two one-pass counters): {workload: (bytes per launch, kernel,
 # sha256 of the kernel's source the counters were taken on, that source file)}.  A changed kernel
 # reports null until the counters are taken again.
-DRAM_TRAFFIC = {"resnet50": (46223636, "umma_conv_kernel (cta pairs)", "4ff63ecf6612fdaa575e9364e14dd7dbbd288c4c227181ca8adec403bfc2828e",
+DRAM_TRAFFIC = {"resnet50": (46245691, "umma_conv_kernel (cta pairs)", "62e1eff8a847e6eaaa5fff8f3f2d34a89c64c72bed6fa101b64178549eee88af",
                              "umma_device.cuh")}
 NOMINAL_INT8_TOPS = 4500.0      # NVIDIA's dense INT8 figure for B200 (context only)
 INT8_OVER_BF16 = 2.0            # nominal dense ratio 4.5 / 2.25 PFLOP/s
